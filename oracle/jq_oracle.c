@@ -1,0 +1,272 @@
+/*
+ * jq_oracle.c -- slow, plain fp64 CPU definition of the Judge Q per-layer
+ * KV-cache eviction pass.  TEST INFRASTRUCTURE ONLY: it is the yardstick the
+ * CUDA library is compared with.  It shares no code, header, table or helper
+ * with the CUDA path, and only the tests, the smoke check and the CPU-baseline
+ * leg of the benchmark may call it.
+ *
+ * What it computes, with the passage of the paper each step follows:
+ *
+ *   score   Eq. 3 ("attention of every soft token with respect to the prompt,
+ *           combined over the token dimension") and the inference section
+ *           ("the attention map of the soft tokens over the input decides what
+ *           is kept"):  for KV head kv, for every query head h of its GQA
+ *           group and every soft token i,
+ *               s_j = (Q[h,i,:] . K[kv,j,:]) / sqrt(d)        j = 0..L-1
+ *               P_j = exp(s_j - max_j s) / sum_j exp(s_j - max_j s)
+ *               score[kv,j] += P_j
+ *           The softmax runs over the L prefix keys only; the sum (not the
+ *           1/n mean of Eq. 3) is taken, a monotone rescale that leaves the
+ *           kept set unchanged.
+ *   pool    Experimental-setting paragraph (all methods share one "pooling
+ *           configuration"): max over a centred window of odd width p, stride
+ *           1, same length, taps outside [0,L) ignored.
+ *   select  Inference section ("retain the pairs with the top-k highest
+ *           scores, discard the rest"): the nkeep = min(budget, L) largest
+ *           pooled values per KV head; equal values are ordered by lower
+ *           index first; the kept indices are returned ascending.
+ *   compact Inference section (the pruned cache is what decoding continues
+ *           with): rows K[kv,idx,:], V[kv,idx,:] copied bit for bit.
+ *
+ * Parity pins (tests/test_oracle_pins.py): softmax rows sum to 1; per-head
+ * score mass equals w*group; g=w=1 equals a library softmax; key-shift
+ * invariance; Q=0 and one-hot closed forms; pooling against an independent
+ * brute force and a library max_pool1d; selection against a library stable
+ * argsort; planted-mistake checks.  Fidelity to the paper's *trained* soft
+ * tokens (its benchmark tables) is parity unpinned: it needs the released
+ * embeddings, model weights and datasets.
+ *
+ * Inputs are bf16 bit patterns (uint16, the top half of an IEEE fp32).  All
+ * inputs must be finite.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double bf16_to_double(uint16_t b)
+{
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int jq_oracle_threads(int units)
+{
+#ifdef _OPENMP
+    int t = omp_get_max_threads();
+    return t < units ? t : units;
+#else
+    (void)units;
+    return 1;
+#endif
+}
+
+/*
+ * Eq. 3 on double inputs.  K [Hkv,L,d], Q [Hq,w,d], score [Hkv,L] (written).
+ * probs, when not NULL, receives every softmax row: [Hq,w,L].
+ * Returns 0, or 1 on bad arguments / allocation failure.
+ */
+int jq_oracle_score_f64(const double *K, const double *Q, int Hkv, int Hq, int L, int d, int w,
+                        double *score, double *probs)
+{
+    if (Hkv < 1 || Hq < 1 || L < 1 || d < 1 || w < 1 || Hq % Hkv != 0) return 1;
+    const int g = Hq / Hkv;
+    const double inv_sqrt_d = 1.0 / sqrt((double)d);
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int kv = 0; kv < Hkv; ++kv) {
+        double *e = (double *)malloc((size_t)L * sizeof(double));
+        if (!e) {
+#pragma omp atomic write
+            failed = 1;
+            continue;
+        }
+        double *sc = score + (size_t)kv * L;
+        for (int j = 0; j < L; ++j) sc[j] = 0.0;
+        for (int h = kv * g; h < kv * g + g; ++h) {
+            for (int i = 0; i < w; ++i) {
+                const double *q = Q + ((size_t)h * w + i) * d;
+                double m = -INFINITY;
+                for (int j = 0; j < L; ++j) {
+                    const double *k = K + ((size_t)kv * L + j) * d;
+                    double dot = 0.0;
+                    for (int c = 0; c < d; ++c) dot += q[c] * k[c];
+                    e[j] = dot * inv_sqrt_d;
+                    if (e[j] > m) m = e[j];
+                }
+                double l = 0.0;
+                for (int j = 0; j < L; ++j) {
+                    e[j] = exp(e[j] - m);
+                    l += e[j];
+                }
+                double *pr = probs ? probs + ((size_t)h * w + i) * L : NULL;
+                for (int j = 0; j < L; ++j) {
+                    double p = e[j] / l;
+                    sc[j] += p;
+                    if (pr) pr[j] = p;
+                }
+            }
+        }
+        free(e);
+    }
+    return failed;
+}
+
+/* Same, from bf16 bit patterns (converted exactly to double first). */
+int jq_oracle_score(const uint16_t *K, const uint16_t *Q, int Hkv, int Hq, int L, int d, int w,
+                    double *score, double *probs)
+{
+    if (Hkv < 1 || Hq < 1 || L < 1 || d < 1 || w < 1) return 1;
+    size_t nk = (size_t)Hkv * L * d, nq = (size_t)Hq * w * d;
+    double *Kd = (double *)malloc(nk * sizeof(double));
+    double *Qd = (double *)malloc(nq * sizeof(double));
+    if (!Kd || !Qd) {
+        free(Kd);
+        free(Qd);
+        return 1;
+    }
+    for (size_t t = 0; t < nk; ++t) Kd[t] = bf16_to_double(K[t]);
+    for (size_t t = 0; t < nq; ++t) Qd[t] = bf16_to_double(Q[t]);
+    int rc = jq_oracle_score_f64(Kd, Qd, Hkv, Hq, L, d, w, score, probs);
+    free(Kd);
+    free(Qd);
+    return rc;
+}
+
+/* Centred window max of odd width p; taps outside [0,L) are ignored. */
+int jq_oracle_pool(const double *score, int Hkv, int L, int p, double *pooled)
+{
+    if (Hkv < 1 || L < 1 || p < 1 || p % 2 == 0) return 1;
+    const int r = (p - 1) / 2;
+    for (int kv = 0; kv < Hkv; ++kv) {
+        const double *s = score + (size_t)kv * L;
+        double *o = pooled + (size_t)kv * L;
+        for (int j = 0; j < L; ++j) {
+            double best = s[j];
+            for (int t = -r; t <= r; ++t) {
+                int u = j + t;
+                if (u < 0 || u >= L) continue;
+                if (s[u] > best) best = s[u];
+            }
+            o[j] = best;
+        }
+    }
+    return 0;
+}
+
+typedef struct {
+    double v;
+    int32_t j;
+} jq_item;
+
+/* larger value first; among equal values the lower index first */
+static int cmp_rank(const void *a, const void *b)
+{
+    const jq_item *x = (const jq_item *)a, *y = (const jq_item *)b;
+    if (x->v > y->v) return -1;
+    if (x->v < y->v) return 1;
+    return (x->j > y->j) - (x->j < y->j);
+}
+
+static int cmp_i32(const void *a, const void *b)
+{
+    int32_t x = *(const int32_t *)a, y = *(const int32_t *)b;
+    return (x > y) - (x < y);
+}
+
+/* Full sort of every head's pooled values; idx [Hkv, min(budget,L)] ascending. */
+int jq_oracle_select(const double *pooled, int Hkv, int L, int budget, int32_t *idx)
+{
+    if (Hkv < 1 || L < 1 || budget < 1) return 1;
+    const int nkeep = budget < L ? budget : L;
+    jq_item *it = (jq_item *)malloc((size_t)L * sizeof(jq_item));
+    if (!it) return 1;
+    for (int kv = 0; kv < Hkv; ++kv) {
+        for (int j = 0; j < L; ++j) {
+            it[j].v = pooled[(size_t)kv * L + j];
+            it[j].j = j;
+        }
+        qsort(it, (size_t)L, sizeof(jq_item), cmp_rank);
+        int32_t *o = idx + (size_t)kv * nkeep;
+        for (int t = 0; t < nkeep; ++t) o[t] = it[t].j;
+        qsort(o, (size_t)nkeep, sizeof(int32_t), cmp_i32);
+    }
+    free(it);
+    return 0;
+}
+
+/*
+ * pool + select on caller-supplied fp32 scores (the stage-isolation entry the
+ * bit-exact tests use; float -> double is exact and max is exact, so the fp32
+ * pooled output is exact too).  pooled_out may be NULL.
+ */
+int jq_oracle_select_f32(const float *score, int Hkv, int L, int budget, int p, int32_t *idx,
+                         float *pooled_out)
+{
+    size_t n = (size_t)Hkv * L;
+    double *s = (double *)malloc(n * sizeof(double));
+    double *q = (double *)malloc(n * sizeof(double));
+    if (!s || !q) {
+        free(s);
+        free(q);
+        return 1;
+    }
+    for (size_t t = 0; t < n; ++t) s[t] = (double)score[t];
+    int rc = jq_oracle_pool(s, Hkv, L, p, q);
+    if (!rc) rc = jq_oracle_select(q, Hkv, L, budget, idx);
+    if (!rc && pooled_out)
+        for (size_t t = 0; t < n; ++t) pooled_out[t] = (float)q[t];
+    free(s);
+    free(q);
+    return rc;
+}
+
+/* Row gather, bit for bit.  K,V [Hkv,L,d]; idx [Hkv,nkeep]; out [Hkv,nkeep,d]. */
+int jq_oracle_compact(const uint16_t *K, const uint16_t *V, const int32_t *idx, int Hkv, int L,
+                      int d, int nkeep, uint16_t *Kout, uint16_t *Vout)
+{
+    if (Hkv < 1 || L < 1 || d < 1 || nkeep < 1 || nkeep > L) return 1;
+    for (int kv = 0; kv < Hkv; ++kv)
+        for (int t = 0; t < nkeep; ++t) {
+            int32_t j = idx[(size_t)kv * nkeep + t];
+            if (j < 0 || j >= L) return 1;
+            for (int c = 0; c < d; ++c) {
+                Kout[((size_t)kv * nkeep + t) * d + c] = K[((size_t)kv * L + j) * d + c];
+                Vout[((size_t)kv * nkeep + t) * d + c] = V[((size_t)kv * L + j) * d + c];
+            }
+        }
+    return 0;
+}
+
+/*
+ * The whole pass.  score_out / pooled_out ([Hkv,L] fp64) may be NULL.
+ */
+int jq_oracle_evict_layer(const uint16_t *K, const uint16_t *V, const uint16_t *Q, int Hkv, int Hq,
+                          int L, int d, int w, int budget, int p, uint16_t *Kout, uint16_t *Vout,
+                          int32_t *idx, double *score_out, double *pooled_out)
+{
+    if (Hkv < 1 || L < 1 || budget < 1) return 1;
+    size_t n = (size_t)Hkv * L;
+    const int nkeep = budget < L ? budget : L;
+    double *s = (double *)malloc(n * sizeof(double));
+    double *q = (double *)malloc(n * sizeof(double));
+    if (!s || !q) {
+        free(s);
+        free(q);
+        return 1;
+    }
+    int rc = jq_oracle_score(K, Q, Hkv, Hq, L, d, w, s, NULL);
+    if (!rc) rc = jq_oracle_pool(s, Hkv, L, p, q);
+    if (!rc) rc = jq_oracle_select(q, Hkv, L, budget, idx);
+    if (!rc) rc = jq_oracle_compact(K, V, idx, Hkv, L, d, nkeep, Kout, Vout);
+    if (!rc && score_out) memcpy(score_out, s, n * sizeof(double));
+    if (!rc && pooled_out) memcpy(pooled_out, q, n * sizeof(double));
+    free(s);
+    free(q);
+    return rc;
+}
