@@ -1,0 +1,325 @@
+"""Benchmark of the per-layer KV-cache eviction pass (prefix tokens evicted per second per layer).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg3|cfg2] [--budget B]
+    python bench.py --impl reference ...      # the fp64 CPU oracle, timed on the host cores
+
+One step = one pass of the whole hot path (scores -> pool -> top-k -> gather) over every layer of
+one synthetic cache: `layers` calls of jq_evict_layer on one stream.  Prints ONE JSON line.
+With N > 1 (torchrun) every rank evicts a cache of its own (independent replicas, no collective on
+the data path); the value is the sum over ranks divided by the slowest rank's time.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import jq_workloads as W  # noqa: E402
+
+METRIC = "prefix tokens evicted/sec per layer"
+UNIT = "tokens/s"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg5", choices=["cfg2", "cfg3", "cfg5"])
+    ap.add_argument("--budget", type=int, default=None)
+    ap.add_argument("--layers", type=int, default=None, help="layer calls per step (default: the workload's)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def pick_workload(args):
+    wl = {"cfg2": W.CFG2, "cfg3": W.CFG3, "cfg5": W.CFG5}[args.workload]
+    if args.workload == "cfg2":
+        wl = W.Workload(wl.name, 2, wl.Hkv, wl.Hq, wl.L, wl.w, wl.budget, layers=32, distinct_layers=32)
+    if args.budget:
+        wl = wl.with_budget(args.budget)
+    return wl
+
+
+def config_of(wl, layers, distinct):
+    return {"workload": wl.name, "L": wl.L, "Hkv": wl.Hkv, "Hq": wl.Hq, "d": wl.d, "w": wl.w,
+            "budget": wl.budget, "pool": wl.pool, "layers_per_step": layers, "distinct_layers": distinct,
+            "l2": "inputs larger than L2 (K of one step: %.0f MiB)" % (distinct * wl.Hkv * wl.L * wl.d * 2 / 2**20)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_time_heads(wl, K, V, Q, heads):
+    """Seconds the oracle takes for the whole pass restricted to the given KV heads (independent units)."""
+    import oracle
+    g = wl.group
+    qrows = np.concatenate([np.arange(kv * g, kv * g + g) for kv in heads])
+    Ks, Vs, Qs = np.ascontiguousarray(K[heads]), np.ascontiguousarray(V[heads]), np.ascontiguousarray(Q[qrows])
+    t0 = time.perf_counter()
+    oracle.evict_layer(Ks, Vs, Qs, wl.budget, wl.pool)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(wl, K, V, Q, max_heads=None):
+    import oracle
+    cores = os.cpu_count() or 1
+    n = min(wl.Hkv, cores if max_heads is None else max_heads)
+    heads = list(range(n))
+    sec = oracle_time_heads(wl, K, V, Q, heads)
+    t_layer = sec * wl.Hkv / n
+    return {"value": wl.L / t_layer, "unit": UNIT, "cores": oracle.threads(n), "kind": "oracle",
+            "sample": "%d of %d KV heads of one layer at full L=%d (heads are independent); %.2f s measured, "
+                      "scaled to a layer; gcc -O2 -fopenmp, fp64" % (n, wl.Hkv, wl.L, sec),
+            "seconds_per_layer": t_layer}
+
+
+def run_reference(args):
+    """The reference arm: the fp64 oracle as it stands, on the host cores, rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    wl = pick_workload(args)
+    K, V, Q, _ = W.make_layer(wl, 0)
+    cores = os.cpu_count() or 1
+    # calibrate on a short prefix of one head, then size the per-step sample for a run of a few minutes
+    Lc = max(wl.L // 16, 256)
+    wc = wl.with_L(Lc)
+    tc = oracle_time_heads(wc, K[:, :Lc], V[:, :Lc], Q, [0])
+    per_head = tc * wl.L / Lc
+    total = args.steps + args.warmup
+    n = max(1, min(wl.Hkv, cores))            # heads run in parallel: a step takes about one head's time
+    Ls = wl.L
+    if total * per_head > 150.0:
+        Ls = max(2048, int(wl.L * 150.0 / (total * per_head)) // 128 * 128)
+    ws = wl.with_L(Ls)
+    Ks, Vs = np.ascontiguousarray(K[:, :Ls]), np.ascontiguousarray(V[:, :Ls])
+    heads = list(range(n))
+    for _ in range(args.warmup):
+        oracle_time_heads(ws, Ks, Vs, Q, heads)
+    t = [oracle_time_heads(ws, Ks, Vs, Q, heads) for _ in range(args.steps)]
+    sec = float(np.mean(t))
+    t_layer = sec * (wl.Hkv / n) * (wl.L / Ls)
+    value = wl.L / t_layer
+    sample = "%d of %d KV heads, first %d of %d keys, per step; scaled linearly to a full layer" % (n, wl.Hkv, Ls, wl.L)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_of(wl, 1, 1),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(n), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- GPU arm
+
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.f.read().strip().splitlines():
+            c = [x.strip() for x in ln.split(",")]
+            if len(c) < 7:
+                continue
+            try:
+                sm.append(float(c[0])); mx.append(float(c[1])); pw.append(float(c[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, c[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), power_w_max=float(max(pw)),
+                       reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2509_10798_b200 as jq
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    jq.lib()                                   # fails loudly if the CUDA library is not built
+
+    wl = pick_workload(args)
+    layers = args.layers or wl.layers
+    distinct = min(wl.distinct_layers, layers)
+    s = jq.shape(wl.Hkv, wl.Hq, wl.L, wl.w, wl.budget, wl.pool, wl.d)
+    nkeep = wl.nkeep
+
+    def dev(bits):
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    host0 = None
+    Ks, Vs, Qs = [], [], []
+    for i in range(distinct):
+        K, V, Q, _ = W.make_layer(wl, layer=i, seq=rank)
+        if i == 0:
+            host0 = (K, V, Q)
+        Ks.append(dev(K)); Vs.append(dev(V)); Qs.append(dev(Q))
+    ws = jq.new_workspace(s)
+    Ko = torch.zeros((wl.Hkv, nkeep, wl.d), dtype=torch.bfloat16, device="cuda")
+    Vo = torch.zeros_like(Ko)
+    idx = torch.zeros((wl.Hkv, nkeep), dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        for i in range(layers):
+            j = i % distinct
+            jq.evict_layer(Ks[j], Vs[j], Qs[j], s, Ko, Vo, idx, ws, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    n0 = jq.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = jq.launch_count() - n0
+    assert jq.last_device_status(ws) == jq.JQ_OK, "device status not ok"
+
+    # per-stage times through the stage entry points (events on the launching stream)
+    scores = torch.empty((wl.Hkv, wl.L), dtype=torch.float32, device="cuda")
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    stage_ms = np.zeros(3)
+    reps = max(args.steps, 5) * min(layers, 8)
+    for rep in range(reps + 3):
+        j = rep % distinct
+        ev[0].record(stream)
+        jq.score(Ks[j], Qs[j], s, scores, ws, stream=stream)
+        ev[1].record(stream)
+        jq.select_topk(scores, s, idx, ws, stream=stream)
+        ev[2].record(stream)
+        jq.compact_kv(Ks[j], Vs[j], idx, s, Ko, Vo, stream=stream)
+        ev[3].record(stream)
+        torch.cuda.synchronize()
+        if rep >= 3:
+            stage_ms += [ev[k].elapsed_time(ev[k + 1]) for k in range(3)]
+    stage_ms /= reps
+    clocks = sampler.stop() if sampler else None
+
+    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    t_layer = ms * 1e-3 / (args.steps * layers)
+    value = world * wl.L / t_layer
+
+    # end to end through the host-buffer entry point: pinned host tensors in, pinned host results out
+    e2e = None
+    if not args.no_e2e:
+        pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
+        hK, hV, hQ = (pin(a) for a in host0)
+        hKo = torch.zeros((wl.Hkv, nkeep, wl.d), dtype=torch.int16).pin_memory()
+        hVo = torch.zeros_like(hKo).pin_memory()
+        hidx = torch.zeros((wl.Hkv, nkeep), dtype=torch.int32).pin_memory()
+        buf = torch.empty(jq.host_call_bytes(s), dtype=torch.uint8, device="cuda")
+        e2e_layers = 2
+        n_e2e = max(3, min(args.steps, 10))
+        for _ in range(2):
+            jq.evict_layer_host(hK, hV, hQ, s, hKo, hVo, hidx, buf, stream=stream)
+        barrier()
+        e0.record(stream)
+        for _ in range(n_e2e * e2e_layers):
+            jq.evict_layer_host(hK, hV, hQ, s, hKo, hVo, hidx, buf, stream=stream)
+        e1.record(stream)
+        barrier()
+        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t_e2e_layer = float(t.item()) * 1e-3 / (n_e2e * e2e_layers)
+        h2d = e2e_layers * (2 * hK.numel() + hQ.numel()) * 2
+        d2h = e2e_layers * (2 * hKo.numel() * 2 + hidx.numel() * 4)
+        e2e = {"value": world * wl.L / t_e2e_layer, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "layers_per_step": e2e_layers, "ms_per_layer": t_e2e_layer * 1e3}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        with open(peaks_path) as f:
+            peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = 6650.0, "fallback"
+    # dominant stage: the two scoring passes (jq_score); algorithmic bytes = two reads of K
+    score_bytes = 2 * wl.Hkv * wl.L * wl.d * 2
+    achieved = score_bytes / (stage_ms[0] * 1e-3) / 1e9
+    layer_gbs = W.formula_bytes(wl) / t_layer / 1e9
+    roofline = {"bound": "hbm", "kernel": "jq_score (pass 1 + pass 2)", "achieved": achieved, "peak": peak,
+                "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                "bytes_per_launch": score_bytes, "ms_per_launch": float(stage_ms[0]),
+                "layer_formula_gbs": layer_gbs, "layer_frac_of_peak": layer_gbs / peak,
+                "layer_frac_of_8tbs": layer_gbs / 8000.0,
+                "stage_ms": {"score": float(stage_ms[0]), "select": float(stage_ms[1]), "compact": float(stage_ms[2])}}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
+            "config": config_of(wl, layers, distinct), "ms_per_layer": t_layer * 1e3,
+            "tokens_discarded_per_s": world * (wl.L - nkeep) / t_layer,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline}
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(wl, *host0)
+    if world > 1:
+        dist.destroy_process_group()
+    print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    a = parse()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

@@ -1,0 +1,153 @@
+/*
+ * jq.h -- C ABI of the B200 (sm_100a) library for the per-layer KV-cache eviction pass of
+ * "Judge Q" (arXiv 2509.10798).
+ *
+ * The pass (inference section of the paper; Eq. 3 defines the attention map it uses): the queries
+ * of the w soft tokens appended to the prompt score every prefix key of one layer,
+ *     s[h,i,j]   = Qwin[h,i,:] . K[h/group, j, :] / sqrt(d)
+ *     P[h,i,:]   = softmax over the L prefix keys of s[h,i,:]
+ *     score[kv,j]= sum over the `group` query heads of KV head kv and the w soft tokens of P[h,i,j]
+ *     pooled     = centred max of odd width `pool` over the key axis (same length, edges clipped)
+ * the min(budget, L) positions with the largest pooled score are kept per KV head (equal values:
+ * the lower index wins), reported in ascending order, and their K and V rows are copied into a
+ * compacted cache.
+ *
+ * Conventions, for every entry point unless it says otherwise:
+ *  - pointers named K, V, Qwin, scores, kept_idx, Kout, Vout, ws are DEVICE pointers owned by the
+ *    caller, contiguous row-major, 16-byte aligned; the library allocates and frees nothing;
+ *  - bf16 tensors are raw 16-bit patterns:  K, V [Hkv, L, d];  Qwin [Hq, w, d];
+ *    Kout, Vout [Hkv, nkeep, d];  scores, pooled [Hkv, L] fp32;  kept_idx [Hkv, nkeep] int32,
+ *    nkeep = jq_num_kept(shape) = min(budget, L);
+ *  - all work is enqueued on `stream` (a cudaStream_t); the call returns without synchronising;
+ *    outputs are valid once the stream reaches the end of the call's work;
+ *  - outputs must not overlap inputs or the workspace; the same workspace may be reused by
+ *    successive calls on ONE stream; calls on different streams need different workspaces;
+ *  - inputs must be finite; NaN or Inf give unspecified kept sets (never a fault);
+ *  - errors are return codes; argument errors are detected on the host before anything is
+ *    launched and leave every output untouched.
+ *
+ * Supported shapes: d == 128;  Hq == Hkv * group;  1 <= group * w <= 256;  pool odd, 1..63;
+ * budget >= 1;  1 <= L <= 2^24;  Hkv >= 1.
+ */
+#ifndef JQ_H_
+#define JQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    JQ_OK = 0,
+    JQ_ERR_INVALID_ARG = 1, /* null or misaligned pointer, inconsistent shape                 */
+    JQ_ERR_UNSUPPORTED = 2, /* a legal shape this build has no kernel for (d != 128, ...)      */
+    JQ_ERR_WORKSPACE = 3,   /* ws_bytes < jq_workspace_bytes(shape)                            */
+    JQ_ERR_CUDA = 4,        /* a CUDA runtime / driver call or a launch failed                 */
+    JQ_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (see jq_last_device_status)  */
+} jq_status;
+
+typedef struct {
+    int Hkv;    /* KV heads                                             */
+    int Hq;     /* query heads, = Hkv * group                           */
+    int group;  /* GQA group size: query head h reads KV head h / group */
+    int L;      /* prefix length (keys per KV head)                     */
+    int d;      /* head dimension (128)                                 */
+    int w;      /* soft-token queries per query head (the paper's n)    */
+    int budget; /* positions to keep per KV head                        */
+    int pool;   /* max-pool width (odd); 1 = no pooling                 */
+} jq_shape;
+
+/* A cudaStream_t, spelled so that this header needs no CUDA header. */
+typedef struct CUstream_st *jq_stream_t;
+
+/* Bytes of device workspace every call below needs for this shape (host-only, no CUDA call);
+ * 0 if the shape is invalid or unsupported. */
+size_t jq_workspace_bytes(const jq_shape *shape);
+
+/*
+ * Zeroes the status word at the head of a workspace.  Call once after allocating `ws` and before
+ * its first use (on the stream that will use it); the status then accumulates over all later calls
+ * until it is read with jq_last_device_status or cleared by calling this again.
+ */
+jq_status jq_workspace_init(void *ws, size_t ws_bytes, jq_stream_t stream);
+
+/* min(budget, L); 0 for an invalid shape. */
+int jq_num_kept(const jq_shape *shape);
+
+/* Why a shape is (not) accepted: JQ_OK, JQ_ERR_INVALID_ARG or JQ_ERR_UNSUPPORTED (host-only). */
+jq_status jq_check_shape(const jq_shape *shape);
+
+/*
+ * Eq. 3 (summed, not averaged, over the soft tokens and over the GQA group): pre-pool scores.
+ * Two streaming passes over K on the tensor cores: pass 1 finds each query row's running max
+ * and sum of exponentials, pass 2 recomputes the logits and accumulates the normalised
+ * probabilities per key (fp32 accumulation of bf16 products).
+ *   K [Hkv,L,d] bf16, Qwin [Hq,w,d] bf16  ->  scores [Hkv,L] fp32.
+ */
+jq_status jq_score(const void *K, const void *Qwin, const jq_shape *shape, float *scores,
+                   void *ws, size_t ws_bytes, jq_stream_t stream);
+
+/*
+ * The same scores computed with plain fp32 FMA on the CUDA cores.  A comparator for profiling the
+ * tensor-core path against (the contraction is small and of low arithmetic intensity per key);
+ * never used by jq_evict_layer.
+ */
+jq_status jq_score_fma(const void *K, const void *Qwin, const jq_shape *shape, float *scores,
+                       void *ws, size_t ws_bytes, jq_stream_t stream);
+
+/*
+ * Max-pool (experimental setting: every method shares one pooling configuration) followed by the
+ * top-k retention of the inference section.  scores [Hkv,L] fp32, all >= 0.
+ *   -> kept_idx [Hkv,nkeep] int32 ascending; ties at the threshold go to the lower index.
+ *   pooled_or_null, if not NULL, receives the pooled scores [Hkv,L] fp32.
+ * Exact: with identical input scores the result is unique.
+ */
+jq_status jq_select_topk(const float *scores, const jq_shape *shape, int32_t *kept_idx,
+                         float *pooled_or_null, void *ws, size_t ws_bytes, jq_stream_t stream);
+
+/*
+ * Compaction of the pruned cache (inference section): Kout[kv,t,:] = K[kv, kept_idx[kv,t], :] and
+ * the same for V, bit for bit.  An index outside [0,L) is clamped into range (never a fault); such
+ * an index cannot come from jq_select_topk.
+ */
+jq_status jq_compact_kv(const void *K, const void *V, const int32_t *kept_idx,
+                        const jq_shape *shape, void *Kout, void *Vout, jq_stream_t stream);
+
+/*
+ * The whole pass for one layer: jq_score -> jq_select_topk -> jq_compact_kv on one stream, with
+ * the scores kept in the workspace.
+ */
+jq_status jq_evict_layer(const void *K, const void *V, const void *Qwin, const jq_shape *shape,
+                         void *Kout, void *Vout, int32_t *kept_idx, void *ws, size_t ws_bytes,
+                         jq_stream_t stream);
+
+/*
+ * jq_evict_layer for callers whose tensors live in HOST memory (pinned memory gives asynchronous
+ * copies).  hK, hV, hQwin are copied to the device, the layer is evicted, and hKout, hVout,
+ * hkept_idx are copied back, all on `stream`; the call returns without synchronising.
+ * dev_buf is a device buffer of at least jq_host_call_bytes(shape) bytes (it holds the device
+ * copies and the workspace).
+ */
+size_t jq_host_call_bytes(const jq_shape *shape);
+jq_status jq_evict_layer_host(const void *hK, const void *hV, const void *hQwin,
+                              const jq_shape *shape, void *hKout, void *hVout, int32_t *hkept_idx,
+                              void *dev_buf, size_t dev_buf_bytes, jq_stream_t stream);
+
+/*
+ * Synchronises `stream` and reads the status word kernels of earlier calls left in the workspace:
+ * JQ_OK, JQ_ERR_TIMEOUT (a bounded wait inside a kernel gave up; outputs are invalid),
+ * JQ_ERR_INVALID_ARG (an out-of-range index was met), or JQ_ERR_CUDA.
+ */
+jq_status jq_last_device_status(const void *ws, jq_stream_t stream);
+
+/* Number of kernels the library has launched in this process (for benchmarks' launch counts). */
+unsigned long long jq_launch_count(void);
+
+const char *jq_status_string(jq_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JQ_H_ */

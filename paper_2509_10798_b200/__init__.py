@@ -1,0 +1,164 @@
+"""B200 (sm_100a) library for the per-layer KV-cache eviction pass of Judge Q (arXiv 2509.10798).
+
+Thin ctypes binding over libjq.so (C ABI in include/jq.h).  The functions here only marshal
+arguments: torch tensors supply device memory and the current CUDA stream, every step of the pass
+runs in the library's own kernels.  There is no CPU or PyTorch fallback: if libjq.so is missing or
+no CUDA device is present, the calls raise.
+"""
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libjq.so")
+
+JQ_OK, JQ_ERR_INVALID_ARG, JQ_ERR_UNSUPPORTED, JQ_ERR_WORKSPACE, JQ_ERR_CUDA, JQ_ERR_TIMEOUT = range(6)
+
+EXPORTS = (
+    "jq_workspace_bytes", "jq_workspace_init", "jq_num_kept", "jq_check_shape", "jq_score",
+    "jq_score_fma", "jq_select_topk", "jq_compact_kv", "jq_evict_layer", "jq_host_call_bytes",
+    "jq_evict_layer_host", "jq_last_device_status", "jq_launch_count", "jq_status_string",
+)
+
+
+class JqShape(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("Hkv", "Hq", "group", "L", "d", "w", "budget", "pool")]
+
+
+class JqError(RuntimeError):
+    def __init__(self, where, code):
+        self.code = int(code)
+        super().__init__("%s: %s (jq_status %d)" % (where, status_string(code), code))
+
+
+_lib = None
+
+
+def lib():
+    """Loads libjq.so (never builds it; see build.py) and declares the prototypes."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libjq.so is not built: run `python -m paper_2509_10798_b200.build` "
+                               "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, ci = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+        sp = ctypes.POINTER(JqShape)
+        L.jq_workspace_bytes.argtypes = [sp]
+        L.jq_workspace_bytes.restype = sz
+        L.jq_host_call_bytes.argtypes = [sp]
+        L.jq_host_call_bytes.restype = sz
+        L.jq_num_kept.argtypes = [sp]
+        L.jq_num_kept.restype = ci
+        L.jq_check_shape.argtypes = [sp]
+        L.jq_check_shape.restype = ci
+        L.jq_workspace_init.argtypes = [vp, sz, vp]
+        L.jq_score.argtypes = [vp, vp, sp, vp, vp, sz, vp]
+        L.jq_score_fma.argtypes = [vp, vp, sp, vp, vp, sz, vp]
+        L.jq_select_topk.argtypes = [vp, sp, vp, vp, vp, sz, vp]
+        L.jq_compact_kv.argtypes = [vp, vp, vp, sp, vp, vp, vp]
+        L.jq_evict_layer.argtypes = [vp, vp, vp, sp, vp, vp, vp, vp, sz, vp]
+        L.jq_evict_layer_host.argtypes = [vp, vp, vp, sp, vp, vp, vp, vp, sz, vp]
+        L.jq_last_device_status.argtypes = [vp, vp]
+        L.jq_launch_count.argtypes = []
+        L.jq_launch_count.restype = ctypes.c_ulonglong
+        L.jq_status_string.argtypes = [ci]
+        L.jq_status_string.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            getattr(L, name)          # AttributeError if the library lacks a declared entry point
+        _lib = L
+    return _lib
+
+
+def status_string(code):
+    return lib().jq_status_string(int(code)).decode()
+
+
+def shape(Hkv, Hq, L, w, budget, pool=7, d=128, group=None):
+    return JqShape(int(Hkv), int(Hq), int(Hq // Hkv if group is None else group), int(L), int(d), int(w),
+                   int(budget), int(pool))
+
+
+def check_shape(s):
+    return int(lib().jq_check_shape(ctypes.byref(s)))
+
+
+def workspace_bytes(s):
+    return int(lib().jq_workspace_bytes(ctypes.byref(s)))
+
+
+def host_call_bytes(s):
+    return int(lib().jq_host_call_bytes(ctypes.byref(s)))
+
+
+def num_kept(s):
+    return int(lib().jq_num_kept(ctypes.byref(s)))
+
+
+def launch_count():
+    return int(lib().jq_launch_count())
+
+
+def _torch():
+    import torch
+    if not torch.cuda.is_available():
+        raise RuntimeError("paper_2509_10798_b200 needs a CUDA device; there is no CPU path")
+    return torch
+
+
+def _stream(stream):
+    if stream is None:
+        stream = _torch().cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _raise(where, rc):
+    if rc != JQ_OK:
+        raise JqError(where, rc)
+
+
+def new_workspace(s, device="cuda", stream=None):
+    """Allocates and initialises a workspace tensor (uint8) for shape `s`."""
+    torch = _torch()
+    n = workspace_bytes(s)
+    if n == 0:
+        raise JqError("jq_workspace_bytes", check_shape(s) or JQ_ERR_INVALID_ARG)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    _raise("jq_workspace_init", lib().jq_workspace_init(_ptr(ws), n, _stream(stream)))
+    return ws
+
+
+def score(K, Qwin, s, scores, ws, stream=None, fma=False):
+    fn = lib().jq_score_fma if fma else lib().jq_score
+    _raise("jq_score_fma" if fma else "jq_score",
+           fn(_ptr(K), _ptr(Qwin), ctypes.byref(s), _ptr(scores), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def select_topk(scores, s, kept_idx, ws, pooled=None, stream=None):
+    _raise("jq_select_topk", lib().jq_select_topk(_ptr(scores), ctypes.byref(s), _ptr(kept_idx), _ptr(pooled),
+                                                  _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def compact_kv(K, V, kept_idx, s, Kout, Vout, stream=None):
+    _raise("jq_compact_kv", lib().jq_compact_kv(_ptr(K), _ptr(V), _ptr(kept_idx), ctypes.byref(s), _ptr(Kout),
+                                                _ptr(Vout), _stream(stream)))
+
+
+def evict_layer(K, V, Qwin, s, Kout, Vout, kept_idx, ws, stream=None):
+    _raise("jq_evict_layer", lib().jq_evict_layer(_ptr(K), _ptr(V), _ptr(Qwin), ctypes.byref(s), _ptr(Kout),
+                                                  _ptr(Vout), _ptr(kept_idx), _ptr(ws), ws.numel(),
+                                                  _stream(stream)))
+
+
+def evict_layer_host(hK, hV, hQwin, s, hKout, hVout, hkept_idx, dev_buf, stream=None):
+    """Host-tensor variant: all h* are CPU tensors (pinned for asynchronous copies)."""
+    _raise("jq_evict_layer_host",
+           lib().jq_evict_layer_host(_ptr(hK), _ptr(hV), _ptr(hQwin), ctypes.byref(s), _ptr(hKout), _ptr(hVout),
+                                     _ptr(hkept_idx), _ptr(dev_buf), dev_buf.numel(), _stream(stream)))
+
+
+def last_device_status(ws, stream=None):
+    return int(lib().jq_last_device_status(_ptr(ws), _stream(stream)))

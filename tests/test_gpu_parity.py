@@ -1,0 +1,229 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU oracle, element by element.
+
+Agreement rules: integer / byte / index work is bit-exact when fed identical scores; pre-pool and
+pooled scores agree within 2e-3 relative + 1e-6 absolute (fp32 accumulation of bf16 products);
+end to end, kept sets may differ only at positions whose oracle pooled score lies within 1e-4
+relative of the k-th pooled score.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import jq_workloads as W
+import paper_2509_10798_b200 as jq
+from gpu_util import (assert_kept_sets_agree, assert_scores_close, dev_bf16, gpu_evict, gpu_score,
+                      gpu_select, host_bits, shape_of)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    import __graft_entry__ as entry
+    entry.build()
+
+
+def small_wl(Hkv, g, w, L, budget, pool=7, config=2):
+    return W.Workload("t", config, Hkv=Hkv, Hq=Hkv * g, L=L, w=w, budget=budget, pool=pool)
+
+
+# ------------------------------------------------------------------ scores (steps 1-3)
+
+SCORE_CASES = [
+    # Hkv, g, w, L : tiles of 128 keys -> below one tile, exact tiles, ragged tails, several tiles
+    (1, 1, 1, 1), (1, 1, 1, 7), (2, 1, 3, 8), (1, 2, 5, 127), (2, 4, 16, 128), (2, 4, 16, 129),
+    (3, 4, 32, 300), (2, 4, 32, 1000), (1, 4, 64, 777), (2, 4, 64, 2049), (8, 4, 32, 1536),
+    (2, 8, 32, 515), (1, 3, 11, 4000),
+]
+
+
+@pytest.mark.parametrize("fma", [False, True], ids=["tensor", "fma"])
+@pytest.mark.parametrize("Hkv,g,w,L", SCORE_CASES)
+def test_score_small_shapes(Hkv, g, w, L, fma):
+    wl = small_wl(Hkv, g, w, L, 1)
+    K, _, Q, _ = W.make_layer(wl, with_v=False)
+    want = oracle.score(K, Q)
+    got = gpu_score(K, Q, shape_of(wl), fma=fma)
+    assert_scores_close(got, want)
+    np.testing.assert_allclose(got.sum(-1), wl.R, rtol=1e-3)
+
+
+@pytest.mark.parametrize("fma", [False, True], ids=["tensor", "fma"])
+@pytest.mark.parametrize("wl", [W.CFG1, W.CFG2, W.CFG4[1].with_L(3000)], ids=lambda w: w.name)
+def test_score_configs(wl, fma):
+    K, _, Q, _ = W.make_layer(wl, with_v=False)
+    assert_scores_close(gpu_score(K, Q, shape_of(wl), fma=fma), oracle.score(K, Q))
+
+
+def test_score_zero_queries_is_uniform():
+    wl = small_wl(2, 4, 16, 999, 1)
+    K, _, Q, _ = W.make_layer(wl, with_v=False)
+    got = gpu_score(K, np.zeros_like(Q), shape_of(wl))
+    np.testing.assert_allclose(got, wl.R / wl.L, rtol=1e-5)
+
+
+def test_score_large_logits_do_not_overflow():
+    """Strongly peaked rows (logit range of several hundred) must stay finite and normalised."""
+    wl = small_wl(1, 2, 8, 640, 1)
+    K, _, Q, _ = W.make_layer(wl, with_v=False)
+    Qs = W.bf16_bits(W.bf16_to_f32(Q) * 24.0)
+    got = gpu_score(K, Qs, shape_of(wl))
+    assert np.all(np.isfinite(got))
+    assert_scores_close(got, oracle.score(K, Qs))
+
+
+# ------------------------------------------------------------------ pool + select (steps 4-5), bit-exact
+
+SELECT_CASES = [(1, 1, 1, 7), (1, 5, 9, 7), (2, 6, 3, 7), (2, 64, 64, 7), (3, 257, 40, 7), (2, 1000, 333, 3),
+                (2, 4096, 1024, 7), (1, 5000, 4999, 9), (2, 33000, 2048, 7), (1, 70001, 4096, 1),
+                (8, 8192, 1024, 7)]
+
+
+@pytest.mark.parametrize("Hkv,L,B,p", SELECT_CASES)
+@pytest.mark.parametrize("kind", ["random", "ties", "oracle_scores"])
+def test_select_bit_exact(Hkv, L, B, p, kind):
+    rng = np.random.default_rng(L * 31 + B)
+    if kind == "random":
+        s32 = rng.random((Hkv, L), dtype=np.float32)
+    elif kind == "ties":
+        s32 = (rng.integers(0, 5, size=(Hkv, L)) / 4.0).astype(np.float32)
+    else:
+        wl = small_wl(Hkv, 2, 4, L, B, p)
+        K, _, Q, _ = W.make_layer(wl, with_v=False)
+        s32 = oracle.score(K, Q).astype(np.float32)
+    want_idx, want_pooled = oracle.select_f32(s32, B, p)
+    s = jq.shape(Hkv, Hkv, L, 1, B, p)
+    got_idx, got_pooled = gpu_select(s32, s)
+    assert np.array_equal(got_pooled.view(np.uint32), want_pooled.view(np.uint32))
+    assert np.array_equal(got_idx, want_idx)
+
+
+def test_select_all_equal_keeps_lowest_indices():
+    s32 = np.full((2, 5000), 0.25, np.float32)
+    idx, _ = gpu_select(s32, jq.shape(2, 2, 5000, 1, 777, 7))
+    assert np.array_equal(idx, np.tile(np.arange(777, dtype=np.int32), (2, 1)))
+
+
+# ------------------------------------------------------------------ compaction (step 6), bit-exact
+
+@pytest.mark.parametrize("Hkv,L,n", [(1, 1, 1), (2, 100, 7), (8, 4096, 1024), (3, 5000, 4999)])
+def test_compact_bit_exact(Hkv, L, n):
+    rng = np.random.default_rng(L + n)
+    K = rng.integers(0, 65536, size=(Hkv, L, 128), dtype=np.uint16)
+    V = rng.integers(0, 65536, size=(Hkv, L, 128), dtype=np.uint16)
+    idx = np.stack([np.sort(rng.choice(L, size=n, replace=False)) for _ in range(Hkv)]).astype(np.int32)
+    s = jq.shape(Hkv, Hkv, L, 1, n, 7)
+    Ko = torch.zeros((Hkv, n, 128), dtype=torch.bfloat16, device="cuda")
+    Vo = torch.zeros_like(Ko)
+    jq.compact_kv(dev_bf16(K), dev_bf16(V), torch.from_numpy(idx).cuda(), s, Ko, Vo)
+    wK, wV = oracle.compact(K, V, idx)
+    assert np.array_equal(host_bits(Ko), wK) and np.array_equal(host_bits(Vo), wV)
+
+
+# ------------------------------------------------------------------ whole pass
+
+def run_e2e(wl, K, V, Q, pooled=None):
+    s = shape_of(wl)
+    gKo, gVo, gidx = gpu_evict(K, V, Q, s)
+    if pooled is None:
+        pooled = oracle.pool(oracle.score(K, Q), wl.pool)
+    oidx = oracle.select(pooled, wl.budget)
+    swaps = assert_kept_sets_agree(gidx, oidx, pooled, wl.nkeep)
+    for kv in range(wl.Hkv):           # gathered bytes are exactly the rows the GPU chose
+        assert np.array_equal(gKo[kv], K[kv][gidx[kv]]) and np.array_equal(gVo[kv], V[kv][gidx[kv]])
+    if swaps == 0:
+        oKo, oVo = oracle.compact(K, V, oidx)
+        assert np.array_equal(gKo, oKo) and np.array_equal(gVo, oVo)
+    return swaps
+
+
+@pytest.mark.parametrize("wl", [W.CFG1, W.CFG2, W.CFG2.with_budget(100000), W.CFG4[0], W.CFG4[1],
+                                small_wl(2, 4, 16, 5, 3), small_wl(1, 4, 64, 1, 1)],
+                         ids=lambda w: "%s-L%d-B%d" % (w.name, w.L, w.budget))
+def test_evict_layer_end_to_end(wl):
+    K, V, Q, _ = W.make_layer(wl)
+    run_e2e(wl, K, V, Q)
+
+
+def test_evict_layer_zero_queries_ties_everywhere():
+    wl = small_wl(2, 4, 16, 3000, 500)
+    K, V, Q, _ = W.make_layer(wl)
+    _, _, gidx = gpu_evict(K, V, np.zeros_like(Q), shape_of(wl))
+    # all scores tie (up to fp32 noise the oracle rule tolerates); the structure must still be valid
+    assert gidx.shape == (2, 500) and np.all(np.diff(gidx, axis=1) > 0)
+
+
+def test_evict_layer_is_deterministic_and_workspace_reusable():
+    wl = W.CFG2.with_L(5000)
+    K, V, Q, _ = W.make_layer(wl)
+    s = shape_of(wl)
+    ws = jq.new_workspace(s)
+    dK, dV, dQ = dev_bf16(K), dev_bf16(V), dev_bf16(Q)
+    outs = []
+    for _ in range(3):
+        Ko = torch.zeros((s.Hkv, wl.nkeep, s.d), dtype=torch.bfloat16, device="cuda")
+        Vo = torch.zeros_like(Ko)
+        idx = torch.zeros((s.Hkv, wl.nkeep), dtype=torch.int32, device="cuda")
+        jq.evict_layer(dK, dV, dQ, s, Ko, Vo, idx, ws)
+        outs.append((host_bits(Ko), host_bits(Vo), idx.cpu().numpy()))
+    assert jq.last_device_status(ws) == jq.JQ_OK
+    for o in outs[1:]:
+        for a, b in zip(outs[0], o):
+            assert np.array_equal(a, b)
+
+
+def test_host_entry_matches_device_entry():
+    wl = W.CFG2.with_L(3000)
+    K, V, Q, _ = W.make_layer(wl)
+    s = shape_of(wl)
+    gKo, gVo, gidx = gpu_evict(K, V, Q, s)
+    pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
+    hK, hV, hQ = pin(K), pin(V), pin(Q)
+    hKo = torch.zeros((s.Hkv, wl.nkeep, s.d), dtype=torch.int16).pin_memory()
+    hVo = torch.zeros_like(hKo).pin_memory()
+    hidx = torch.zeros((s.Hkv, wl.nkeep), dtype=torch.int32).pin_memory()
+    buf = torch.empty(jq.host_call_bytes(s), dtype=torch.uint8, device="cuda")
+    jq.evict_layer_host(hK, hV, hQ, s, hKo, hVo, hidx, buf)
+    torch.cuda.synchronize()
+    assert np.array_equal(hidx.numpy(), gidx)
+    assert np.array_equal(hKo.numpy().view(np.uint16), gKo) and np.array_equal(hVo.numpy().view(np.uint16), gVo)
+
+
+# ------------------------------------------------------------------ full-size workloads (bench launch configuration)
+
+def test_cfg3_full_size_layer_budget_sweep():
+    K, V, Q, _ = W.make_layer(W.CFG3, layer=7)
+    pooled = oracle.pool(oracle.score(K, Q), W.CFG3.pool)     # scores do not depend on the budget
+    for budget in W.CFG3_BUDGETS:
+        run_e2e(W.CFG3.with_budget(budget), K, V, Q, pooled)
+
+
+def test_cfg4_longest_sequence():
+    wl = W.CFG4[3]
+    K, V, Q, _ = W.make_layer(wl, layer=1, seq=3)
+    run_e2e(wl, K, V, Q)
+
+
+def test_cfg5_full_size_sampled_heads():
+    """L = 131072, R = 256.  The GPU runs the whole layer; the oracle recomputes two of the eight KV
+    heads (heads are independent) and those are compared in full, for every budget of the sweep."""
+    wl = W.CFG5
+    K, V, Q, _ = W.make_layer(wl)
+    s = shape_of(wl)
+    heads = [0, 5]
+    g = wl.group
+    qrows = np.concatenate([np.arange(kv * g, kv * g + g) for kv in heads])
+    sc = oracle.score(K[heads], Q[qrows])
+    got = gpu_score(K, Q, s)
+    assert_scores_close(got[heads], sc)
+    np.testing.assert_allclose(got.sum(-1), wl.R, rtol=1e-3)
+    po = oracle.pool(sc, wl.pool)
+    for budget in W.CFG5_BUDGETS:
+        wb = wl.with_budget(budget)
+        gKo, gVo, gidx = gpu_evict(K, V, Q, shape_of(wb))
+        oidx = oracle.select(po, budget)
+        assert_kept_sets_agree(gidx[heads], oidx, po, wb.nkeep)
+        for kv in range(wl.Hkv):
+            assert np.all(np.diff(gidx[kv]) > 0)
+            assert np.array_equal(gKo[kv], K[kv][gidx[kv]]) and np.array_equal(gVo[kv], V[kv][gidx[kv]])
