@@ -17,6 +17,7 @@
 // word, raises a CTA-wide abort flag that every other wait polls, and leaves through the common exit
 // (which frees the tensor memory).
 #include "jq_internal.cuh"
+#include "jq_tmem_ld.cuh"
 #include <cuda.h>
 #include <cstddef>
 #include <mutex>
@@ -31,7 +32,7 @@ constexpr uint32_t kHalfBytes = kTile * 128;     // one 64-column half of a K ti
 constexpr uint32_t kStageBytes = 2 * kHalfBytes; // 32 KiB
 constexpr uint32_t kCtlBytes = 4096;             // barriers, flags, M_r
 constexpr uint32_t kTmemCols = 512;
-constexpr unsigned long long kWaitNs = 2000000000ull;   // 2 s per wait
+constexpr long long kWaitCycles = 4000000000ll;         // about 2 s of SM clock per wait
 
 struct Ctl {
     uint64_t full[kStages], empty[kStages];
@@ -50,6 +51,7 @@ struct Params {
     int h0, nheads, tph;     // KV heads [h0, h0+nheads) ; tiles per head
     float c;                 // log2(e) / sqrt(d)
     float2 *part;            // [Hkv][kSlots][R]
+    float *Mrow;             // [Hkv][R]   c*m + log2(l) per query row
     float *scores;           // [Hkv][L]
     int *status;
 };
@@ -80,22 +82,18 @@ __device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity)
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ unsigned long long now_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
 // Bounded wait.  false: the wait ran out (status recorded) or another thread of the CTA aborted.
+// The clock is only consulted after a few thousand failed polls, so a normal wait never pays for it.
 __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, Ctl *ctl, int *status)
 {
-    const unsigned long long t0 = now_ns();
+    for (int i = 0; i < 4096; ++i)
+        if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
     for (;;) {
         for (int i = 0; i < 256; ++i)
             if (mbar_try(bar, parity)) return true;
         if (*(volatile int *)&ctl->abort_flag) return false;
-        if (now_ns() - t0 > kWaitNs) {
+        if (clock64() - t0 > kWaitCycles) {
             *(volatile int *)&ctl->abort_flag = 1;
             atomicMax(status, (int)JQ_ERR_TIMEOUT);
             return false;
@@ -145,17 +143,6 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
-
-#define JQ_TMEM_LD32(taddr, v)                                                                              \
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                  \
-                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "                  \
-                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"  \
-                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),     \
-                   "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), \
-                   "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]),           \
-                   "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]),           \
-                   "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])            \
-                 : "r"(taddr) : "memory")
 
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -298,26 +285,9 @@ score_pass(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUt
                 if (PASS == 1) {
                     if (seg >= 0) flush_partial(prev_kv);
                 } else {
-                    // M_r of the new head from the partials of the CTAs whose pass-1 range met this head
+                    // stage the row normalisers M_r of the new head
                     const int sb = (seg + 1) & 1;
-                    if (et < P.R) {
-                        const long long first = (long long)(kv - P.h0) * P.tph;
-                        const int b_lo = owner_of_tile(first, T, G), b_hi = owner_of_tile(first + P.tph - 1, T, G);
-                        const int g_lo = (P.Rbox == 256) ? (et >> 7) : 0, g_hi = (P.Rbox == 256) ? (et >> 7) : 1;
-                        float m = -INFINITY, l = 0.f;
-                        for (int b = b_lo; b <= b_hi; ++b) {
-                            if ((long long)b * T / G == ((long long)b + 1) * T / G) continue;   // CTA b had no tile
-                            for (int g = g_lo; g <= g_hi; ++g) {
-                                const float2 p = __ldcg(&P.part[((size_t)kv * kSlots + 2 * b + g) * P.R + et]);
-                                if (p.y > 0.f) {
-                                    const float mn = fmaxf(m, p.x);
-                                    l = l * ex2(c * (m - mn)) + p.y * ex2(c * (p.x - mn));
-                                    m = mn;
-                                }
-                            }
-                        }
-                        ctl->Ms[sb][et] = c * m + log2f(l);
-                    }
+                    if (et < P.R) ctl->Ms[sb][et] = __ldcg(&P.Mrow[(size_t)kv * P.R + et]);
                     mbar_arrive(&ctl->m_ready[sb]);
                     if (!mbar_wait(&ctl->m_ready[sb], ((seg + 1) >> 1) & 1, ctl, P.status)) break;
                 }
@@ -329,64 +299,82 @@ score_pass(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUt
                 if (!mbar_wait(&ctl->t_full[slot], (unit / nslots) & 1, ctl, P.status)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t taddr = lane_addr + slot * slot_cols;
-                uint32_t v[32];
+                uint32_t v[128];
                 if (PASS == 1) {
+                    // the whole 128-key row segment in one tensor-memory read; the slot is free right after
+                    JQ_TMEM_LD128(taddr, v);
+                    tmem_ld_wait();
+                    tc_fence_before();
+                    mbar_arrive(&ctl->t_empty[slot]);
                     const int valid = min(kTile, P.L - j0);
-#pragma unroll 1
-                    for (int c0 = 0; c0 < kTile; c0 += 32) {
-                        JQ_TMEM_LD32(taddr + c0, v);
-                        tmem_ld_wait();
-                        if (c0 + 32 >= kTile) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot]); }
-                        const int nv = valid - c0;               // columns of this chunk that are real keys
-                        if (nv <= 0) continue;
-                        float cm = -INFINITY;
-                        if (nv >= 32) {
+                    if (valid < kTile) {
 #pragma unroll
-                            for (int t = 0; t < 32; ++t) cm = fmaxf(cm, __uint_as_float(v[t]));
-                        } else {
+                        for (int t = 0; t < 128; ++t) if (t >= valid) v[t] = 0xff800000u;   // -inf: not a key
+                    }
+                    float c0 = -INFINITY, c1 = -INFINITY, c2 = -INFINITY, c3 = -INFINITY;
 #pragma unroll
-                            for (int t = 0; t < 32; ++t) if (t < nv) cm = fmaxf(cm, __uint_as_float(v[t]));
-                        }
-                        if (cm > m_run) {
-                            const float f = ex2(c * (m_run - cm));
-                            l0 *= f; l1 *= f; l2 *= f; l3 *= f;
-                            m_run = cm;
-                        }
-                        const float mc = m_run * c;
-                        if (nv >= 32) {
+                    for (int t = 0; t < 128; t += 4) {
+                        c0 = fmaxf(c0, __uint_as_float(v[t + 0])); c1 = fmaxf(c1, __uint_as_float(v[t + 1]));
+                        c2 = fmaxf(c2, __uint_as_float(v[t + 2])); c3 = fmaxf(c3, __uint_as_float(v[t + 3]));
+                    }
+                    const float cm = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));
+                    if (cm > m_run) {
+                        const float f = ex2(c * (m_run - cm));
+                        l0 *= f; l1 *= f; l2 *= f; l3 *= f;
+                        m_run = cm;
+                    }
+                    const float mc = m_run * c;
 #pragma unroll
-                            for (int t = 0; t < 32; t += 4) {
-                                l0 += ex2(fmaf(__uint_as_float(v[t + 0]), c, -mc));
-                                l1 += ex2(fmaf(__uint_as_float(v[t + 1]), c, -mc));
-                                l2 += ex2(fmaf(__uint_as_float(v[t + 2]), c, -mc));
-                                l3 += ex2(fmaf(__uint_as_float(v[t + 3]), c, -mc));
-                            }
-                        } else {
-#pragma unroll
-                            for (int t = 0; t < 32; ++t) if (t < nv) l0 += ex2(fmaf(__uint_as_float(v[t]), c, -mc));
-                        }
+                    for (int t = 0; t < 128; t += 4) {
+                        l0 += ex2(fmaf(__uint_as_float(v[t + 0]), c, -mc));
+                        l1 += ex2(fmaf(__uint_as_float(v[t + 1]), c, -mc));
+                        l2 += ex2(fmaf(__uint_as_float(v[t + 2]), c, -mc));
+                        l3 += ex2(fmaf(__uint_as_float(v[t + 3]), c, -mc));
                     }
                 } else {
                     const float *Ms = ctl->Ms[seg & 1];
                     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll 1
-                    for (int c0 = 0; c0 < Rpad; c0 += 32) {
-                        JQ_TMEM_LD32(taddr + c0, v);
-                        tmem_ld_wait();
-                        if (c0 + 32 >= Rpad) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot]); }
-                        const int nv = P.R - c0;                 // columns of this chunk that are real query rows
-                        if (nv >= 32) {
+                    for (int c0 = 0; c0 < Rpad; c0 += 128) {
+                        if (Rpad - c0 >= 128) {
+                            JQ_TMEM_LD128(taddr + c0, v);
+                            tmem_ld_wait();
+                            if (c0 + 128 >= Rpad) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot]); }
+                            const int nv = P.R - c0;             // columns that are real query rows
+                            if (nv >= 128) {
 #pragma unroll
-                            for (int t = 0; t < 32; t += 4) {
-                                const float4 mm = *(const float4 *)(Ms + c0 + t);
-                                a0 += ex2(fmaf(__uint_as_float(v[t + 0]), c, -mm.x));
-                                a1 += ex2(fmaf(__uint_as_float(v[t + 1]), c, -mm.y));
-                                a2 += ex2(fmaf(__uint_as_float(v[t + 2]), c, -mm.z));
-                                a3 += ex2(fmaf(__uint_as_float(v[t + 3]), c, -mm.w));
+                                for (int t = 0; t < 128; t += 4) {
+                                    const float4 mm = *(const float4 *)(Ms + c0 + t);
+                                    a0 += ex2(fmaf(__uint_as_float(v[t + 0]), c, -mm.x));
+                                    a1 += ex2(fmaf(__uint_as_float(v[t + 1]), c, -mm.y));
+                                    a2 += ex2(fmaf(__uint_as_float(v[t + 2]), c, -mm.z));
+                                    a3 += ex2(fmaf(__uint_as_float(v[t + 3]), c, -mm.w));
+                                }
+                            } else {
+#pragma unroll
+                                for (int t = 0; t < 128; ++t) if (t < nv) a0 += ex2(fmaf(__uint_as_float(v[t]), c, -Ms[c0 + t]));
                             }
                         } else {
+#pragma unroll 1
+                            for (int c1 = c0; c1 < Rpad; c1 += 32) {
+                                JQ_TMEM_LD32(taddr + c1, v);
+                                tmem_ld_wait();
+                                if (c1 + 32 >= Rpad) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot]); }
+                                const int nv = P.R - c1;
+                                if (nv >= 32) {
 #pragma unroll
-                            for (int t = 0; t < 32; ++t) if (t < nv) a0 += ex2(fmaf(__uint_as_float(v[t]), c, -Ms[c0 + t]));
+                                    for (int t = 0; t < 32; t += 4) {
+                                        const float4 mm = *(const float4 *)(Ms + c1 + t);
+                                        a0 += ex2(fmaf(__uint_as_float(v[t + 0]), c, -mm.x));
+                                        a1 += ex2(fmaf(__uint_as_float(v[t + 1]), c, -mm.y));
+                                        a2 += ex2(fmaf(__uint_as_float(v[t + 2]), c, -mm.z));
+                                        a3 += ex2(fmaf(__uint_as_float(v[t + 3]), c, -mm.w));
+                                    }
+                                } else {
+#pragma unroll
+                                    for (int t = 0; t < 32; ++t) if (t < nv) a0 += ex2(fmaf(__uint_as_float(v[t]), c, -Ms[c1 + t]));
+                                }
+                            }
                         }
                     }
                     const int key = j0 + quarter * 32 + lane;
@@ -406,6 +394,48 @@ score_pass(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUt
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
+}
+
+// Combines the per-CTA partial (m, l) of pass 1 into M_r = c*m_r + log2(l_r).  One warp per query
+// row, lanes over the partial slots, then a butterfly; the order is fixed, hence deterministic.
+// grid (ceil(R/8), nheads), block 256.
+__device__ __forceinline__ void merge_ml(float &m, float &l, float m2, float l2, float c)
+{
+    if (l2 > 0.f) {
+        if (l > 0.f) {
+            const float mn = fmaxf(m, m2);
+            l = l * ex2(c * (m - mn)) + l2 * ex2(c * (m2 - mn));
+            m = mn;
+        } else {
+            m = m2; l = l2;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+merge_partials(const float2 *__restrict__ part, float *__restrict__ Mrow, int R, int Rbox, int h0, int tph,
+               int nheads, int G, float c)
+{
+    const int lane = threadIdx.x & 31, r = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (r >= R) return;
+    const int kv = h0 + blockIdx.y;
+    const long long T = (long long)nheads * tph, first = (long long)blockIdx.y * tph;
+    const int b_lo = owner_of_tile(first, T, G), b_hi = owner_of_tile(first + tph - 1, T, G);
+    const int ng = (Rbox == 256) ? 1 : 2, g0 = (Rbox == 256) ? (r >> 7) : 0;
+    const int nsl = (b_hi - b_lo + 1) * ng;
+    float m = -INFINITY, l = 0.f;
+    for (int i = lane; i < nsl; i += 32) {
+        const int b = b_lo + i / ng, g = g0 + i % ng;
+        if ((long long)b * T / G == ((long long)b + 1) * T / G) continue;   // CTA b had no tile
+        const float2 p = __ldcg(&part[((size_t)kv * kSlots + 2 * b + g) * R + r]);
+        merge_ml(m, l, p.x, p.y, c);
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, m, o), l2 = __shfl_xor_sync(0xffffffffu, l, o);
+        merge_ml(m, l, m2, l2, c);
+    }
+    if (lane == 0) Mrow[(size_t)kv * R + r] = c * m + log2f(l);
 }
 
 // ------------------------------------------------------------------ host side
@@ -483,7 +513,7 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
     P.L = s.L; P.R = R; P.Rbox = R <= 128 ? 128 : 256;
     P.tph = (s.L + kTile - 1) / kTile;
     P.c = 1.4426950408889634f / sqrtf((float)s.d);
-    P.part = w.part; P.scores = scores; P.status = w.status;
+    P.part = w.part; P.Mrow = w.Mrow; P.scores = scores; P.status = w.status;
     CUtensorMap mapK, mapQ;
     if (!make_map(&mapK, K, s.L, s.Hkv, kTile) || !make_map(&mapQ, Q, R, s.Hkv, P.Rbox)) return JQ_ERR_CUDA;
     const size_t smem = kCtlBytes + 1024 + (size_t)(P.Rbox == 128 ? 2 : 1) * P.Rbox * kD * 2 + (size_t)kStages * kStageBytes;
@@ -493,13 +523,15 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
     const long long head_bytes = (long long)s.L * kD * 2;
     long long per_group = (dev.l2 / 2) / head_bytes;
     if (per_group < 1) per_group = 1;
-    if (per_group > s.Hkv) per_group = s.Hkv;
+    const long long ngroups = (s.Hkv + per_group - 1) / per_group;
+    per_group = (s.Hkv + ngroups - 1) / ngroups;       // even split
     for (int h0 = 0; h0 < s.Hkv; h0 += (int)per_group) {
         P.h0 = h0;
         P.nheads = (int)(h0 + per_group <= s.Hkv ? per_group : s.Hkv - h0);
         score_pass<1><<<grid, kThreads, smem, st>>>(mapK, mapQ, P);
+        merge_partials<<<dim3((R + 7) / 8, P.nheads), 256, 0, st>>>(w.part, w.Mrow, R, P.Rbox, h0, P.tph, P.nheads, grid, P.c);
         score_pass<2><<<grid, kThreads, smem, st>>>(mapK, mapQ, P);
-        count_launch(2);
+        count_launch(3);
     }
     return check_launch();
 }
