@@ -1,19 +1,41 @@
-// Max-pool + exact top-k selection per KV head.
+// Max-pool + exact top-k selection per KV head, one thread-block cluster of 8 CTAs per head.
 //
-//   1. pool_keys: pooled[j] = max of the centred window (edges clipped); stored as an
-//      order-preserving 32-bit integer key (float order == unsigned order).
-//   2. radix_select: 4 rounds of 8 bits, most significant first, over integer histograms, find the
-//      key tau of the nkeep-th largest element and how many elements equal to tau are kept.
-//      Max-pooling copies every peak into up to `pool` neighbours, so ties at tau are the normal
-//      case: all keys > tau are kept, then the lowest-index keys == tau.
-//   3. ordered compaction: kept positions are written in ascending order.
+//   1. pool: pooled[j] = max of the centred window (edges clipped), turned into an order-preserving
+//      32-bit integer key (float order == unsigned order).  Each CTA owns a contiguous eighth of
+//      the positions and keeps its keys in shared memory (in the workspace for very long prefixes).
+//   2. radix select, 3 rounds of 11/11/10 bits, most significant first: local integer histograms
+//      are summed into the leading CTA through distributed shared memory, which finds the digit
+//      holding the nkeep-th largest key and broadcasts it.  Result: the key tau of the nkeep-th
+//      largest element and how many elements equal to tau are kept.  Max-pooling copies every peak
+//      into up to `pool` neighbours, so ties at tau are the normal case: all keys > tau are kept,
+//      then the lowest-index keys == tau.
+//   3. ordered compaction: kept positions are written in ascending order (CTA rank, warp,
+//      iteration and lane order all follow the position order).
 // Everything is integer arithmetic on bit patterns, hence deterministic and exact.
 #include "jq_internal.cuh"
+#include <cooperative_groups.h>
+
+namespace cg = cooperative_groups;
 
 namespace jq {
 namespace {
 
+constexpr int kCl = 8;             // CTAs per cluster (= per KV head)
 constexpr int kSelThreads = 1024;
+constexpr int kBins = 2048;
+constexpr int kRawTile = 4096;     // scores staged per pooling step
+constexpr int kHalo = 32;          // >= pool radius
+constexpr int kKeysSmemMax = 36864; // keys a CTA can keep in shared memory
+
+struct SelCtl {
+    uint32_t prefix;
+    int krem;
+    int found_prefix_digit, found_krem;
+    int counts_gt[kCl], counts_eq[kCl];
+    int warp_gt[32], warp_eq[32];
+    int tot_gt, tot_eq;
+    int scan[33];
+};
 
 __device__ __forceinline__ uint32_t order_key(float x)
 {
@@ -21,25 +43,8 @@ __device__ __forceinline__ uint32_t order_key(float x)
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-// grid (ceil(L/256), Hkv), block 256.
-__global__ void __launch_bounds__(256)
-pool_keys(const float *__restrict__ scores, int L, int radius, uint32_t *__restrict__ keys,
-          float *__restrict__ pooled)
-{
-    const int kv = blockIdx.y;
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= L) return;
-    const float *s = scores + (size_t)kv * L;
-    const int lo = max(j - radius, 0), hi = min(j + radius, L - 1);
-    float best = s[j];
-    for (int u = lo; u <= hi; ++u) best = fmaxf(best, s[u]);
-    keys[(size_t)kv * L + j] = order_key(best);
-    if (pooled) pooled[(size_t)kv * L + j] = best;
-}
-
-// Block-wide exclusive scan of one int per thread (1024 threads); returns the exclusive prefix and
-// the block total through `total`.
-__device__ __forceinline__ int block_excl_scan(int v, int *warp_sums, int &total)
+// Block-wide exclusive scan of one int per thread (1024 threads).
+__device__ __forceinline__ int block_excl_scan(int v, int *warp_sums)
 {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     int inc = v;
@@ -59,88 +64,158 @@ __device__ __forceinline__ int block_excl_scan(int v, int *warp_sums, int &total
             if (lane >= o) winc += n;
         }
         warp_sums[lane] = winc - ws;       // exclusive warp offsets
-        if (lane == 31) warp_sums[32] = winc;
     }
     __syncthreads();
     const int excl = warp_sums[wid] + inc - v;
-    total = warp_sums[32];
     __syncthreads();
     return excl;
 }
 
-// grid (Hkv), block 1024.
-__global__ void __launch_bounds__(kSelThreads)
-radix_select_compact(const uint32_t *__restrict__ keys, int L, int nkeep, int32_t *__restrict__ idx)
+// grid (Hkv * 8), cluster 8, block 1024.
+__global__ void __cluster_dims__(kCl, 1, 1) __launch_bounds__(kSelThreads, 1)
+select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, int32_t *__restrict__ idx,
+               float *__restrict__ pooled, uint32_t *__restrict__ gkeys, int chunk, int keys_in_smem)
 {
-    __shared__ int hist[256];
-    __shared__ int warp_sums[33];
-    __shared__ uint32_t s_prefix;
-    __shared__ int s_krem;
-    const int kv = blockIdx.x;
-    const uint32_t *key = keys + (size_t)kv * L;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    const int kv = blockIdx.x / kCl;
+    extern __shared__ __align__(16) uint8_t sm[];
+    uint32_t *ghist = (uint32_t *)sm;                       // [3][kBins]; the leading CTA's copy accumulates the cluster
+    uint32_t *hist = ghist + 3 * kBins;                     // [kBins]
+    float *raw = (float *)(hist + kBins);                   // [kRawTile + 2*kHalo]
+    uint32_t *keys_s = (uint32_t *)(raw + kRawTile + 2 * kHalo);
+    __shared__ SelCtl ctl;
+
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int j0 = min(rank * chunk, L), j1 = min(j0 + chunk, L), n = j1 - j0;
+    const float *s = scores + (size_t)kv * L;
+    uint32_t *mykeys = keys_in_smem ? keys_s : gkeys + (size_t)kv * L + j0;
     int32_t *out = idx + (size_t)kv * nkeep;
 
-    if (nkeep >= L) {  // everything is kept
-        for (int j = threadIdx.x; j < L; j += blockDim.x) out[j] = j;
+    // ---- 1. max-pool -> keys
+    for (int t0 = 0; t0 < n; t0 += kRawTile) {
+        const int tile = min(kRawTile, n - t0);
+        __syncthreads();
+        for (int i = tid; i < tile + 2 * radius; i += kSelThreads) {
+            const int j = j0 + t0 - radius + i;
+            raw[i] = (j >= 0 && j < L) ? s[j] : -INFINITY;
+        }
+        __syncthreads();
+        for (int e = tid; e < tile; e += kSelThreads) {
+            float best = raw[e];
+            for (int u = 1; u <= 2 * radius; ++u) best = fmaxf(best, raw[e + u]);
+            mykeys[t0 + e] = order_key(best);
+            if (pooled) pooled[(size_t)kv * L + j0 + t0 + e] = best;
+        }
+    }
+    if (nkeep >= L) {   // everything is kept (uniform over the cluster; no cluster traffic yet)
+        for (int e = tid; e < n; e += kSelThreads) out[j0 + e] = j0 + e;
         return;
     }
-    if (threadIdx.x == 0) { s_prefix = 0; s_krem = nkeep; }
-    for (int round = 0; round < 4; ++round) {
-        const int shift = 24 - 8 * round;
-        if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+    for (int i = tid; i < 3 * kBins; i += kSelThreads) ghist[i] = 0;
+    if (tid == 0) { ctl.prefix = 0; ctl.krem = nkeep; }
+    cluster.sync();
+
+    // ---- 2. radix select
+    const int n_up = (n + kSelThreads - 1) / kSelThreads * kSelThreads;
+    for (int round = 0; round < 3; ++round) {
+        const int shift = (round == 0) ? 21 : (round == 1 ? 10 : 0);
+        const int width = (round == 2) ? 10 : 11;
+        const uint32_t mask = (1u << width) - 1u;
+        for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
         __syncthreads();
-        const uint32_t prefix = s_prefix;
-        // uniform trip count so that the warp-level match sees whole warps
-        for (int base = 0; base < L; base += blockDim.x) {
-            const int j = base + threadIdx.x;
+        const uint32_t prefix = ctl.prefix;
+        for (int base = 0; base < n_up; base += kSelThreads) {   // uniform trip count: whole warps reach the match
+            const int e = base + tid;
             bool live = false;
             uint32_t digit = 0;
-            if (j < L) {
-                const uint32_t k = key[j];
-                live = (round == 0) || ((k >> (shift + 8)) == prefix);
-                digit = (k >> shift) & 255u;
+            if (e < n) {
+                const uint32_t k = mykeys[e];
+                live = (round == 0) || ((k >> (shift + width)) == prefix);
+                digit = (k >> shift) & mask;
             }
-            const uint32_t tag = live ? digit : 256u;
+            const uint32_t tag = live ? digit : 0xffffffffu;
             const uint32_t peers = __match_any_sync(0xffffffffu, tag);
-            if (live && (__ffs(peers) - 1) == (threadIdx.x & 31)) atomicAdd(&hist[digit], __popc(peers));
+            if (live && (__ffs(peers) - 1) == lane) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
         }
         __syncthreads();
-        if (threadIdx.x == 0) {
-            int krem = s_krem, above = 0, dsel = 0;
-            for (int dg = 255; dg >= 0; --dg) {
-                const int h = hist[dg];
-                if (above + h >= krem) { dsel = dg; break; }
-                above += h;
+        uint32_t *g0 = cluster.map_shared_rank(ghist + round * kBins, 0);
+        for (int i = tid; i < kBins; i += kSelThreads) {
+            const uint32_t v = hist[i];
+            if (v) atomicAdd(&g0[i], v);
+        }
+        cluster.sync();
+        if (rank == 0) {
+            // bins in descending order: thread t looks at bins 2047-2t and 2046-2t
+            const uint32_t *g = ghist + round * kBins;
+            const int hi = kBins - 1 - 2 * tid, lo = hi - 1;
+            const int h_hi = (int)g[hi], h_lo = (int)g[lo];
+            const int above = block_excl_scan(h_hi + h_lo, ctl.scan);
+            const int krem = ctl.krem;
+            if (above < krem && krem <= above + h_hi) {
+                ctl.found_prefix_digit = hi; ctl.found_krem = krem - above;
+            } else if (above + h_hi < krem && krem <= above + h_hi + h_lo) {
+                ctl.found_prefix_digit = lo; ctl.found_krem = krem - above - h_hi;
             }
-            s_krem = krem - above;
-            s_prefix = (prefix << 8) | (uint32_t)dsel;
+            __syncthreads();
+            if (tid < kCl) {
+                SelCtl *rc = cluster.map_shared_rank(&ctl, tid);
+                rc->prefix = (prefix << width) | (uint32_t)ctl.found_prefix_digit;
+                rc->krem = ctl.found_krem;
+            }
         }
-        __syncthreads();
+        cluster.sync();
     }
-    const uint32_t tau = s_prefix;
-    const int need_eq = s_krem;  // how many of the keys == tau are kept (lowest indices first)
+    const uint32_t tau = ctl.prefix;
+    const int need_eq = ctl.krem;   // how many of the keys == tau are kept (lowest positions first)
 
-    // ordered compaction: thread t owns the contiguous positions [t*seg, (t+1)*seg)
-    const int seg = (L + blockDim.x - 1) / blockDim.x;
-    const int j0 = min(threadIdx.x * seg, L), j1 = min(j0 + seg, L);
-    int gt = 0, eq = 0;
-    for (int j = j0; j < j1; ++j) {
-        const uint32_t k = key[j];
-        gt += (k > tau);
-        eq += (k == tau);
+    // ---- 3. ordered compaction; warp w owns the contiguous elements [w*seg, (w+1)*seg)
+    const int seg = ((n + 31) / 32 + 31) / 32 * 32;
+    const int w0 = min(wid * seg, n), w1 = min(w0 + seg, n);
+    int cgt = 0, ceq = 0;
+    for (int base = w0; base < w1; base += 32) {
+        const int e = base + lane;
+        const uint32_t k = (e < w1) ? mykeys[e] : 0u;
+        const bool in = e < w1;
+        cgt += __popc(__ballot_sync(0xffffffffu, in && k > tau));
+        ceq += __popc(__ballot_sync(0xffffffffu, in && k == tau));
     }
-    int tot_gt, tot_eq;
-    int gt_before = block_excl_scan(gt, warp_sums, tot_gt);
-    int eq_before = block_excl_scan(eq, warp_sums, tot_eq);
-    for (int j = j0; j < j1; ++j) {
-        const uint32_t k = key[j];
-        if (k > tau) {
-            out[gt_before + min(eq_before, need_eq)] = j;
-            ++gt_before;
-        } else if (k == tau) {
-            if (eq_before < need_eq) out[gt_before + eq_before] = j;
-            ++eq_before;
+    if (lane == 0) { ctl.warp_gt[wid] = cgt; ctl.warp_eq[wid] = ceq; }
+    __syncthreads();
+    if (wid == 0) {
+        const int g = ctl.warp_gt[lane], q = ctl.warp_eq[lane];
+        int gi = g, qi = q;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int a = __shfl_up_sync(0xffffffffu, gi, o), b = __shfl_up_sync(0xffffffffu, qi, o);
+            if (lane >= o) { gi += a; qi += b; }
         }
+        ctl.warp_gt[lane] = gi - g; ctl.warp_eq[lane] = qi - q;   // exclusive
+        if (lane == 31) { ctl.tot_gt = gi; ctl.tot_eq = qi; }
+    }
+    __syncthreads();
+    if (tid < kCl) {
+        SelCtl *rc = cluster.map_shared_rank(&ctl, tid);
+        rc->counts_gt[rank] = ctl.tot_gt;
+        rc->counts_eq[rank] = ctl.tot_eq;
+    }
+    cluster.sync();
+    int gt_before = ctl.warp_gt[wid], eq_before = ctl.warp_eq[wid];
+    for (int q = 0; q < rank; ++q) { gt_before += ctl.counts_gt[q]; eq_before += ctl.counts_eq[q]; }
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    for (int base = w0; base < w1; base += 32) {
+        const int e = base + lane;
+        const bool in = e < w1;
+        const uint32_t k = in ? mykeys[e] : 0u;
+        const uint32_t bg = __ballot_sync(0xffffffffu, in && k > tau);
+        const uint32_t be = __ballot_sync(0xffffffffu, in && k == tau);
+        const int g_here = gt_before + __popc(bg & lt_mask), e_here = eq_before + __popc(be & lt_mask);
+        if (in) {
+            if (k > tau) out[g_here + min(e_here, need_eq)] = j0 + e;
+            else if (k == tau && e_here < need_eq) out[g_here + e_here] = j0 + e;
+        }
+        gt_before += __popc(bg);
+        eq_before += __popc(be);
     }
 }
 
@@ -150,9 +225,22 @@ jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, fl
                         const Workspace &w, cudaStream_t st)
 {
     const int nkeep = s.budget < s.L ? s.budget : s.L;
-    pool_keys<<<dim3((s.L + 255) / 256, s.Hkv), 256, 0, st>>>(scores, s.L, (s.pool - 1) / 2, w.keys, pooled);
-    radix_select_compact<<<s.Hkv, kSelThreads, 0, st>>>(w.keys, s.L, nkeep, idx);
-    count_launch(2);
+    int chunk = (s.L + kCl - 1) / kCl;
+    chunk = (chunk + 31) / 32 * 32;
+    const int in_smem = chunk <= kKeysSmemMax;
+    const size_t smem = (size_t)(4 * kBins + kRawTile + 2 * kHalo) * 4 + (in_smem ? (size_t)chunk * 4 : 0);
+    static bool attr_done[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return JQ_ERR_CUDA;
+    if (!attr_done[dev]) {
+        const int max_smem = (4 * kBins + kRawTile + 2 * kHalo + kKeysSmemMax) * 4;
+        if (cudaFuncSetAttribute(select_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
+            return JQ_ERR_CUDA;
+        attr_done[dev] = true;
+    }
+    select_cluster<<<s.Hkv * kCl, kSelThreads, smem, st>>>(scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, w.keys,
+                                                          chunk, in_smem);
+    count_launch(1);
     return check_launch();
 }
 
