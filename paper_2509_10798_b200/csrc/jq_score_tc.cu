@@ -1,59 +1,75 @@
-// Tensor-core scoring for sm_100a: Eq. 3 in two streaming passes over K.
+// Tensor-core scoring for sm_100a: Eq. 3 in two streaming passes over K, ONE persistent kernel per call.
 //
-// Both passes are persistent, warp-specialised kernels (one CTA per SM):
+// The grid is one CTA per SM, launched cooperatively (all CTAs are resident, so they may wait on one
+// another).  A CTA is warp-specialised:
 //   warp 0      TMA producer: K tiles of 128 keys (two 64-column halves, 128-byte swizzle) into a
-//               ring of shared-memory stages; the query rows of a KV head into a stationary buffer;
+//               ring of shared-memory stages; the query rows of a KV head into one of two stationary buffers;
 //   warp 1      issues tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory) and owns the TMEM allocation;
-//   warps 2-9   two epilogue groups of 128 threads that read accumulators with tcgen05.ld.
+//   warps 2-9   two epilogue groups of 128 threads that read accumulators with tcgen05.ld;
+//   warp 10     merges the per-CTA partial row statistics of pass 1 across the grid.
 // The operand roles are swapped between the passes so that no reduction crosses threads:
 //   pass 1  S[R x 128] = Q K^T   (A = query rows, M = 128): a thread owns a QUERY ROW and keeps its
 //           running max m and sum l = sum_j exp2(c (s_j - m)); per-CTA partial (m, l) go to the workspace;
 //   pass 2  S^T[128 x R] = K Q^T (A = key tile, N = R):     a thread owns a KEY and adds
 //           exp2(c s - M_r) over the R rows, M_r = c m_r + log2(l_r) merged from the partials.
-// Tiles are split statically and contiguously over the CTAs; pass 2 walks its range backwards so the
-// tiles pass 1 read last (most likely still in L2) are read first.
 //
-// Every wait is bounded: when one runs out, the CTA records JQ_ERR_TIMEOUT in the workspace status
-// word, raises a CTA-wide abort flag that every other wait polls, and leaves through the common exit
-// (which frees the tensor memory).
+// KV heads are taken in groups whose keys fit in a share of the L2.  The tiles of a group are split
+// statically and contiguously over the CTAs, the same split in both passes, and pass 2 walks its range
+// backwards, so a CTA re-reads what it read itself, most recent first.  The segments are ordered
+//   P1(0) P1(1) P2(0) P1(2) P2(1) ... P2(last)
+// so that the grid-wide merge of group g (counter -> merge warp -> counter) happens while every CTA is busy
+// with pass 1 of group g+1; only the epilogue warps ever wait for it, and normally find it done.
+//
+// Grid-wide counters live in the status block at the head of the workspace (zeroed by
+// jq_workspace_init): a ring of four per kind, with cumulative targets, reset by the last CTA to
+// leave.  Every wait (mbarrier or counter) is bounded: when one runs out, the CTA records
+// JQ_ERR_TIMEOUT in the status word, raises a CTA-wide abort flag that every other wait polls, runs
+// through its remaining barriers without touching data, and leaves through the common exit (which
+// frees the tensor memory).
 #include "jq_internal.cuh"
 #include "jq_tmem_ld.cuh"
 #include <cuda.h>
 #include <cstddef>
+#include <cstdlib>
 #include <mutex>
 
 namespace jq {
 namespace {
 
 constexpr int kTile = 128;                       // keys per tile
-constexpr int kStages = 4;                       // K ring depth
-constexpr int kThreads = 320;
+constexpr int kMaxStages = 5;                    // K ring depth (5 when R <= 128, 3 above)
+constexpr int kThreads = 352;                    // 11 warps
 constexpr uint32_t kHalfBytes = kTile * 128;     // one 64-column half of a K tile (128-byte rows)
 constexpr uint32_t kStageBytes = 2 * kHalfBytes; // 32 KiB
-constexpr uint32_t kCtlBytes = 4096;             // barriers, flags, M_r
+constexpr uint32_t kCtlBytes = 2048;             // barriers, flags, M_r
 constexpr uint32_t kTmemCols = 512;
-constexpr long long kWaitCycles = 4000000000ll;         // about 2 s of SM clock per wait
+constexpr long long kWaitCycles = 4000000000ll;  // about 2 s of SM clock per wait
+constexpr int kRing = 4;                         // grid counters per kind
+// words of the workspace status block
+constexpr int kWStatus = 0, kWDone = 1, kWCnt1 = 8, kWCnt2 = 12;
 
 struct Ctl {
-    uint64_t full[kStages], empty[kStages];
+    uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t q_full[2], q_empty[2];
     uint64_t t_full[4], t_empty[4];
-    uint64_t m_ready[2];
     uint32_t tmem_base;
     int abort_flag;
-    alignas(16) float Ms[2][kMaxR];   // read as float4
+    alignas(16) float Ms[kMaxR];   // read as float4
 };
 static_assert(offsetof(Ctl, Ms) % 16 == 0, "Ms must be 16-byte aligned");
 static_assert(sizeof(Ctl) <= kCtlBytes, "control block too large");
 
 struct Params {
-    int L, R, Rbox;          // Rbox = 128 or 256: query rows staged per KV head (rows >= R are zero)
-    int h0, nheads, tph;     // KV heads [h0, h0+nheads) ; tiles per head
+    int L, R, Rbox, Rpad;    // Rbox = 128 or 256: query rows staged per KV head (rows >= R are zero)
+    int Hkv, tph;            // KV heads; tiles per head
+    int hpg, ngroups;        // heads per group, groups
+    int stages;              // K ring depth
+    int pipelined;           // 1: P1(0) P1(1) P2(0) P1(2) ... ; 0: P1(0) P2(0) P1(1) P2(1) ...
     float c;                 // log2(e) / sqrt(d)
     float2 *part;            // [Hkv][kSlots][R]
     float *Mrow;             // [Hkv][R]   c*m + log2(l) per query row
     float *scores;           // [Hkv][L]
-    int *status;
+    int *status;             // status block (kStatusWords ints)
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -68,9 +84,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar, uint32_t count)
 {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
 __device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity)
 {
@@ -86,6 +102,7 @@ __device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity)
 // The clock is only consulted after a few thousand failed polls, so a normal wait never pays for it.
 __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, Ctl *ctl, int *status)
 {
+    if (*(volatile int *)&ctl->abort_flag) return false;
     for (int i = 0; i < 4096; ++i)
         if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
@@ -95,7 +112,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, Ctl 
         if (*(volatile int *)&ctl->abort_flag) return false;
         if (clock64() - t0 > kWaitCycles) {
             *(volatile int *)&ctl->abort_flag = 1;
-            atomicMax(status, (int)JQ_ERR_TIMEOUT);
+            atomicMax(status + kWStatus, (int)JQ_ERR_TIMEOUT);
             return false;
         }
     }
@@ -105,6 +122,27 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, Ctl *c
     if (mbar_try(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, ctl, status);
 }
+
+// Bounded wait for a grid-wide counter to reach `target` (acquire).
+__device__ __noinline__ bool wait_counter(const int *p, int target, Ctl *ctl, int *status)
+{
+    const long long t0 = clock64();
+    for (;;) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+        if (v >= target) return true;
+        if (*(volatile int *)&ctl->abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *(volatile int *)&ctl->abort_flag = 1;
+            atomicMax(status + kWStatus, (int)JQ_ERR_TIMEOUT);
+            return false;
+        }
+        __nanosleep(64);
+    }
+}
+
+// Barrier among the 256 epilogue threads only.
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2)
 {
@@ -159,34 +197,67 @@ __device__ __forceinline__ int owner_of_tile(long long t, long long T, long long
     return (int)(((t + 1) * G - 1) / T);
 }
 
+// ------------------------------------------------------------------ schedule
+
+// Segment s of the 2 * ngroups segments every CTA walks: a pass over this CTA's share of one group.
+struct Seg {
+    int pass, g, h0, t_begin, t_end;
+};
+
+__device__ __forceinline__ Seg segment(int s, const Params &P)
+{
+    Seg sg;
+    const int NG = P.ngroups;
+    if (!P.pipelined) { sg.g = s >> 1; sg.pass = 1 + (s & 1); }
+    else if (s == 0) { sg.pass = 1; sg.g = 0; }
+    else if (s == 2 * NG - 1) { sg.pass = 2; sg.g = NG - 1; }
+    else if (s & 1) { sg.pass = 1; sg.g = (s + 1) >> 1; }
+    else { sg.pass = 2; sg.g = (s >> 1) - 1; }
+    sg.h0 = sg.g * P.hpg;
+    const int nh = min(P.hpg, P.Hkv - sg.h0);
+    const long long T = (long long)nh * P.tph, G = gridDim.x;
+    sg.t_begin = (int)((long long)blockIdx.x * T / G);
+    sg.t_end = (int)(((long long)blockIdx.x + 1) * T / G);
+    return sg;
+}
+
+// Merge of two partial (max, sum of exp2(c (s - max))) pairs; an empty partial has l == 0.
+__device__ __forceinline__ void merge_ml(float &m, float &l, float m2, float l2, float c)
+{
+    if (l2 > 0.f) {
+        if (l > 0.f) {
+            const float mn = fmaxf(m, m2);
+            l = l * ex2(c * (m - mn)) + l2 * ex2(c * (m2 - mn));
+            m = mn;
+        } else {
+            m = m2; l = l2;
+        }
+    }
+}
+
 // ------------------------------------------------------------------ the kernel
 
-template <int PASS>
 __global__ void __launch_bounds__(kThreads, 1)
-score_pass(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ, const Params P)
+score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ, const Params P)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    Ctl *ctl = (Ctl *)smem_raw;
-    const uint32_t base = (smem_u32(smem_raw) + kCtlBytes + 1023u) & ~1023u;   // 1024-byte aligned data
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned data
     uint8_t *data = smem_raw + (base - smem_u32(smem_raw));
-    const int nq = (P.Rbox == 128) ? 2 : 1;                  // query buffers (double-buffered when they fit)
     const uint32_t q_bytes = (uint32_t)P.Rbox * kD * 2;
-    uint8_t *qbuf = data;
-    uint8_t *kbuf = data + (size_t)nq * q_bytes;
+    uint8_t *qbuf = data;                                    // two query buffers
+    uint8_t *kbuf = data + 2 * (size_t)q_bytes;              // K ring
+    Ctl *ctl = (Ctl *)(kbuf + (size_t)P.stages * kStageBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long T = (long long)P.nheads * P.tph, G = gridDim.x;
-    const int t_begin = (int)((long long)blockIdx.x * T / G), t_end = (int)(((long long)blockIdx.x + 1) * T / G);
-    const int ntiles = t_end - t_begin;
-    const int nmb = (PASS == 1) ? P.Rbox / 128 : 1;          // accumulator blocks per tile
-    const int Rpad = (P.R + 15) & ~15;
-    const int nslots = (PASS == 1) ? 4 : (Rpad <= 128 ? 4 : 2);
+    const int G = gridDim.x, stages = P.stages;
+    const int nslots = (P.Rbox == 256) ? 2 : 4;
     const uint32_t slot_cols = kTmemCols / nslots;
+    const int nseg = 2 * P.ngroups;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&ctl->q_full[s], 1); mbar_init(&ctl->q_empty[s], 1); mbar_init(&ctl->m_ready[s], 256); }
-        for (int s = 0; s < 4; ++s) { mbar_init(&ctl->t_full[s], 1); mbar_init(&ctl->t_empty[s], 128); }
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&ctl->q_full[s], 1); mbar_init(&ctl->q_empty[s], 1); }
+        for (int s = 0; s < 4; ++s) { mbar_init(&ctl->t_full[s], 1); mbar_init(&ctl->t_empty[s], P.Rbox == 256 ? 256 : 128); }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -202,110 +273,121 @@ score_pass(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUt
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            int seg = -1, prev_kv = -1;
-            for (int n = 0; n < ntiles; ++n) {
-                const int i = (PASS == 1) ? t_begin + n : t_end - 1 - n;
-                const int kv = P.h0 + i / P.tph, j0 = (i % P.tph) * kTile;
-                if (kv != prev_kv) {
-                    prev_kv = kv; ++seg;
-                    const int qb = seg % nq;
-                    if (!mbar_wait(&ctl->q_empty[qb], ((seg / nq) & 1) ^ 1, ctl, P.status)) break;
-                    mbar_expect_tx(&ctl->q_full[qb], q_bytes);
-                    tma_load_3d(qbuf + (size_t)qb * q_bytes, &mapQ, &ctl->q_full[qb], 0, 0, kv);
-                    tma_load_3d(qbuf + (size_t)qb * q_bytes + q_bytes / 2, &mapQ, &ctl->q_full[qb], 64, 0, kv);
+            uint32_t it = 0, qn = 0;
+            int prev_kv = -1;
+            bool ok = true;
+            for (int s = 0; s < nseg && ok; ++s) {
+                const Seg sg = segment(s, P);
+                const int ntiles = sg.t_end - sg.t_begin;
+                for (int n = 0; n < ntiles; ++n, ++it) {
+                    const int i = (sg.pass == 1) ? sg.t_begin + n : sg.t_end - 1 - n;
+                    const int kv = sg.h0 + i / P.tph, j0 = (i % P.tph) * kTile;
+                    if (kv != prev_kv) {
+                        const uint32_t qb = qn & 1;
+                        if (!mbar_wait(&ctl->q_empty[qb], ((qn >> 1) & 1) ^ 1, ctl, P.status)) { ok = false; break; }
+                        mbar_expect_tx(&ctl->q_full[qb], q_bytes);
+                        tma_load_3d(qbuf + (size_t)qb * q_bytes, &mapQ, &ctl->q_full[qb], 0, 0, kv);
+                        tma_load_3d(qbuf + (size_t)qb * q_bytes + q_bytes / 2, &mapQ, &ctl->q_full[qb], 64, 0, kv);
+                        prev_kv = kv; ++qn;
+                    }
+                    const uint32_t st = it % stages;
+                    if (!mbar_wait(&ctl->empty[st], ((it / stages) & 1) ^ 1, ctl, P.status)) { ok = false; break; }
+                    mbar_expect_tx(&ctl->full[st], kStageBytes);
+                    tma_load_3d(kbuf + (size_t)st * kStageBytes, &mapK, &ctl->full[st], 0, j0, kv);
+                    tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, &mapK, &ctl->full[st], 64, j0, kv);
                 }
-                const int st = n % kStages;
-                if (!mbar_wait(&ctl->empty[st], ((n / kStages) & 1) ^ 1, ctl, P.status)) break;
-                mbar_expect_tx(&ctl->full[st], kStageBytes);
-                tma_load_3d(kbuf + (size_t)st * kStageBytes, &mapK, &ctl->full[st], 0, j0, kv);
-                tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, &mapK, &ctl->full[st], 64, j0, kv);
             }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = (PASS == 1) ? instr_desc(128, kTile) : instr_desc(kTile, Rpad);
-            int seg = -1, prev_kv = -1;
-            uint32_t unit = 0;
+            const uint32_t idesc1 = instr_desc(128, kTile), idesc2 = instr_desc(kTile, P.Rpad);
+            const int nmb = P.Rbox / 128;                     // pass 1: accumulator blocks of 128 query rows
+            uint32_t it = 0, qn = 0;
+            int prev_kv = -1;
             bool ok = true;
-            for (int n = 0; n < ntiles && ok; ++n) {
-                const int i = (PASS == 1) ? t_begin + n : t_end - 1 - n;
-                const int kv = P.h0 + i / P.tph;
-                if (kv != prev_kv) {
-                    if (seg >= 0) tc_commit(&ctl->q_empty[seg % nq]);   // previous head's queries are free once its MMAs retire
-                    prev_kv = kv; ++seg;
-                    if (!mbar_wait(&ctl->q_full[seg % nq], (seg / nq) & 1, ctl, P.status)) break;
-                }
-                const int st = n % kStages;
-                if (!mbar_wait(&ctl->full[st], (n / kStages) & 1, ctl, P.status)) break;
-                tc_fence_after();
-                const uint32_t k_addr = smem_u32(kbuf + (size_t)st * kStageBytes);
-                const uint32_t q_addr = smem_u32(qbuf + (size_t)(seg % nq) * q_bytes);
-                for (int mb = 0; mb < nmb; ++mb, ++unit) {
-                    const uint32_t slot = unit % nslots;
-                    if (!mbar_wait(&ctl->t_empty[slot], ((unit / nslots) & 1) ^ 1, ctl, P.status)) { ok = false; break; }
+            for (int s = 0; s < nseg && ok; ++s) {
+                const Seg sg = segment(s, P);
+                const int ntiles = sg.t_end - sg.t_begin;
+                for (int n = 0; n < ntiles; ++n, ++it) {
+                    const int i = (sg.pass == 1) ? sg.t_begin + n : sg.t_end - 1 - n;
+                    const int kv = sg.h0 + i / P.tph;
+                    if (kv != prev_kv) {
+                        if (qn > 0) tc_commit(&ctl->q_empty[(qn - 1) & 1]);   // the previous head's queries are free once its MMAs retire
+                        if (!mbar_wait(&ctl->q_full[qn & 1], (qn >> 1) & 1, ctl, P.status)) { ok = false; break; }
+                        prev_kv = kv; ++qn;
+                    }
+                    const uint32_t st = it % stages, slot = it % nslots;
+                    if (!mbar_wait(&ctl->full[st], (it / stages) & 1, ctl, P.status)) { ok = false; break; }
+                    if (!mbar_wait(&ctl->t_empty[slot], ((it / nslots) & 1) ^ 1, ctl, P.status)) { ok = false; break; }
                     tc_fence_after();
+                    const uint32_t k_addr = smem_u32(kbuf + (size_t)st * kStageBytes);
+                    const uint32_t q_addr = smem_u32(qbuf + (size_t)((qn - 1) & 1) * q_bytes);
                     const uint32_t d = tmem + slot * slot_cols;
+                    if (sg.pass == 1) {
+                        for (int mb = 0; mb < nmb; ++mb) {
 #pragma unroll
-                    for (int ks = 0; ks < kD / 16; ++ks) {
-                        const uint32_t koff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                        const uint32_t qoff = (uint32_t)(ks >> 2) * (q_bytes / 2) + (uint32_t)(ks & 3) * 32u;
-                        if (PASS == 1)
-                            tc_mma(d, smem_desc(q_addr + qoff + (uint32_t)mb * kHalfBytes), smem_desc(k_addr + koff), idesc, ks > 0);
-                        else
-                            tc_mma(d, smem_desc(k_addr + koff), smem_desc(q_addr + qoff), idesc, ks > 0);
+                            for (int ks = 0; ks < kD / 16; ++ks) {
+                                const uint32_t koff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                                const uint32_t qoff = (uint32_t)(ks >> 2) * (q_bytes / 2) + (uint32_t)(ks & 3) * 32u;
+                                tc_mma(d + (uint32_t)mb * 128u, smem_desc(q_addr + qoff + (uint32_t)mb * kHalfBytes),
+                                       smem_desc(k_addr + koff), idesc1, ks > 0);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int ks = 0; ks < kD / 16; ++ks) {
+                            const uint32_t koff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                            const uint32_t qoff = (uint32_t)(ks >> 2) * (q_bytes / 2) + (uint32_t)(ks & 3) * 32u;
+                            tc_mma(d, smem_desc(k_addr + koff), smem_desc(q_addr + qoff), idesc2, ks > 0);
+                        }
                     }
                     tc_commit(&ctl->t_full[slot]);
+                    tc_commit(&ctl->empty[st]);
                 }
-                tc_commit(&ctl->empty[st]);
             }
         }
-    } else {
+    } else if (warp < 10) {
         // ---------------------------------------------------------------- epilogue groups
         const int grp = (warp - 2) >> 2, quarter = warp & 3;
         const int et = threadIdx.x - 64;                        // 0..255
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
-        int seg = -1, prev_kv = -1;
-        uint32_t unit = 0;
-        float m_run = -INFINITY, l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-        bool ok = true;
+        const bool wide = P.Rbox == 256;
+        const int my_row = (wide ? grp * 128 : 0) + quarter * 32 + lane;   // pass 1: the query row this thread owns
         const float c = P.c;
+        uint32_t it = 0;
+        bool ok = true;
 
-        auto flush_partial = [&](int kv) {                      // pass 1: one (m, l) per row and group
-            const int row = ((nmb == 2) ? grp * 128 : 0) + quarter * 32 + lane;
-            if (row < P.R)
-                P.part[((size_t)kv * kSlots + 2 * blockIdx.x + grp) * P.R + row] = make_float2(m_run, (l0 + l1) + (l2 + l3));
-            m_run = -INFINITY; l0 = l1 = l2 = l3 = 0.f;
-        };
-
-        for (int n = 0; n < ntiles && ok; ++n) {
-            const int i = (PASS == 1) ? t_begin + n : t_end - 1 - n;
-            const int kv = P.h0 + i / P.tph, j0 = (i % P.tph) * kTile;
-            if (kv != prev_kv) {
-                if (PASS == 1) {
-                    if (seg >= 0) flush_partial(prev_kv);
-                } else {
-                    // stage the row normalisers M_r of the new head
-                    const int sb = (seg + 1) & 1;
-                    if (et < P.R) ctl->Ms[sb][et] = __ldcg(&P.Mrow[(size_t)kv * P.R + et]);
-                    mbar_arrive(&ctl->m_ready[sb]);
-                    if (!mbar_wait(&ctl->m_ready[sb], ((seg + 1) >> 1) & 1, ctl, P.status)) break;
-                }
-                prev_kv = kv; ++seg;
-            }
-            for (int mb = 0; mb < nmb; ++mb, ++unit) {
-                if ((int)(unit & 1) != grp) continue;
-                const uint32_t slot = unit % nslots;
-                if (!mbar_wait(&ctl->t_full[slot], (unit / nslots) & 1, ctl, P.status)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t taddr = lane_addr + slot * slot_cols;
-                uint32_t v[128];
-                if (PASS == 1) {
+        for (int s = 0; s < nseg; ++s) {
+            const Seg sg = segment(s, P);
+            const int ntiles = sg.t_end - sg.t_begin;
+            int prev_kv = -1;
+            if (sg.pass == 1) {
+                float m_run = -INFINITY, l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+                auto flush_partial = [&](int kv) {
+                    if (my_row < P.R && ok)
+                        P.part[((size_t)kv * kSlots + 2 * blockIdx.x + grp) * P.R + my_row] = make_float2(m_run, (l0 + l1) + (l2 + l3));
+                    m_run = -INFINITY; l0 = l1 = l2 = l3 = 0.f;
+                };
+                for (int n = 0; n < ntiles; ++n, ++it) {
+                    const int i = sg.t_begin + n;
+                    const int kv = sg.h0 + i / P.tph, j0 = (i % P.tph) * kTile;
+                    if (kv != prev_kv) {
+                        if (prev_kv >= 0) flush_partial(prev_kv);
+                        prev_kv = kv;
+                    }
+                    if (!wide && (int)(it & 1) != grp) continue;
+                    const uint32_t slot = it % nslots;
+                    if (ok) ok = mbar_wait(&ctl->t_full[slot], (it / nslots) & 1, ctl, P.status);
+                    if (!ok) continue;
+                    tc_fence_after();
+                    const uint32_t taddr = lane_addr + slot * slot_cols + (wide ? (uint32_t)grp * 128u : 0u);
+                    uint32_t v[128];
                     // the whole 128-key row segment in one tensor-memory read; the slot is free right after
                     JQ_TMEM_LD128(taddr, v);
                     tmem_ld_wait();
                     tc_fence_before();
-                    mbar_arrive(&ctl->t_empty[slot]);
+                    mbar_arrive(&ctl->t_empty[slot], 1);
                     const int valid = min(kTile, P.L - j0);
                     if (valid < kTile) {
 #pragma unroll
@@ -331,15 +413,43 @@ score_pass(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUt
                         l2 += ex2(fmaf(__uint_as_float(v[t + 2]), c, -mc));
                         l3 += ex2(fmaf(__uint_as_float(v[t + 3]), c, -mc));
                     }
-                } else {
-                    const float *Ms = ctl->Ms[seg & 1];
+                }
+                if (prev_kv >= 0) flush_partial(prev_kv);
+                // this CTA's share of pass 1 of the group is published: count it in
+                __threadfence();
+                epi_sync();
+                if (et == 0) atomicAdd(P.status + kWCnt1 + (sg.g & (kRing - 1)), 1);
+            } else {
+                if (et == 0 && ok)
+                    ok = wait_counter(P.status + kWCnt2 + (sg.g & (kRing - 1)), (sg.g / kRing + 1) * G, ctl, P.status);
+                for (int n = 0; n < ntiles; ++n, ++it) {
+                    const int i = sg.t_end - 1 - n;
+                    const int kv = sg.h0 + i / P.tph, j0 = (i % P.tph) * kTile;
+                    if (kv != prev_kv) {
+                        // stage the row normalisers M_r of the new head (all readers of the old ones are past them)
+                        epi_sync();
+                        if (et < P.R) ctl->Ms[et] = __ldcg(&P.Mrow[(size_t)kv * P.R + et]);
+                        epi_sync();
+                        if (*(volatile int *)&ctl->abort_flag) ok = false;
+                        prev_kv = kv;
+                    }
+                    if ((int)(it & 1) != grp) continue;
+                    const uint32_t slot = it % nslots;
+                    if (ok) ok = mbar_wait(&ctl->t_full[slot], (it / nslots) & 1, ctl, P.status);
+                    if (!ok) continue;
+                    tc_fence_after();
+                    const uint32_t taddr = lane_addr + slot * slot_cols;
+                    const uint32_t arrive_n = wide ? 2u : 1u;
+                    const float *Ms = ctl->Ms;
+                    const int Rpad = P.Rpad;
+                    uint32_t v[128];
                     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll 1
                     for (int c0 = 0; c0 < Rpad; c0 += 128) {
                         if (Rpad - c0 >= 128) {
                             JQ_TMEM_LD128(taddr + c0, v);
                             tmem_ld_wait();
-                            if (c0 + 128 >= Rpad) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot]); }
+                            if (c0 + 128 >= Rpad) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], arrive_n); }
                             const int nv = P.R - c0;             // columns that are real query rows
                             if (nv >= 128) {
 #pragma unroll
@@ -359,7 +469,7 @@ score_pass(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUt
                             for (int c1 = c0; c1 < Rpad; c1 += 32) {
                                 JQ_TMEM_LD32(taddr + c1, v);
                                 tmem_ld_wait();
-                                if (c1 + 32 >= Rpad) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot]); }
+                                if (c1 + 32 >= Rpad) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], arrive_n); }
                                 const int nv = P.R - c1;
                                 if (nv >= 32) {
 #pragma unroll
@@ -382,7 +492,46 @@ score_pass(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUt
                 }
             }
         }
-        if (PASS == 1 && seg >= 0 && ok) flush_partial(prev_kv);
+    } else {
+        // ---------------------------------------------------------------- grid-wide merge of the pass-1 partials
+        // Group g: once every CTA has published its partials, this CTA combines the rows b, b+G, b+2G, ...
+        // of the group (lanes over the contributing slots, then a butterfly: a fixed order, hence
+        // deterministic) into M_r = c*m_r + log2(l_r), and counts itself in.
+        const float c = P.c;
+        for (int g = 0; g < P.ngroups; ++g) {
+            int ok = 1;
+            if (lane == 0) ok = wait_counter(P.status + kWCnt1 + (g & (kRing - 1)), (g / kRing + 1) * G, ctl, P.status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            const int h0 = g * P.hpg, nh = min(P.hpg, P.Hkv - h0);
+            const long long T = (long long)nh * P.tph;
+            const int ng = (P.Rbox == 256) ? 1 : 2;
+            for (int item = blockIdx.x; item < nh * P.R; item += G) {
+                const int hl = item / P.R, r = item - hl * P.R, kv = h0 + hl;
+                const long long first = (long long)hl * P.tph;
+                const int b_lo = owner_of_tile(first, T, G), b_hi = owner_of_tile(first + P.tph - 1, T, G);
+                const int g0 = (P.Rbox == 256) ? (r >> 7) : 0;
+                const int nsl = (b_hi - b_lo + 1) * ng;
+                float m = -INFINITY, l = 0.f;
+                for (int i = lane; i < nsl; i += 32) {
+                    const int b = b_lo + i / ng, gg = g0 + i % ng;
+                    if ((long long)b * T / G == ((long long)b + 1) * T / G) continue;   // CTA b had no tile
+                    const float2 p = __ldcg(&P.part[((size_t)kv * kSlots + 2 * b + gg) * P.R + r]);
+                    merge_ml(m, l, p.x, p.y, c);
+                }
+#pragma unroll
+                for (int o = 16; o >= 1; o >>= 1) {
+                    const float m2 = __shfl_xor_sync(0xffffffffu, m, o), l2 = __shfl_xor_sync(0xffffffffu, l, o);
+                    merge_ml(m, l, m2, l2, c);
+                }
+                if (lane == 0) P.Mrow[(size_t)kv * P.R + r] = c * m + log2f(l);
+            }
+            __syncwarp();
+            if (lane == 0) {
+                __threadfence();
+                atomicAdd(P.status + kWCnt2 + (g & (kRing - 1)), 1);
+            }
+        }
     }
 
     // ---------------------------------------------------------------- common exit
@@ -394,48 +543,14 @@ score_pass(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUt
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
-}
-
-// Combines the per-CTA partial (m, l) of pass 1 into M_r = c*m_r + log2(l_r).  One warp per query
-// row, lanes over the partial slots, then a butterfly; the order is fixed, hence deterministic.
-// grid (ceil(R/8), nheads), block 256.
-__device__ __forceinline__ void merge_ml(float &m, float &l, float m2, float l2, float c)
-{
-    if (l2 > 0.f) {
-        if (l > 0.f) {
-            const float mn = fmaxf(m, m2);
-            l = l * ex2(c * (m - mn)) + l2 * ex2(c * (m2 - mn));
-            m = mn;
-        } else {
-            m = m2; l = l2;
+    if (threadIdx.x == 0) {
+        // the last CTA to leave clears the grid counters for the next call on this workspace
+        __threadfence();
+        if (atomicAdd(P.status + kWDone, 1) == G - 1) {
+            for (int i = 0; i < kRing; ++i) { P.status[kWCnt1 + i] = 0; P.status[kWCnt2 + i] = 0; }
+            P.status[kWDone] = 0;
         }
     }
-}
-
-__global__ void __launch_bounds__(256)
-merge_partials(const float2 *__restrict__ part, float *__restrict__ Mrow, int R, int Rbox, int h0, int tph,
-               int nheads, int G, float c)
-{
-    const int lane = threadIdx.x & 31, r = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (r >= R) return;
-    const int kv = h0 + blockIdx.y;
-    const long long T = (long long)nheads * tph, first = (long long)blockIdx.y * tph;
-    const int b_lo = owner_of_tile(first, T, G), b_hi = owner_of_tile(first + tph - 1, T, G);
-    const int ng = (Rbox == 256) ? 1 : 2, g0 = (Rbox == 256) ? (r >> 7) : 0;
-    const int nsl = (b_hi - b_lo + 1) * ng;
-    float m = -INFINITY, l = 0.f;
-    for (int i = lane; i < nsl; i += 32) {
-        const int b = b_lo + i / ng, g = g0 + i % ng;
-        if ((long long)b * T / G == ((long long)b + 1) * T / G) continue;   // CTA b had no tile
-        const float2 p = __ldcg(&part[((size_t)kv * kSlots + 2 * b + g) * R + r]);
-        merge_ml(m, l, p.x, p.y, c);
-    }
-#pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) {
-        const float m2 = __shfl_xor_sync(0xffffffffu, m, o), l2 = __shfl_xor_sync(0xffffffffu, l, o);
-        merge_ml(m, l, m2, l2, c);
-    }
-    if (lane == 0) Mrow[(size_t)kv * R + r] = c * m + log2f(l);
 }
 
 // ------------------------------------------------------------------ host side
@@ -473,8 +588,13 @@ bool make_map(CUtensorMap *map, const void *ptr, int rows, int heads, int box_ro
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+constexpr size_t smem_bytes(int Rbox, int stages)
+{
+    return 1024 + 2 * (size_t)Rbox * kD * 2 + (size_t)stages * kStageBytes + kCtlBytes;
+}
+
 struct DeviceInfo {
-    int sms = 0;
+    int sms = 0;        // CTAs of score_fused that can be resident at once (one per SM)
     long long l2 = 0;
     bool ready = false;
 };
@@ -488,17 +608,28 @@ bool device_info(DeviceInfo *out)
     std::lock_guard<std::mutex> lock(mu);
     DeviceInfo &d = info[dev];
     if (!d.ready) {
-        int l2 = 0;
-        if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+        int l2 = 0, sms = 0, coop = 0, per_sm = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
         if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess) return false;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return false;
+        const size_t smem = smem_bytes(256, 3) > smem_bytes(128, 5) ? smem_bytes(256, 3) : smem_bytes(128, 5);
+        if (cudaFuncSetAttribute(score_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, score_fused, kThreads, smem) != cudaSuccess || per_sm < 1)
+            return false;
+        d.sms = sms;
         d.l2 = l2;
-        const int smem = (int)(kCtlBytes + 1024 + 2 * 128 * kD * 2 + kStages * kStageBytes);
-        if (cudaFuncSetAttribute(score_pass<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
-        if (cudaFuncSetAttribute(score_pass<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
         d.ready = true;
     }
     *out = d;
     return true;
+}
+
+// Overrides for tuning runs (read once): JQ_SCORE_GROUP_MIB = K bytes per head group, JQ_SCORE_ORDER = 0
+// for the unpipelined segment order.
+long long env_ll(const char *name, long long dflt)
+{
+    const char *v = getenv(name);
+    return (v && *v) ? atoll(v) : dflt;
 }
 
 }  // namespace
@@ -508,31 +639,61 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
 {
     DeviceInfo dev;
     if (!device_info(&dev)) return JQ_ERR_CUDA;
+    static const long long group_mib = env_ll("JQ_SCORE_GROUP_MIB", 32);
+    static const long long order = env_ll("JQ_SCORE_ORDER", 1);
     const int R = s.group * s.w;
     Params P;
-    P.L = s.L; P.R = R; P.Rbox = R <= 128 ? 128 : 256;
+    P.L = s.L; P.R = R; P.Rbox = R <= 128 ? 128 : 256; P.Rpad = (R + 15) & ~15;
+    P.Hkv = s.Hkv;
     P.tph = (s.L + kTile - 1) / kTile;
+    P.stages = P.Rbox == 128 ? 5 : 3;
+    P.pipelined = order != 0;
     P.c = 1.4426950408889634f / sqrtf((float)s.d);
     P.part = w.part; P.Mrow = w.Mrow; P.scores = scores; P.status = w.status;
     CUtensorMap mapK, mapQ;
     if (!make_map(&mapK, K, s.L, s.Hkv, kTile) || !make_map(&mapQ, Q, R, s.Hkv, P.Rbox)) return JQ_ERR_CUDA;
-    const size_t smem = kCtlBytes + 1024 + (size_t)(P.Rbox == 128 ? 2 : 1) * P.Rbox * kD * 2 + (size_t)kStages * kStageBytes;
-    int grid = dev.sms;
-    if (2 * grid > kSlots) grid = kSlots / 2;
+
+    int sms = dev.sms;
+    if (2 * sms > kSlots) sms = kSlots / 2;
     // KV heads are scored in groups whose keys fit in a share of the L2, so that pass 2 finds them there.
+    // Among the admissible group sizes, take the one that wastes the fewest CTA-tile slots.
     const long long head_bytes = (long long)s.L * kD * 2;
-    long long per_group = (dev.l2 / 2) / head_bytes;
-    if (per_group < 1) per_group = 1;
-    const long long ngroups = (s.Hkv + per_group - 1) / per_group;
-    per_group = (s.Hkv + ngroups - 1) / ngroups;       // even split
-    for (int h0 = 0; h0 < s.Hkv; h0 += (int)per_group) {
-        P.h0 = h0;
-        P.nheads = (int)(h0 + per_group <= s.Hkv ? per_group : s.Hkv - h0);
-        score_pass<1><<<grid, kThreads, smem, st>>>(mapK, mapQ, P);
-        merge_partials<<<dim3((R + 7) / 8, P.nheads), 256, 0, st>>>(w.part, w.Mrow, R, P.Rbox, h0, P.tph, P.nheads, grid, P.c);
-        score_pass<2><<<grid, kThreads, smem, st>>>(mapK, mapQ, P);
-        count_launch(3);
+    long long hmax = (group_mib << 20) / head_bytes;
+    if (hmax < 1) hmax = 1;
+    if (hmax > s.Hkv) hmax = s.Hkv;
+    int best_hpg = 1;
+    double best_eff = -1.0;
+    for (int hpg = 1; hpg <= (int)hmax; ++hpg) {
+        long long work = 0, slots = 0;
+        for (int h0 = 0; h0 < s.Hkv; h0 += hpg) {
+            const long long T = (long long)(h0 + hpg <= s.Hkv ? hpg : s.Hkv - h0) * P.tph;
+            work += T;
+            slots += (T + sms - 1) / sms;
+        }
+        const double eff = (double)work / ((double)slots * sms);
+        if (eff >= best_eff - 1e-9) { best_eff = eff > best_eff ? eff : best_eff; best_hpg = hpg; }
+        if (hmax > 64 && hpg >= 64) break;   // the scan is only worth it over a small range
     }
+    P.hpg = best_hpg;
+    P.ngroups = (s.Hkv + P.hpg - 1) / P.hpg;
+    long long tmax = (long long)(P.hpg < s.Hkv ? P.hpg : s.Hkv) * P.tph;
+    const int grid = (int)(tmax < sms ? tmax : sms);
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_bytes(P.Rbox, P.stages);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, score_fused, mapK, mapQ, P) != cudaSuccess) {
+        cudaGetLastError();
+        return JQ_ERR_CUDA;
+    }
+    count_launch(1);
     return check_launch();
 }
 
