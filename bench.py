@@ -228,24 +228,27 @@ def run_ours(args):
     launches = jq.launch_count() - n0
     assert jq.last_device_status(ws) == jq.JQ_OK, "device status not ok"
 
-    # per-stage times through the stage entry points (events on the launching stream)
-    scores = torch.empty((wl.Hkv, wl.L), dtype=torch.float32, device="cuda")
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    # per-stage times through the stage entry points: batches of back-to-back calls between events on the
+    # launching stream, so that host launch latency is not counted as device time
+    scores = [torch.empty((wl.Hkv, wl.L), dtype=torch.float32, device="cuda") for _ in range(min(distinct, 4))]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    nb = max(distinct, 8)
     stage_ms = np.zeros(3)
-    reps = max(args.steps, 5) * min(layers, 8)
-    for rep in range(reps + 3):
-        j = rep % distinct
-        ev[0].record(stream)
-        jq.score(Ks[j], Qs[j], s, scores, ws, stream=stream)
-        ev[1].record(stream)
-        jq.select_topk(scores, s, idx, ws, stream=stream)
-        ev[2].record(stream)
-        jq.compact_kv(Ks[j], Vs[j], idx, s, Ko, Vo, stream=stream)
-        ev[3].record(stream)
+
+    def timed(fn):
+        for j in range(3):
+            fn(j % distinct)
         torch.cuda.synchronize()
-        if rep >= 3:
-            stage_ms += [ev[k].elapsed_time(ev[k + 1]) for k in range(3)]
-    stage_ms /= reps
+        ev[0].record(stream)
+        for j in range(nb):
+            fn(j % distinct)
+        ev[1].record(stream)
+        torch.cuda.synchronize()
+        return ev[0].elapsed_time(ev[1]) / nb
+
+    stage_ms[0] = timed(lambda j: jq.score(Ks[j], Qs[j], s, scores[j % len(scores)], ws, stream=stream))
+    stage_ms[1] = timed(lambda j: jq.select_topk(scores[j % len(scores)], s, idx, ws, stream=stream))
+    stage_ms[2] = timed(lambda j: jq.compact_kv(Ks[j], Vs[j], idx, s, Ko, Vo, stream=stream))
     clocks = sampler.stop() if sampler else None
 
     t = torch.tensor([ms], dtype=torch.float64, device="cuda")

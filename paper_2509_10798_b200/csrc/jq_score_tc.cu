@@ -191,6 +191,34 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
+
+// acc (two lanes) += exp2(v * c + b) for two accumulator columns, on packed fp32 pairs.
+__device__ __forceinline__ void exp_acc2(float2 &acc, uint32_t v0, uint32_t v1, float2 cc, float2 b)
+{
+    const float2 x = __ffma2_rn(make_float2(__uint_as_float(v0), __uint_as_float(v1)), cc, b);
+    acc = __fadd2_rn(acc, make_float2(ex2(x.x), ex2(x.y)));
+}
+
+// Largest of the 128 values of a row segment.
+__device__ __forceinline__ float max128(const uint32_t (&v)[128])
+{
+    float c0 = -INFINITY, c1 = -INFINITY, c2 = -INFINITY, c3 = -INFINITY;
+#pragma unroll
+    for (int t = 0; t < 128; t += 8) {
+        c0 = max3(c0, __uint_as_float(v[t + 0]), __uint_as_float(v[t + 1]));
+        c1 = max3(c1, __uint_as_float(v[t + 2]), __uint_as_float(v[t + 3]));
+        c2 = max3(c2, __uint_as_float(v[t + 4]), __uint_as_float(v[t + 5]));
+        c3 = max3(c3, __uint_as_float(v[t + 6]), __uint_as_float(v[t + 7]));
+    }
+    return fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));
+}
+
 // Which CTA owns tile t when T tiles are split contiguously over G CTAs as [b*T/G, (b+1)*T/G).
 __device__ __forceinline__ int owner_of_tile(long long t, long long T, long long G)
 {
@@ -363,11 +391,18 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             const int ntiles = sg.t_end - sg.t_begin;
             int prev_kv = -1;
             if (sg.pass == 1) {
-                float m_run = -INFINITY, l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+                // l = sum_j exp2(c (s_j - m_run)) against a REFERENCE m_run that need not be the row max: it
+                // is the max of the first tile seen and is only raised when a later tile would push the sum
+                // towards overflow (the tile is then redone from its registers).  Any reference gives the
+                // same M_r = c m + log2(l) after the merge.
+                float m_run = -INFINITY;
+                float2 l01 = make_float2(0.f, 0.f), l23 = make_float2(0.f, 0.f);
                 auto flush_partial = [&](int kv) {
                     if (my_row < P.R && ok)
-                        P.part[((size_t)kv * kSlots + 2 * blockIdx.x + grp) * P.R + my_row] = make_float2(m_run, (l0 + l1) + (l2 + l3));
-                    m_run = -INFINITY; l0 = l1 = l2 = l3 = 0.f;
+                        P.part[((size_t)kv * kSlots + 2 * blockIdx.x + grp) * P.R + my_row] =
+                            make_float2(m_run, (l01.x + l01.y) + (l23.x + l23.y));
+                    m_run = -INFINITY;
+                    l01 = l23 = make_float2(0.f, 0.f);
                 };
                 for (int n = 0; n < ntiles; ++n, ++it) {
                     const int i = sg.t_begin + n;
@@ -393,25 +428,29 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll
                         for (int t = 0; t < 128; ++t) if (t >= valid) v[t] = 0xff800000u;   // -inf: not a key
                     }
-                    float c0 = -INFINITY, c1 = -INFINITY, c2 = -INFINITY, c3 = -INFINITY;
+                    if (m_run == -INFINITY) m_run = max128(v);
+                    const float2 keep01 = l01, keep23 = l23;
+                    const float2 cc = make_float2(c, c);
+                    float2 mb = make_float2(-m_run * c, -m_run * c);
 #pragma unroll
                     for (int t = 0; t < 128; t += 4) {
-                        c0 = fmaxf(c0, __uint_as_float(v[t + 0])); c1 = fmaxf(c1, __uint_as_float(v[t + 1]));
-                        c2 = fmaxf(c2, __uint_as_float(v[t + 2])); c3 = fmaxf(c3, __uint_as_float(v[t + 3]));
+                        exp_acc2(l01, v[t + 0], v[t + 1], cc, mb);
+                        exp_acc2(l23, v[t + 2], v[t + 3], cc, mb);
                     }
-                    const float cm = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));
-                    if (cm > m_run) {
+                    const float lsum = (l01.x + l01.y) + (l23.x + l23.y);
+                    if (!(lsum < 1.0e30f)) {
+                        // the reference is too far below this tile's values: raise it to the tile max and redo the tile
+                        const float cm = fmaxf(max128(v), m_run);
                         const float f = ex2(c * (m_run - cm));
-                        l0 *= f; l1 *= f; l2 *= f; l3 *= f;
+                        l01 = make_float2(keep01.x * f, keep01.y * f);
+                        l23 = make_float2(keep23.x * f, keep23.y * f);
                         m_run = cm;
-                    }
-                    const float mc = m_run * c;
+                        mb = make_float2(-m_run * c, -m_run * c);
 #pragma unroll
-                    for (int t = 0; t < 128; t += 4) {
-                        l0 += ex2(fmaf(__uint_as_float(v[t + 0]), c, -mc));
-                        l1 += ex2(fmaf(__uint_as_float(v[t + 1]), c, -mc));
-                        l2 += ex2(fmaf(__uint_as_float(v[t + 2]), c, -mc));
-                        l3 += ex2(fmaf(__uint_as_float(v[t + 3]), c, -mc));
+                        for (int t = 0; t < 128; t += 4) {
+                            exp_acc2(l01, v[t + 0], v[t + 1], cc, mb);
+                            exp_acc2(l23, v[t + 2], v[t + 3], cc, mb);
+                        }
                     }
                 }
                 if (prev_kv >= 0) flush_partial(prev_kv);
@@ -428,7 +467,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     if (kv != prev_kv) {
                         // stage the row normalisers M_r of the new head (all readers of the old ones are past them)
                         epi_sync();
-                        if (et < P.R) ctl->Ms[et] = __ldcg(&P.Mrow[(size_t)kv * P.R + et]);
+                        if (et < P.R) ctl->Ms[et] = -__ldcg(&P.Mrow[(size_t)kv * P.R + et]);   // stored negated: x = c s + (-M_r)
                         epi_sync();
                         if (*(volatile int *)&ctl->abort_flag) ok = false;
                         prev_kv = kv;
@@ -443,7 +482,8 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     const float *Ms = ctl->Ms;
                     const int Rpad = P.Rpad;
                     uint32_t v[128];
-                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+                    float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
+                    const float2 cc = make_float2(c, c);
 #pragma unroll 1
                     for (int c0 = 0; c0 < Rpad; c0 += 128) {
                         if (Rpad - c0 >= 128) {
@@ -455,14 +495,12 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll
                                 for (int t = 0; t < 128; t += 4) {
                                     const float4 mm = *(const float4 *)(Ms + c0 + t);
-                                    a0 += ex2(fmaf(__uint_as_float(v[t + 0]), c, -mm.x));
-                                    a1 += ex2(fmaf(__uint_as_float(v[t + 1]), c, -mm.y));
-                                    a2 += ex2(fmaf(__uint_as_float(v[t + 2]), c, -mm.z));
-                                    a3 += ex2(fmaf(__uint_as_float(v[t + 3]), c, -mm.w));
+                                    exp_acc2(a01, v[t + 0], v[t + 1], cc, make_float2(mm.x, mm.y));
+                                    exp_acc2(a23, v[t + 2], v[t + 3], cc, make_float2(mm.z, mm.w));
                                 }
                             } else {
 #pragma unroll
-                                for (int t = 0; t < 128; ++t) if (t < nv) a0 += ex2(fmaf(__uint_as_float(v[t]), c, -Ms[c0 + t]));
+                                for (int t = 0; t < 128; ++t) if (t < nv) a01.x += ex2(fmaf(__uint_as_float(v[t]), c, Ms[c0 + t]));
                             }
                         } else {
 #pragma unroll 1
@@ -475,20 +513,18 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll
                                     for (int t = 0; t < 32; t += 4) {
                                         const float4 mm = *(const float4 *)(Ms + c1 + t);
-                                        a0 += ex2(fmaf(__uint_as_float(v[t + 0]), c, -mm.x));
-                                        a1 += ex2(fmaf(__uint_as_float(v[t + 1]), c, -mm.y));
-                                        a2 += ex2(fmaf(__uint_as_float(v[t + 2]), c, -mm.z));
-                                        a3 += ex2(fmaf(__uint_as_float(v[t + 3]), c, -mm.w));
+                                        exp_acc2(a01, v[t + 0], v[t + 1], cc, make_float2(mm.x, mm.y));
+                                        exp_acc2(a23, v[t + 2], v[t + 3], cc, make_float2(mm.z, mm.w));
                                     }
                                 } else {
 #pragma unroll
-                                    for (int t = 0; t < 32; ++t) if (t < nv) a0 += ex2(fmaf(__uint_as_float(v[t]), c, -Ms[c1 + t]));
+                                    for (int t = 0; t < 32; ++t) if (t < nv) a01.x += ex2(fmaf(__uint_as_float(v[t]), c, Ms[c1 + t]));
                                 }
                             }
                         }
                     }
                     const int key = j0 + quarter * 32 + lane;
-                    if (key < P.L) P.scores[(size_t)kv * P.L + key] = (a0 + a1) + (a2 + a3);
+                    if (key < P.L) P.scores[(size_t)kv * P.L + key] = (a01.x + a01.y) + (a23.x + a23.y);
                 }
             }
         }

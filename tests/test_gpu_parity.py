@@ -73,6 +73,22 @@ def test_score_large_logits_do_not_overflow():
     assert_scores_close(got, oracle.score(K, Qs))
 
 
+def test_score_rising_logits_raise_the_running_reference():
+    """Keys whose logits climb by hundreds from tile to tile: pass 1 must raise its reference and stay exact."""
+    wl = small_wl(1, 2, 8, 1500, 1)
+    rng = np.random.default_rng(5)
+    u = rng.standard_normal(128).astype(np.float32)
+    u /= np.linalg.norm(u)
+    ramp = np.linspace(-40.0, 40.0, wl.L, dtype=np.float32)[:, None]
+    Kf = ramp * u[None, :] + 0.1 * rng.standard_normal((wl.L, 128)).astype(np.float32)
+    Qf = 300.0 * u[None, None, :] + rng.standard_normal((wl.Hq, wl.w, 128)).astype(np.float32)
+    K, Q = W.bf16_bits(Kf[None]), W.bf16_bits(Qf)
+    got = gpu_score(K, Q, shape_of(wl))
+    assert np.all(np.isfinite(got))
+    assert_scores_close(got, oracle.score(K, Q))
+    np.testing.assert_allclose(got.sum(-1), wl.R, rtol=1e-3)
+
+
 # ------------------------------------------------------------------ pool + select (steps 4-5), bit-exact
 
 SELECT_CASES = [(1, 1, 1, 7), (1, 5, 9, 7), (2, 6, 3, 7), (2, 64, 64, 7), (3, 257, 40, 7), (2, 1000, 333, 3),
