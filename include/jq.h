@@ -90,6 +90,27 @@ jq_status jq_score(const void *K, const void *Qwin, const jq_shape *shape, float
                    void *ws, size_t ws_bytes, jq_stream_t stream);
 
 /*
+ * jq_score for callers that cannot allocate device memory: an inference server that has handed every
+ * free byte of the GPU to its KV-cache pool, a plug-in running inside somebody else's memory budget, a
+ * call site that must not touch the allocator.  (The paper has no counterpart; this is a property of
+ * the library.)  Same inputs, same output and the same kernel as jq_score, but no workspace argument:
+ * the scratch the kernel needs sits in a device array built into the library, about 5.3 MB that every
+ * GPU using the library holds until the process exits.
+ *  - Limit: Hkv * group * w <= 2048 query rows in total; a larger shape returns JQ_ERR_UNSUPPORTED and
+ *    launches nothing.
+ *  - The call allocates and frees nothing (no cudaMalloc, cudaFree or allocating library routine).
+ *    Its first call on a device looks up the array's device address; make that first call outside any
+ *    stream capture.
+ *  - All calls share the one array, and it keeps the previous call's contents (the part that must start
+ *    from zero is cleared on `stream` by every call).  Calls whose work can overlap on the GPU, from
+ *    different streams or threads, race on it: keep them on one stream, or order them yourself.
+ *  - A bounded device-side wait that runs out leaves its record inside the array, where
+ *    jq_last_device_status cannot see it; callers that need that status use jq_score.
+ */
+jq_status jq_score_static(const void *K, const void *Qwin, const jq_shape *shape, float *scores,
+                          jq_stream_t stream);
+
+/*
  * The same scores computed with plain fp32 FMA on the CUDA cores.  A comparator for profiling the
  * tensor-core path against (the contraction is small and of low arithmetic intensity per key);
  * never used by jq_evict_layer.

@@ -17,6 +17,7 @@ EXPORTS = (
     "jq_workspace_bytes", "jq_workspace_init", "jq_num_kept", "jq_check_shape", "jq_score",
     "jq_score_fma", "jq_select_topk", "jq_compact_kv", "jq_evict_layer", "jq_host_call_bytes",
     "jq_evict_layer_host", "jq_last_device_status", "jq_launch_count", "jq_status_string",
+    "jq_score_static",
 )
 
 
@@ -54,6 +55,7 @@ def lib():
         L.jq_workspace_init.argtypes = [vp, sz, vp]
         L.jq_score.argtypes = [vp, vp, sp, vp, vp, sz, vp]
         L.jq_score_fma.argtypes = [vp, vp, sp, vp, vp, sz, vp]
+        L.jq_score_static.argtypes = [vp, vp, sp, vp, vp]
         L.jq_select_topk.argtypes = [vp, sp, vp, vp, vp, sz, vp]
         L.jq_compact_kv.argtypes = [vp, vp, vp, sp, vp, vp, vp]
         L.jq_evict_layer.argtypes = [vp, vp, vp, sp, vp, vp, vp, vp, sz, vp]
@@ -135,6 +137,14 @@ def score(K, Qwin, s, scores, ws, stream=None, fma=False):
     fn = lib().jq_score_fma if fma else lib().jq_score
     _raise("jq_score_fma" if fma else "jq_score",
            fn(_ptr(K), _ptr(Qwin), ctypes.byref(s), _ptr(scores), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def score_static(K, Qwin, s, scores, stream=None):
+    """jq_score without a workspace, for callers that may not allocate device memory: the scratch is a
+    fixed array inside the library (at most 2048 query rows over all KV heads; calls share it, so keep
+    them on one stream)."""
+    _raise("jq_score_static",
+           lib().jq_score_static(_ptr(K), _ptr(Qwin), ctypes.byref(s), _ptr(scores), _stream(stream)))
 
 
 def select_topk(scores, s, kept_idx, ws, pooled=None, stream=None):
