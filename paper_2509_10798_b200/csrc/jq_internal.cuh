@@ -8,7 +8,7 @@ namespace jq {
 
 constexpr int kD = 128;          // head dimension the kernels are built for
 constexpr int kMaxR = 256;       // query rows per KV head (group * w)
-constexpr int kSlots = 320;      // partial (max, sum-exp) slots per KV head in the workspace (2 per CTA)
+constexpr int kSlots = 640;      // partial (reference, sum-exp) slots per KV head in the workspace (up to 4 per CTA)
 constexpr int kStatusWords = 64; // first 256 bytes of the workspace
 
 // Device status word values (sticky since jq_workspace_init): 0 ok, else a jq_status.

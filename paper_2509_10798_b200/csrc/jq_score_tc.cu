@@ -2,30 +2,40 @@
 //
 // The grid is one CTA per SM, launched cooperatively (all CTAs are resident, so they may wait on one
 // another).  A CTA is warp-specialised:
-//   warp 0      TMA producer: K tiles of 128 keys (two 64-column halves, 128-byte swizzle) into a
-//               ring of shared-memory stages; the query rows of a KV head into one of two stationary buffers;
-//   warp 1      issues tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory) and owns the TMEM allocation;
-//   warps 2-9   two epilogue groups of 128 threads that read accumulators with tcgen05.ld;
-//   warp 10     merges the per-CTA partial row statistics of pass 1 across the grid.
+//   warp 0        TMA producer: K tiles of 128 keys (two 64-column halves, 128-byte swizzle) into a ring of
+//                 shared-memory stages; the query rows of a KV head into one of two stationary buffers;
+//   warp 1        issues tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory) and owns the TMEM allocation;
+//   warps 2..     kGroups epilogue groups of 128 threads.  Accumulator block u (128 TMEM lanes x 128
+//                 columns) sits in slot u % 4 and is taken by group u % kGroups, 32 columns at a time;
+//   then          one warp that merges the per-warp partial row statistics of pass 1 across the grid,
+//                 and one that stages the merged row normalisers of the next KV head of pass 2.
 // The operand roles are swapped between the passes so that no reduction crosses threads:
-//   pass 1  S[R x 128] = Q K^T   (A = query rows, M = 128): a thread owns a QUERY ROW and keeps its
-//           running max m and sum l = sum_j exp2(c (s_j - m)); per-CTA partial (m, l) go to the workspace;
-//   pass 2  S^T[128 x R] = K Q^T (A = key tile, N = R):     a thread owns a KEY and adds
-//           exp2(c s - M_r) over the R rows, M_r = c m_r + log2(l_r) merged from the partials.
+//   pass 1  S[128 x 128] = Q K^T  (A = a block of 128 query rows): a thread owns a QUERY ROW and keeps
+//           l = sum_j exp2(c (s_j - m)) against a reference m; per-warp partial (m, l) go to the workspace;
+//   pass 2  S^T[128 x N] = K Q^T  (A = key tile, B = a block of up to 128 query rows): a thread owns a KEY
+//           and adds exp2(c s - M_r) over the rows, M_r = c m_r + log2(l_r) merged from the partials.
+//           With more than 128 query rows a key gets two blocks, added into the scores with red.add
+//           (two commutative additions onto zero: the result does not depend on their order).
+// A share of the exponentials can be evaluated on the FMA pipe (round, degree-4 polynomial on
+// [-1/2, 1/2], exponent insertion) because the ex2 unit, at 16 results per clock per SM, is the binding unit.
 //
 // KV heads are taken in groups whose keys fit in a share of the L2.  The tiles of a group are split
 // statically and contiguously over the CTAs, the same split in both passes, and pass 2 walks its range
 // backwards, so a CTA re-reads what it read itself, most recent first.  The segments are ordered
 //   P1(0) P1(1) P2(0) P1(2) P2(1) ... P2(last)
-// so that the grid-wide merge of group g (counter -> merge warp -> counter) happens while every CTA is busy
-// with pass 1 of group g+1; only the epilogue warps ever wait for it, and normally find it done.
+// so that the grid-wide merge of group g (counter -> merge warps -> counter) happens while every CTA is
+// busy with pass 1 of group g+1.
 //
 // Grid-wide counters live in the status block at the head of the workspace (zeroed by
 // jq_workspace_init): a ring of four per kind, with cumulative targets, reset by the last CTA to
 // leave.  Every wait (mbarrier or counter) is bounded: when one runs out, the CTA records
-// JQ_ERR_TIMEOUT in the status word, raises a CTA-wide abort flag that every other wait polls, runs
-// through its remaining barriers without touching data, and leaves through the common exit (which
+// JQ_ERR_TIMEOUT in the status word and raises a CTA-wide abort flag that every other wait polls; all
+// roles then run out of their loops without touching data and leave through the common exit (which
 // frees the tensor memory).
+//
+// The code is kept small on purpose (rolled loops over 32-column pieces, one copy of each block routine,
+// 32-bit index arithmetic, no division per tile): the roles run different code on one SM, and what falls
+// out of the instruction cache costs hundreds of cycles at every turn of the outer loops.
 #include "jq_internal.cuh"
 #include "jq_tmem_ld.cuh"
 #include <cuda.h>
@@ -36,25 +46,52 @@
 namespace jq {
 namespace {
 
+// Optional per-warp cycle accounting (compiled in with -DJQ_TRACE, for tuning only): every role adds the
+// cycles it spends in each kind of wait or work to sixteen counters and writes them out on exit.
+#ifdef JQ_TRACE
+#define TR_DECL long long tr_[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}; const long long tr_start_ = clock64(); long long tr_t_ = tr_start_
+#define TR_ADD(i) do { const long long n_ = clock64(); tr_[i] += n_ - tr_t_; tr_t_ = n_; } while (0)
+#define TR_DUMP do { tr_[15] = clock64() - tr_start_; if (P.trace && lane == 0) for (int k_ = 0; k_ < 16; ++k_) P.trace[((size_t)blockIdx.x * 32 + warp) * 16 + k_] = tr_[k_]; } while (0)
+#else
+#define TR_DECL
+#define TR_ADD(i)
+#define TR_DUMP
+#endif
+
+#ifndef JQ_GROUPS
+#define JQ_GROUPS 3
+#endif
+#ifndef JQ_POLY_OF8
+#define JQ_POLY_OF8 2
+#endif
+
 constexpr int kTile = 128;                       // keys per tile
 constexpr int kMaxStages = 5;                    // K ring depth (5 when R <= 128, 3 above)
-constexpr int kThreads = 352;                    // 11 warps
+constexpr int kGroups = JQ_GROUPS;               // epilogue groups of 128 threads
+constexpr int kTSlots = 4;                       // accumulator slots in tensor memory
+constexpr int kEpiWarps = 4 * kGroups;
+constexpr int kMergeWarp = 2 + kEpiWarps, kStageWarp = kMergeWarp + 1;
+constexpr int kThreads = (kStageWarp + 1) * 32;
 constexpr uint32_t kHalfBytes = kTile * 128;     // one 64-column half of a K tile (128-byte rows)
 constexpr uint32_t kStageBytes = 2 * kHalfBytes; // 32 KiB
-constexpr uint32_t kCtlBytes = 2048;             // barriers, flags, M_r
+constexpr uint32_t kCtlBytes = 3072;             // barriers, flags, M_r
 constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kSlotCols = kTmemCols / kTSlots;
 constexpr long long kWaitCycles = 4000000000ll;  // about 2 s of SM clock per wait
 constexpr int kRing = 4;                         // grid counters per kind
+constexpr int kPolyOf8 = JQ_POLY_OF8;            // of every 8 pairs of exponentials, this many go to the FMA pipe
 // words of the workspace status block
 constexpr int kWStatus = 0, kWDone = 1, kWCnt1 = 8, kWCnt2 = 12;
+static_assert(kSlots >= kGroups * 148, "one partial slot per epilogue group and CTA");
 
 struct Ctl {
     uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t q_full[2], q_empty[2];
-    uint64_t t_full[4], t_empty[4];
+    uint64_t t_full[kTSlots], t_empty[kTSlots];
+    uint64_t ms_full[2], ms_empty[2];
     uint32_t tmem_base;
     int abort_flag;
-    alignas(16) float Ms[kMaxR];   // read as float4
+    alignas(16) float Ms[2][kMaxR];   // -M_r of the KV head being scored in pass 2, double-buffered; read as float4
 };
 static_assert(offsetof(Ctl, Ms) % 16 == 0, "Ms must be 16-byte aligned");
 static_assert(sizeof(Ctl) <= kCtlBytes, "control block too large");
@@ -70,6 +107,9 @@ struct Params {
     float *Mrow;             // [Hkv][R]   c*m + log2(l) per query row
     float *scores;           // [Hkv][L]
     int *status;             // status block (kStatusWords ints)
+#ifdef JQ_TRACE
+    long long *trace;
+#endif
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -141,9 +181,6 @@ __device__ __noinline__ bool wait_counter(const int *p, int target, Ctl *ctl, in
     }
 }
 
-// Barrier among the 256 epilogue threads only.
-__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2)
 {
     asm volatile(
@@ -157,23 +194,6 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint64_t *bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
-// D[tmem] (+)= A[smem] * B[smem]^T, both operands K-major bf16, fp32 accumulate.
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-// Shared-memory matrix descriptor: K-major, 128-byte swizzle, rows of 128 bytes, 8-row groups 1024
-// bytes apart (stride byte offset), leading byte offset 16 (unused for swizzled K-major), version 1.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
-{
-    return (uint64_t)((addr >> 4) & 0x3fffu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, shape M x N.
@@ -198,41 +218,131 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     return y;
 }
 
-// acc (two lanes) += exp2(v * c + b) for two accumulator columns, on packed fp32 pairs.
-__device__ __forceinline__ void exp_acc2(float2 &acc, uint32_t v0, uint32_t v1, float2 cc, float2 b)
-{
-    const float2 x = __ffma2_rn(make_float2(__uint_as_float(v0), __uint_as_float(v1)), cc, b);
-    acc = __fadd2_rn(acc, make_float2(ex2(x.x), ex2(x.y)));
-}
 
-// Largest of the 128 values of a row segment.
-__device__ __forceinline__ float max128(const uint32_t (&v)[128])
+// Shared-memory matrix descriptor: K-major, 128-byte swizzle, rows of 128 bytes, 8-row groups 1024
+// bytes apart (stride byte offset), leading byte offset 16 (unused for swizzled K-major), version 1.
+// Only the low word depends on the address (in 16-byte units); the high word is a constant.
+constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr) { return ((addr >> 4) & 0x3fffu) | (1u << 16); }
+
+// One accumulator block: D[tmem] = A[smem] * B[smem]^T over the whole head dimension (8 steps of 16),
+// both operands K-major bf16 in two 64-column halves `a_half` / `b_half` bytes apart, fp32 accumulate.
+// A single straight-line sequence: the issuing thread shares its scheduler with epilogue warps, so
+// every instruction it does not execute is time the tensor pipe does not wait.
+__device__ __forceinline__ void tc_mma_block(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_half,
+                                             uint32_t b_half, uint32_t idesc)
 {
-    float c0 = -INFINITY, c1 = -INFINITY, c2 = -INFINITY, c3 = -INFINITY;
-#pragma unroll
-    for (int t = 0; t < 128; t += 8) {
-        c0 = max3(c0, __uint_as_float(v[t + 0]), __uint_as_float(v[t + 1]));
-        c1 = max3(c1, __uint_as_float(v[t + 2]), __uint_as_float(v[t + 3]));
-        c2 = max3(c2, __uint_as_float(v[t + 4]), __uint_as_float(v[t + 5]));
-        c3 = max3(c3, __uint_as_float(v[t + 6]), __uint_as_float(v[t + 7]));
-    }
-    return fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));
+    const uint32_t a1 = a_lo + (a_half >> 4), b1 = b_lo + (b_half >> 4);
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pz, po;\n\t"
+        ".reg .b64 da, db;\n\t"
+        ".reg .b32 ta, tb;\n\t"
+        "setp.ne.u32 pz, %0, %0;\n\t"
+        "setp.eq.u32 po, %0, %0;\n\t"
+        "mov.b64 da, {%1, %5};\n\t mov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, pz;\n\t"
+        "add.u32 ta, %1, 2;\n\t add.u32 tb, %2, 2;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "add.u32 ta, %1, 4;\n\t add.u32 tb, %2, 4;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "add.u32 ta, %1, 6;\n\t add.u32 tb, %2, 6;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "mov.b64 da, {%3, %5};\n\t mov.b64 db, {%4, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "add.u32 ta, %3, 2;\n\t add.u32 tb, %4, 2;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "add.u32 ta, %3, 4;\n\t add.u32 tb, %4, 4;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "add.u32 ta, %3, 6;\n\t add.u32 tb, %4, 6;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(a1), "r"(b1), "r"(kDescHi), "r"(idesc) : "memory");
 }
 
 // Which CTA owns tile t when T tiles are split contiguously over G CTAs as [b*T/G, (b+1)*T/G).
-__device__ __forceinline__ int owner_of_tile(long long t, long long T, long long G)
+// (T * G stays far below 2^32: a group has at most 2^17 tiles and the grid at most 160 CTAs.)
+__device__ __forceinline__ int owner_of_tile(uint32_t t, uint32_t T, uint32_t G)
 {
     return (int)(((t + 1) * G - 1) / T);
+}
+
+// Whether CTA b gets a tile at all when T < G tiles are split over G CTAs (rare; kept out of line).
+__device__ __noinline__ bool cta_has_tile(uint32_t b, uint32_t T, uint32_t G) { return b * T / G != (b + 1) * T / G; }
+
+// ------------------------------------------------------------------ exponentials
+
+// exp2 of a pair on the FMA pipe.  x is clamped to [-126, 127] (so that the exponent insertion cannot
+// wrap; 2^-126 stands in for anything smaller), split into n = round(x) and r = x - n in [-1/2, 1/2]
+// by the add-a-large-constant trick, 2^r comes from a degree-4 polynomial (relative error < 3e-6,
+// a least-maximum fit of 2^r on that interval) and n is added into the exponent field.
+__device__ __forceinline__ float2 exp2_fma_pair(float2 x)
+{
+    const float kMagic = 12582912.f;   // 1.5 * 2^23: x + kMagic holds round(x) in its low mantissa bits
+    x.x = fminf(fmaxf(x.x, -126.f), 127.f);
+    x.y = fminf(fmaxf(x.y, -126.f), 127.f);
+    const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
+    const float2 nn = __ffma2_rn(t, make_float2(-1.f, -1.f), make_float2(kMagic, kMagic));   // -round(x)
+    const float2 r = __fadd2_rn(x, nn);
+    float2 p = __ffma2_rn(make_float2(0.009570101276040077f, 0.009570101276040077f), r,
+                          make_float2(0.05591785907745361f, 0.05591785907745361f));
+    p = __ffma2_rn(p, r, make_float2(0.240247443318367f, 0.240247443318367f));
+    p = __ffma2_rn(p, r, make_float2(0.6931217908859253f, 0.6931217908859253f));
+    p = __ffma2_rn(p, r, make_float2(0.9999992847442627f, 0.9999992847442627f));
+    return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23)),
+                       __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23)));
+}
+
+// acc += exp2(v * c + b) for two values; POLY picks the pipe.
+template <bool POLY>
+__device__ __forceinline__ void exp_acc2(float2 &acc, uint32_t v0, uint32_t v1, float2 cc, float2 b)
+{
+    const float2 x = __ffma2_rn(make_float2(__uint_as_float(v0), __uint_as_float(v1)), cc, b);
+    acc = __fadd2_rn(acc, POLY ? exp2_fma_pair(x) : make_float2(ex2(x.x), ex2(x.y)));
+}
+
+// 32 values, value t against bias[t] (shared memory, or a register array holding one bias 32 times
+// would waste registers: pass 1 passes a pointer to a 4-float broadcast instead, see STRIDE).
+// STRIDE = 1: bias[t]; STRIDE = 0: the same 4 floats for every quad.
+template <int STRIDE>
+__device__ __forceinline__ void exp_acc32(float2 &a0, float2 &a1, const uint32_t (&v)[32], float2 cc, const float4 *bias)
+{
+#pragma unroll
+    for (int t = 0; t < 32; t += 16) {
+        const float4 b0 = bias[STRIDE * (t / 4)], b1 = bias[STRIDE * (t / 4 + 1)];
+        const float4 b2 = bias[STRIDE * (t / 4 + 2)], b3 = bias[STRIDE * (t / 4 + 3)];
+        exp_acc2<(kPolyOf8 > 0)>(a0, v[t + 0], v[t + 1], cc, make_float2(b0.x, b0.y));
+        exp_acc2<false>(a1, v[t + 2], v[t + 3], cc, make_float2(b0.z, b0.w));
+        exp_acc2<(kPolyOf8 > 4)>(a0, v[t + 4], v[t + 5], cc, make_float2(b1.x, b1.y));
+        exp_acc2<(kPolyOf8 > 2)>(a1, v[t + 6], v[t + 7], cc, make_float2(b1.z, b1.w));
+        exp_acc2<(kPolyOf8 > 1)>(a0, v[t + 8], v[t + 9], cc, make_float2(b2.x, b2.y));
+        exp_acc2<false>(a1, v[t + 10], v[t + 11], cc, make_float2(b2.z, b2.w));
+        exp_acc2<(kPolyOf8 > 5)>(a0, v[t + 12], v[t + 13], cc, make_float2(b3.x, b3.y));
+        exp_acc2<(kPolyOf8 > 3)>(a1, v[t + 14], v[t + 15], cc, make_float2(b3.z, b3.w));
+    }
+}
+
+__device__ __forceinline__ float max32(const uint32_t (&v)[32])
+{
+    float c0 = -INFINITY, c1 = -INFINITY;
+#pragma unroll
+    for (int t = 0; t < 32; t += 4) {
+        c0 = max3(c0, __uint_as_float(v[t + 0]), __uint_as_float(v[t + 1]));
+        c1 = max3(c1, __uint_as_float(v[t + 2]), __uint_as_float(v[t + 3]));
+    }
+    return fmaxf(c0, c1);
 }
 
 // ------------------------------------------------------------------ schedule
 
 // Segment s of the 2 * ngroups segments every CTA walks: a pass over this CTA's share of one group.
 struct Seg {
-    int pass, g, h0, t_begin, t_end;
+    int pass, g, h0, ntiles;
+    int kv0, t0;   // KV head and tile within the head of the first tile in walking order
 };
 
-__device__ __forceinline__ Seg segment(int s, const Params &P)
+// (Not inlined: five roles call it once per segment.)
+__device__ __noinline__ Seg segment(int s, const Params &P)
 {
     Seg sg;
     const int NG = P.ngroups;
@@ -243,24 +353,21 @@ __device__ __forceinline__ Seg segment(int s, const Params &P)
     else { sg.pass = 2; sg.g = (s >> 1) - 1; }
     sg.h0 = sg.g * P.hpg;
     const int nh = min(P.hpg, P.Hkv - sg.h0);
-    const long long T = (long long)nh * P.tph, G = gridDim.x;
-    sg.t_begin = (int)((long long)blockIdx.x * T / G);
-    sg.t_end = (int)(((long long)blockIdx.x + 1) * T / G);
+    const uint32_t T = (uint32_t)nh * P.tph, G = gridDim.x;
+    const uint32_t t_begin = blockIdx.x * T / G, t_end = (blockIdx.x + 1) * T / G;
+    sg.ntiles = (int)(t_end - t_begin);
+    const uint32_t first = (sg.pass == 1) ? t_begin : (t_end > 0 ? t_end - 1 : 0);
+    sg.kv0 = sg.h0 + (int)(first / P.tph);
+    sg.t0 = (int)(first % P.tph);
     return sg;
 }
 
-// Merge of two partial (max, sum of exp2(c (s - max))) pairs; an empty partial has l == 0.
-__device__ __forceinline__ void merge_ml(float &m, float &l, float m2, float l2, float c)
+// Next tile in walking order (forwards in pass 1, backwards in pass 2), without a division: the
+// reciprocal a division needs would queue behind the exponentials in the special-function unit.
+__device__ __forceinline__ void walk(int pass, int tph, int &kv, int &t)
 {
-    if (l2 > 0.f) {
-        if (l > 0.f) {
-            const float mn = fmaxf(m, m2);
-            l = l * ex2(c * (m - mn)) + l2 * ex2(c * (m2 - mn));
-            m = mn;
-        } else {
-            m = m2; l = l2;
-        }
-    }
+    if (pass == 1) { if (++t == tph) { t = 0; ++kv; } }
+    else { if (--t < 0) { t = tph - 1; --kv; } }
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -269,23 +376,27 @@ __global__ void __launch_bounds__(kThreads, 1)
 score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ, const Params P)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 1024-byte aligned data
-    uint8_t *data = smem_raw + (base - smem_u32(smem_raw));
+    if (smem_u32(smem_raw) & 1023u) {   // the swizzled tiles need 1024-byte alignment; nothing has been started yet
+        if (threadIdx.x == 0) atomicMax(P.status + kWStatus, (int)JQ_ERR_CUDA);
+        return;
+    }
     const uint32_t q_bytes = (uint32_t)P.Rbox * kD * 2;
-    uint8_t *qbuf = data;                                    // two query buffers
-    uint8_t *kbuf = data + 2 * (size_t)q_bytes;              // K ring
+    uint8_t *qbuf = smem_raw;                                 // two query buffers
+    uint8_t *kbuf = smem_raw + 2 * (size_t)q_bytes;           // K ring
     Ctl *ctl = (Ctl *)(kbuf + (size_t)P.stages * kStageBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, stages = P.stages;
-    const int nslots = (P.Rbox == 256) ? 2 : 4;
-    const uint32_t slot_cols = kTmemCols / nslots;
+    const int nblk = P.Rbox / 128;                            // accumulator blocks per tile, both passes
     const int nseg = 2 * P.ngroups;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&ctl->q_full[s], 1); mbar_init(&ctl->q_empty[s], 1); }
-        for (int s = 0; s < 4; ++s) { mbar_init(&ctl->t_full[s], 1); mbar_init(&ctl->t_empty[s], P.Rbox == 256 ? 256 : 128); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&ctl->q_full[s], 1); mbar_init(&ctl->q_empty[s], 1);
+            mbar_init(&ctl->ms_full[s], 1); mbar_init(&ctl->ms_empty[s], kEpiWarps);
+        }
+        for (int s = 0; s < kTSlots; ++s) { mbar_init(&ctl->t_full[s], 1); mbar_init(&ctl->t_empty[s], 128); }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -301,15 +412,17 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
+            TR_DECL;
             uint32_t it = 0, qn = 0;
             int prev_kv = -1;
             bool ok = true;
+#pragma unroll 1
             for (int s = 0; s < nseg && ok; ++s) {
                 const Seg sg = segment(s, P);
-                const int ntiles = sg.t_end - sg.t_begin;
-                for (int n = 0; n < ntiles; ++n, ++it) {
-                    const int i = (sg.pass == 1) ? sg.t_begin + n : sg.t_end - 1 - n;
-                    const int kv = sg.h0 + i / P.tph, j0 = (i % P.tph) * kTile;
+                int kv = sg.kv0, tt = sg.t0;
+#pragma unroll 1
+                for (int n = 0; n < sg.ntiles; ++n, ++it, walk(sg.pass, P.tph, kv, tt)) {
+                    TR_ADD(2);
                     if (kv != prev_kv) {
                         const uint32_t qb = qn & 1;
                         if (!mbar_wait(&ctl->q_empty[qb], ((qn >> 1) & 1) ^ 1, ctl, P.status)) { ok = false; break; }
@@ -317,255 +430,317 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                         tma_load_3d(qbuf + (size_t)qb * q_bytes, &mapQ, &ctl->q_full[qb], 0, 0, kv);
                         tma_load_3d(qbuf + (size_t)qb * q_bytes + q_bytes / 2, &mapQ, &ctl->q_full[qb], 64, 0, kv);
                         prev_kv = kv; ++qn;
+                        TR_ADD(0);
                     }
                     const uint32_t st = it % stages;
                     if (!mbar_wait(&ctl->empty[st], ((it / stages) & 1) ^ 1, ctl, P.status)) { ok = false; break; }
+                    TR_ADD(1);
                     mbar_expect_tx(&ctl->full[st], kStageBytes);
-                    tma_load_3d(kbuf + (size_t)st * kStageBytes, &mapK, &ctl->full[st], 0, j0, kv);
-                    tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, &mapK, &ctl->full[st], 64, j0, kv);
+                    tma_load_3d(kbuf + (size_t)st * kStageBytes, &mapK, &ctl->full[st], 0, tt * kTile, kv);
+                    tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, &mapK, &ctl->full[st], 64, tt * kTile, kv);
                 }
             }
+            TR_DUMP;
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            const uint32_t idesc1 = instr_desc(128, kTile), idesc2 = instr_desc(kTile, P.Rpad);
-            const int nmb = P.Rbox / 128;                     // pass 1: accumulator blocks of 128 query rows
-            uint32_t it = 0, qn = 0;
+            TR_DECL;
+            const uint32_t idesc1 = instr_desc(128, kTile);
+            // pass 2: a block's columns are the query rows it covers, rounded up to 16
+            const uint32_t idesc2a = instr_desc(kTile, min(128, P.Rpad)), idesc2b = instr_desc(kTile, max(16, P.Rpad - 128));
+            uint32_t it = 0, qn = 0, u = 0;                   // tiles, query loads, accumulator blocks so far
             int prev_kv = -1;
             bool ok = true;
+#pragma unroll 1
             for (int s = 0; s < nseg && ok; ++s) {
                 const Seg sg = segment(s, P);
-                const int ntiles = sg.t_end - sg.t_begin;
-                for (int n = 0; n < ntiles; ++n, ++it) {
-                    const int i = (sg.pass == 1) ? sg.t_begin + n : sg.t_end - 1 - n;
-                    const int kv = sg.h0 + i / P.tph;
+                int kv = sg.kv0, tt = sg.t0;
+#pragma unroll 1
+                for (int n = 0; n < sg.ntiles && ok; ++n, ++it, walk(sg.pass, P.tph, kv, tt)) {
+                    TR_ADD(4);
                     if (kv != prev_kv) {
                         if (qn > 0) tc_commit(&ctl->q_empty[(qn - 1) & 1]);   // the previous head's queries are free once its MMAs retire
                         if (!mbar_wait(&ctl->q_full[qn & 1], (qn >> 1) & 1, ctl, P.status)) { ok = false; break; }
                         prev_kv = kv; ++qn;
+                        TR_ADD(0);
                     }
-                    const uint32_t st = it % stages, slot = it % nslots;
+                    const uint32_t st = it % stages;
                     if (!mbar_wait(&ctl->full[st], (it / stages) & 1, ctl, P.status)) { ok = false; break; }
-                    if (!mbar_wait(&ctl->t_empty[slot], ((it / nslots) & 1) ^ 1, ctl, P.status)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t k_addr = smem_u32(kbuf + (size_t)st * kStageBytes);
-                    const uint32_t q_addr = smem_u32(qbuf + (size_t)((qn - 1) & 1) * q_bytes);
-                    const uint32_t d = tmem + slot * slot_cols;
-                    if (sg.pass == 1) {
-                        for (int mb = 0; mb < nmb; ++mb) {
-#pragma unroll
-                            for (int ks = 0; ks < kD / 16; ++ks) {
-                                const uint32_t koff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                                const uint32_t qoff = (uint32_t)(ks >> 2) * (q_bytes / 2) + (uint32_t)(ks & 3) * 32u;
-                                tc_mma(d + (uint32_t)mb * 128u, smem_desc(q_addr + qoff + (uint32_t)mb * kHalfBytes),
-                                       smem_desc(k_addr + koff), idesc1, ks > 0);
-                            }
-                        }
-                    } else {
-#pragma unroll
-                        for (int ks = 0; ks < kD / 16; ++ks) {
-                            const uint32_t koff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                            const uint32_t qoff = (uint32_t)(ks >> 2) * (q_bytes / 2) + (uint32_t)(ks & 3) * 32u;
-                            tc_mma(d, smem_desc(k_addr + koff), smem_desc(q_addr + qoff), idesc2, ks > 0);
-                        }
+                    TR_ADD(1);
+                    const uint32_t k_lo = desc_lo(smem_u32(kbuf) + st * kStageBytes);
+                    const uint32_t q_lo = desc_lo(smem_u32(qbuf) + ((qn - 1) & 1) * q_bytes);
+#pragma unroll 1
+                    for (int blk = 0; blk < nblk; ++blk, ++u) {
+                        const uint32_t slot = u % kTSlots;
+                        if (!mbar_wait(&ctl->t_empty[slot], ((u / kTSlots) & 1) ^ 1, ctl, P.status)) { ok = false; break; }
+                        TR_ADD(2);
+                        tc_fence_after();
+                        const uint32_t d = tmem + slot * kSlotCols;
+                        const uint32_t qb_lo = q_lo + (uint32_t)blk * (kHalfBytes >> 4);   // query rows [128 blk, 128 blk + 128)
+                        if (sg.pass == 1) tc_mma_block(d, qb_lo, k_lo, q_bytes / 2, kHalfBytes, idesc1);
+                        else tc_mma_block(d, k_lo, qb_lo, kHalfBytes, q_bytes / 2, blk == 0 ? idesc2a : idesc2b);
+                        tc_commit(&ctl->t_full[slot]);
+                        TR_ADD(3);
                     }
-                    tc_commit(&ctl->t_full[slot]);
-                    tc_commit(&ctl->empty[st]);
+                    if (ok) tc_commit(&ctl->empty[st]);
                 }
             }
+            TR_DUMP;
         }
-    } else if (warp < 10) {
+    } else if (warp < kMergeWarp) {
         // ---------------------------------------------------------------- epilogue groups
         const int grp = (warp - 2) >> 2, quarter = warp & 3;
-        const int et = threadIdx.x - 64;                        // 0..255
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
-        const bool wide = P.Rbox == 256;
-        const int my_row = (wide ? grp * 128 : 0) + quarter * 32 + lane;   // pass 1: the query row this thread owns
+        const int row0 = quarter * 32 + lane;                   // TMEM lane: query row within its block (pass 1), key within its tile (pass 2)
         const float c = P.c;
-        uint32_t it = 0;
+        const float2 cc = make_float2(c, c);
+        uint32_t u = 0, hs = 0;                                 // accumulator blocks so far; pass-2 heads so far
         bool ok = true;
+        TR_DECL;
 
+#pragma unroll 1
         for (int s = 0; s < nseg; ++s) {
             const Seg sg = segment(s, P);
-            const int ntiles = sg.t_end - sg.t_begin;
             int prev_kv = -1;
+            int kv = sg.kv0, tt = sg.t0;
             if (sg.pass == 1) {
-                // l = sum_j exp2(c (s_j - m_run)) against a REFERENCE m_run that need not be the row max: it
-                // is the max of the first tile seen and is only raised when a later tile would push the sum
-                // towards overflow (the tile is then redone from its registers).  Any reference gives the
-                // same M_r = c m + log2(l) after the merge.
-                float m_run = -INFINITY;
-                float2 l01 = make_float2(0.f, 0.f), l23 = make_float2(0.f, 0.f);
-                auto flush_partial = [&](int kv) {
-                    if (my_row < P.R && ok)
-                        P.part[((size_t)kv * kSlots + 2 * blockIdx.x + grp) * P.R + my_row] =
-                            make_float2(m_run, (l01.x + l01.y) + (l23.x + l23.y));
-                    m_run = -INFINITY;
-                    l01 = l23 = make_float2(0.f, 0.f);
-                };
-                for (int n = 0; n < ntiles; ++n, ++it) {
-                    const int i = sg.t_begin + n;
-                    const int kv = sg.h0 + i / P.tph, j0 = (i % P.tph) * kTile;
-                    if (kv != prev_kv) {
-                        if (prev_kv >= 0) flush_partial(prev_kv);
-                        prev_kv = kv;
-                    }
-                    if (!wide && (int)(it & 1) != grp) continue;
-                    const uint32_t slot = it % nslots;
-                    if (ok) ok = mbar_wait(&ctl->t_full[slot], (it / nslots) & 1, ctl, P.status);
-                    if (!ok) continue;
-                    tc_fence_after();
-                    const uint32_t taddr = lane_addr + slot * slot_cols + (wide ? (uint32_t)grp * 128u : 0u);
-                    uint32_t v[128];
-                    // the whole 128-key row segment in one tensor-memory read; the slot is free right after
-                    JQ_TMEM_LD128(taddr, v);
-                    tmem_ld_wait();
-                    tc_fence_before();
-                    mbar_arrive(&ctl->t_empty[slot], 1);
-                    const int valid = min(kTile, P.L - j0);
-                    if (valid < kTile) {
-#pragma unroll
-                        for (int t = 0; t < 128; ++t) if (t >= valid) v[t] = 0xff800000u;   // -inf: not a key
-                    }
-                    if (m_run == -INFINITY) m_run = max128(v);
-                    const float2 keep01 = l01, keep23 = l23;
-                    const float2 cc = make_float2(c, c);
-                    float2 mb = make_float2(-m_run * c, -m_run * c);
-#pragma unroll
-                    for (int t = 0; t < 128; t += 4) {
-                        exp_acc2(l01, v[t + 0], v[t + 1], cc, mb);
-                        exp_acc2(l23, v[t + 2], v[t + 3], cc, mb);
-                    }
-                    const float lsum = (l01.x + l01.y) + (l23.x + l23.y);
-                    if (!(lsum < 1.0e30f)) {
-                        // the reference is too far below this tile's values: raise it to the tile max and redo the tile
-                        const float cm = fmaxf(max128(v), m_run);
-                        const float f = ex2(c * (m_run - cm));
-                        l01 = make_float2(keep01.x * f, keep01.y * f);
-                        l23 = make_float2(keep23.x * f, keep23.y * f);
-                        m_run = cm;
-                        mb = make_float2(-m_run * c, -m_run * c);
-#pragma unroll
-                        for (int t = 0; t < 128; t += 4) {
-                            exp_acc2(l01, v[t + 0], v[t + 1], cc, mb);
-                            exp_acc2(l23, v[t + 2], v[t + 3], cc, mb);
-                        }
-                    }
-                }
-                if (prev_kv >= 0) flush_partial(prev_kv);
-                // this CTA's share of pass 1 of the group is published: count it in
-                __threadfence();
-                epi_sync();
-                if (et == 0) atomicAdd(P.status + kWCnt1 + (sg.g & (kRing - 1)), 1);
-            } else {
-                if (et == 0 && ok)
-                    ok = wait_counter(P.status + kWCnt2 + (sg.g & (kRing - 1)), (sg.g / kRing + 1) * G, ctl, P.status);
-                for (int n = 0; n < ntiles; ++n, ++it) {
-                    const int i = sg.t_end - 1 - n;
-                    const int kv = sg.h0 + i / P.tph, j0 = (i % P.tph) * kTile;
-                    if (kv != prev_kv) {
-                        // stage the row normalisers M_r of the new head (all readers of the old ones are past them)
-                        epi_sync();
-                        if (et < P.R) ctl->Ms[et] = -__ldcg(&P.Mrow[(size_t)kv * P.R + et]);   // stored negated: x = c s + (-M_r)
-                        epi_sync();
-                        if (*(volatile int *)&ctl->abort_flag) ok = false;
-                        prev_kv = kv;
-                    }
-                    if ((int)(it & 1) != grp) continue;
-                    const uint32_t slot = it % nslots;
-                    if (ok) ok = mbar_wait(&ctl->t_full[slot], (it / nslots) & 1, ctl, P.status);
-                    if (!ok) continue;
-                    tc_fence_after();
-                    const uint32_t taddr = lane_addr + slot * slot_cols;
-                    const uint32_t arrive_n = wide ? 2u : 1u;
-                    const float *Ms = ctl->Ms;
-                    const int Rpad = P.Rpad;
-                    uint32_t v[128];
-                    float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
-                    const float2 cc = make_float2(c, c);
+                // Per block of 128 query rows: l = sum_j exp2(c (s_j - m)) against a REFERENCE m that need
+                // not be the row max: it is the max of the first 32 values seen and is only raised when later
+                // values would push the sum towards overflow (those 32 are then redone from their
+                // registers).  Any reference gives the same M_r = c m + log2(l) after the merge.
+                struct RowState { float m; float2 l01, l23; };
+                RowState st0 = {-INFINITY, make_float2(0.f, 0.f), make_float2(0.f, 0.f)}, st1 = st0;
 #pragma unroll 1
-                    for (int c0 = 0; c0 < Rpad; c0 += 128) {
-                        if (Rpad - c0 >= 128) {
-                            JQ_TMEM_LD128(taddr + c0, v);
+                for (int n = 0; n <= sg.ntiles; ++n, walk(1, P.tph, kv, tt)) {
+                    if (n == sg.ntiles || kv != prev_kv) {
+                        if (prev_kv >= 0) {
+                            // publish this warp's partials of the head just left
+                            float2 *dst = P.part + ((size_t)prev_kv * kSlots + kGroups * blockIdx.x + grp) * P.R;
+                            if (ok && row0 < P.R) dst[row0] = make_float2(st0.m, (st0.l01.x + st0.l01.y) + (st0.l23.x + st0.l23.y));
+                            if (ok && nblk == 2 && row0 + 128 < P.R)
+                                dst[row0 + 128] = make_float2(st1.m, (st1.l01.x + st1.l01.y) + (st1.l23.x + st1.l23.y));
+                            st0.m = st1.m = -INFINITY;
+                            st0.l01 = st0.l23 = st1.l01 = st1.l23 = make_float2(0.f, 0.f);
+                        }
+                        if (n == sg.ntiles) break;
+                        prev_kv = kv;
+                    }
+                    const int valid = min(kTile, P.L - tt * kTile);
+#pragma unroll 1
+                    for (int blk = 0; blk < nblk; ++blk, ++u) {
+                        if ((int)(u % kGroups) != grp) continue;
+                        const uint32_t slot = u % kTSlots;
+                        TR_ADD(8);
+                        if (ok) ok = mbar_wait(&ctl->t_full[slot], (u / kTSlots) & 1, ctl, P.status);
+                        if (!ok) continue;
+                        TR_ADD(0);
+                        tc_fence_after();
+                        const uint32_t taddr = lane_addr + slot * kSlotCols;
+                        // one copy of the block code: the second row block borrows the first one's registers
+                        if (blk == 1) { const RowState t = st0; st0 = st1; st1 = t; }
+#pragma unroll 1
+                        for (int c0 = 0; c0 < kTile; c0 += 32) {
+                            uint32_t v[32];
+                            JQ_TMEM_LD32(taddr + c0, v);
                             tmem_ld_wait();
-                            if (c0 + 128 >= Rpad) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], arrive_n); }
-                            const int nv = P.R - c0;             // columns that are real query rows
-                            if (nv >= 128) {
+                            TR_ADD(1);
+                            if (c0 + 32 == kTile) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], 1); }
+                            if (valid < c0 + 32) {
 #pragma unroll
-                                for (int t = 0; t < 128; t += 4) {
-                                    const float4 mm = *(const float4 *)(Ms + c0 + t);
-                                    exp_acc2(a01, v[t + 0], v[t + 1], cc, make_float2(mm.x, mm.y));
-                                    exp_acc2(a23, v[t + 2], v[t + 3], cc, make_float2(mm.z, mm.w));
-                                }
-                            } else {
-#pragma unroll
-                                for (int t = 0; t < 128; ++t) if (t < nv) a01.x += ex2(fmaf(__uint_as_float(v[t]), c, Ms[c0 + t]));
+                                for (int t = 0; t < 32; ++t) if (c0 + t >= valid) v[t] = 0xff800000u;   // -inf: not a key
                             }
-                        } else {
+                            if (st0.m == -INFINITY) st0.m = max32(v);
+                            const float2 keep01 = st0.l01, keep23 = st0.l23;
 #pragma unroll 1
-                            for (int c1 = c0; c1 < Rpad; c1 += 32) {
-                                JQ_TMEM_LD32(taddr + c1, v);
-                                tmem_ld_wait();
-                                if (c1 + 32 >= Rpad) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], arrive_n); }
-                                const int nv = P.R - c1;
-                                if (nv >= 32) {
-#pragma unroll
-                                    for (int t = 0; t < 32; t += 4) {
-                                        const float4 mm = *(const float4 *)(Ms + c1 + t);
-                                        exp_acc2(a01, v[t + 0], v[t + 1], cc, make_float2(mm.x, mm.y));
-                                        exp_acc2(a23, v[t + 2], v[t + 3], cc, make_float2(mm.z, mm.w));
-                                    }
-                                } else {
-#pragma unroll
-                                    for (int t = 0; t < 32; ++t) if (t < nv) a01.x += ex2(fmaf(__uint_as_float(v[t]), c, Ms[c1 + t]));
-                                }
+                            for (int attempt = 0; attempt < 2; ++attempt) {
+                                const float nb = -st0.m * c;
+                                const float4 b4 = make_float4(nb, nb, nb, nb);
+                                exp_acc32<0>(st0.l01, st0.l23, v, cc, &b4);
+                                const float lsum = (st0.l01.x + st0.l01.y) + (st0.l23.x + st0.l23.y);
+                                if (lsum < 1.0e30f) break;
+                                // the reference is too far below these values: raise it to their max and redo them
+                                const float cm = fmaxf(max32(v), st0.m);
+                                const float f = ex2(c * (st0.m - cm));
+                                st0.l01 = make_float2(keep01.x * f, keep01.y * f);
+                                st0.l23 = make_float2(keep23.x * f, keep23.y * f);
+                                st0.m = cm;
                             }
+                            TR_ADD(2);
+                        }
+                        if (blk == 1) { const RowState t = st0; st0 = st1; st1 = t; }
+                    }
+                }
+                TR_ADD(8);
+                // this warp's share of pass 1 of the group is published: count it in
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(P.status + kWCnt1 + (sg.g & (kRing - 1)), 1);
+                TR_ADD(6);
+            } else {
+                const float *Ms = ctl->Ms[0];
+#pragma unroll 1
+                for (int n = 0; n < sg.ntiles; ++n, walk(2, P.tph, kv, tt)) {
+                    if (kv != prev_kv) {
+                        TR_ADD(10);
+                        // done with the previous head's normalisers; wait for this head's
+                        if (prev_kv >= 0) {
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&ctl->ms_empty[(hs - 1) & 1], 1);
+                        }
+                        if (ok) ok = mbar_wait(&ctl->ms_full[hs & 1], (hs >> 1) & 1, ctl, P.status);
+                        Ms = ctl->Ms[hs & 1];
+                        ++hs;
+                        prev_kv = kv;
+                        TR_ADD(4);
+                    }
+#pragma unroll 1
+                    for (int blk = 0; blk < nblk; ++blk, ++u) {
+                        if ((int)(u % kGroups) != grp) continue;
+                        const uint32_t slot = u % kTSlots;
+                        TR_ADD(10);
+                        if (ok) ok = mbar_wait(&ctl->t_full[slot], (u / kTSlots) & 1, ctl, P.status);
+                        if (!ok) continue;
+                        TR_ADD(3);
+                        tc_fence_after();
+                        const uint32_t taddr = lane_addr + slot * kSlotCols;
+                        const int ncols = min(128, P.Rpad - blk * 128);    // accumulator columns of this block
+                        const float *bias = Ms + blk * 128;                 // columns that are not query rows carry a bias of -inf
+                        float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
+#pragma unroll 1
+                        for (int c0 = 0; c0 < ncols; c0 += 32) {
+                            uint32_t v[32];
+                            JQ_TMEM_LD32(taddr + c0, v);
+                            tmem_ld_wait();
+                            TR_ADD(1);
+                            if (c0 + 32 >= ncols) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], 1); }
+                            exp_acc32<1>(a01, a23, v, cc, (const float4 *)(bias + c0));
+                            TR_ADD(5);
+                        }
+                        const int key = tt * kTile + row0;
+                        if (key < P.L) {
+                            float *dst = P.scores + (size_t)kv * P.L + key;
+                            const float sum = (a01.x + a01.y) + (a23.x + a23.y);
+                            if (nblk == 1) *dst = sum;
+                            else atomicAdd(dst, sum);              // two blocks per key, onto a zero the stage warp wrote
                         }
                     }
-                    const int key = j0 + quarter * 32 + lane;
-                    if (key < P.L) P.scores[(size_t)kv * P.L + key] = (a01.x + a01.y) + (a23.x + a23.y);
                 }
+                if (prev_kv >= 0) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->ms_empty[(hs - 1) & 1], 1);
+                }
+                TR_ADD(10);
             }
         }
-    } else {
+        TR_DUMP;
+    } else if (warp == kMergeWarp) {
         // ---------------------------------------------------------------- grid-wide merge of the pass-1 partials
-        // Group g: once every CTA has published its partials, this CTA combines the rows b, b+G, b+2G, ...
-        // of the group (lanes over the contributing slots, then a butterfly: a fixed order, hence
-        // deterministic) into M_r = c*m_r + log2(l_r), and counts itself in.
+        // Group g: once every epilogue warp of every CTA has published its partials, this CTA combines its
+        // share of the group's rows into M_r = c*m_r + log2(l_r), and counts itself in.
         const float c = P.c;
+        const uint32_t Gu = (uint32_t)G;
+#pragma unroll 1
         for (int g = 0; g < P.ngroups; ++g) {
             int ok = 1;
-            if (lane == 0) ok = wait_counter(P.status + kWCnt1 + (g & (kRing - 1)), (g / kRing + 1) * G, ctl, P.status) ? 1 : 0;
+            if (lane == 0)
+                ok = wait_counter(P.status + kWCnt1 + (g & (kRing - 1)), (g / kRing + 1) * G * kEpiWarps, ctl, P.status) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             const int h0 = g * P.hpg, nh = min(P.hpg, P.Hkv - h0);
-            const long long T = (long long)nh * P.tph;
-            const int ng = (P.Rbox == 256) ? 1 : 2;
-            for (int item = blockIdx.x; item < nh * P.R; item += G) {
+            const uint32_t T = (uint32_t)nh * P.tph;
+            // This CTA's rows of the group are blockIdx.x + k G.  They are taken `rows_par` at a time, each by a
+            // sub-group of 32 / rows_par lanes that splits the row's partial slots, eight loads in flight per
+            // lane; an empty partial (or one of a CTA that had no tile of the head) counts as (-inf, 0).
+            const int nitems = nh * P.R;
+            const int nrows = (nitems > (int)blockIdx.x) ? (nitems - 1 - (int)blockIdx.x) / G + 1 : 0;
+            int rows_par = 1;
+            while (rows_par < nrows && rows_par < 32) rows_par <<= 1;
+            const int lpr = 32 / rows_par, sub = lane % lpr;
+#pragma unroll 1
+            for (int base = 0; base < nrows; base += rows_par) {
+                const int my = base + lane / lpr;
+                const bool have = my < nrows;
+                const int item = blockIdx.x + (have ? my : 0) * G;
                 const int hl = item / P.R, r = item - hl * P.R, kv = h0 + hl;
-                const long long first = (long long)hl * P.tph;
-                const int b_lo = owner_of_tile(first, T, G), b_hi = owner_of_tile(first + P.tph - 1, T, G);
-                const int g0 = (P.Rbox == 256) ? (r >> 7) : 0;
-                const int nsl = (b_hi - b_lo + 1) * ng;
+                const uint32_t first = (uint32_t)hl * P.tph;
+                const int b_lo = owner_of_tile(first, T, Gu), b_hi = owner_of_tile(first + P.tph - 1, T, Gu);
+                const int nsl = have ? (b_hi - b_lo + 1) * kGroups : 0;   // every epilogue group of a contributing CTA wrote a partial
+                const float2 *src = P.part + ((size_t)kv * kSlots + kGroups * b_lo) * P.R + r;
                 float m = -INFINITY, l = 0.f;
-                for (int i = lane; i < nsl; i += 32) {
-                    const int b = b_lo + i / ng, gg = g0 + i % ng;
-                    if ((long long)b * T / G == ((long long)b + 1) * T / G) continue;   // CTA b had no tile
-                    const float2 p = __ldcg(&P.part[((size_t)kv * kSlots + 2 * b + gg) * P.R + r]);
-                    merge_ml(m, l, p.x, p.y, c);
-                }
+#pragma unroll 1
+                for (int i0 = sub; i0 < nsl; i0 += lpr * 8) {
+                    float2 p[8];
 #pragma unroll
-                for (int o = 16; o >= 1; o >>= 1) {
-                    const float m2 = __shfl_xor_sync(0xffffffffu, m, o), l2 = __shfl_xor_sync(0xffffffffu, l, o);
-                    merge_ml(m, l, m2, l2, c);
+                    for (int k = 0; k < 8; ++k) {
+                        const int i = i0 + lpr * k;
+                        p[k] = make_float2(-INFINITY, 0.f);
+                        // (a CTA between b_lo and b_hi always has a tile of this head unless the group has fewer tiles than CTAs)
+                        if (i < nsl && (T >= Gu || cta_has_tile(b_lo + i / kGroups, T, Gu)))
+                            p[k] = __ldcg(src + (size_t)i * P.R);
+                    }
+                    float mn = m;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) if (p[k].y > 0.f) mn = fmaxf(mn, p[k].x);
+                    if (mn > -INFINITY) {
+                        float acc = (l > 0.f) ? l * ex2(c * (m - mn)) : 0.f;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) if (p[k].y > 0.f) acc += p[k].y * ex2(c * (p[k].x - mn));
+                        m = mn; l = acc;
+                    }
                 }
-                if (lane == 0) P.Mrow[(size_t)kv * P.R + r] = c * m + log2f(l);
+                // butterfly over the sub-group (a fixed order, hence deterministic): first the common
+                // reference, then the sum against it
+                float mw = (l > 0.f) ? m : -INFINITY;
+                for (int o = lpr >> 1; o >= 1; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, o));
+                l = (l > 0.f) ? l * ex2(c * (m - mw)) : 0.f;
+                for (int o = lpr >> 1; o >= 1; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+                if (have && sub == 0) P.Mrow[(size_t)kv * P.R + r] = c * mw + log2f(l);
             }
             __syncwarp();
             if (lane == 0) {
                 __threadfence();
                 atomicAdd(P.status + kWCnt2 + (g & (kRing - 1)), 1);
+            }
+        }
+    } else if (warp == kStageWarp) {
+        // ---------------------------------------------------------------- pass-2 stager
+        // Walks the pass-2 segments in order.  Per segment: with two blocks per key, zeroes the scores of
+        // this CTA's keys (the epilogue adds into them); waits until the group's normalisers are merged;
+        // then feeds -M_r of each KV head of the segment into the double-buffered shared array.
+        uint32_t hs = 0;
+        int ok = 1;
+#pragma unroll 1
+        for (int s = 0; s < nseg && ok; ++s) {
+            const Seg sg = segment(s, P);
+            if (sg.pass != 2 || sg.ntiles == 0) continue;
+            if (nblk == 2) {
+                int kv = sg.kv0, tt = sg.t0;
+                for (int n = 0; n < sg.ntiles; ++n, walk(2, P.tph, kv, tt)) {
+                    float *dst = P.scores + (size_t)kv * P.L + tt * kTile;
+                    for (int t = lane; t < kTile && tt * kTile + t < P.L; t += 32) dst[t] = 0.f;
+                }
+                __threadfence();
+            }
+            if (lane == 0)
+                ok = wait_counter(P.status + kWCnt2 + (sg.g & (kRing - 1)), (sg.g / kRing + 1) * G, ctl, P.status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            int prev_kv = -1;
+            int kv = sg.kv0, tt = sg.t0;
+#pragma unroll 1
+            for (int n = 0; n < sg.ntiles && ok; ++n, walk(2, P.tph, kv, tt)) {
+                if (kv == prev_kv) continue;
+                prev_kv = kv;
+                const uint32_t buf = hs & 1;
+                ok = mbar_wait(&ctl->ms_empty[buf], ((hs >> 1) & 1) ^ 1, ctl, P.status) ? 1 : 0;
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                for (int r = lane; r < kMaxR; r += 32)   // stored negated: x = c s + (-M_r); -inf silences a padding column
+                    ctl->Ms[buf][r] = (r < P.R) ? -__ldcg(&P.Mrow[(size_t)kv * P.R + r]) : -INFINITY;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->ms_full[buf], 1);
+                ++hs;
             }
         }
     }
@@ -626,7 +801,7 @@ bool make_map(CUtensorMap *map, const void *ptr, int rows, int heads, int box_ro
 
 constexpr size_t smem_bytes(int Rbox, int stages)
 {
-    return 1024 + 2 * (size_t)Rbox * kD * 2 + (size_t)stages * kStageBytes + kCtlBytes;
+    return 2 * (size_t)Rbox * kD * 2 + (size_t)stages * kStageBytes + kCtlBytes;
 }
 
 struct DeviceInfo {
@@ -670,6 +845,11 @@ long long env_ll(const char *name, long long dflt)
 
 }  // namespace
 
+#ifdef JQ_TRACE
+static long long *g_trace = nullptr;
+extern "C" void jq_debug_set_trace(long long *p) { g_trace = p; }   // [grid][32 warps][16] int64, device memory
+#endif
+
 jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float *scores, const Workspace &w,
                           cudaStream_t st)
 {
@@ -686,11 +866,14 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
     P.pipelined = order != 0;
     P.c = 1.4426950408889634f / sqrtf((float)s.d);
     P.part = w.part; P.Mrow = w.Mrow; P.scores = scores; P.status = w.status;
+#ifdef JQ_TRACE
+    P.trace = g_trace;
+#endif
     CUtensorMap mapK, mapQ;
     if (!make_map(&mapK, K, s.L, s.Hkv, kTile) || !make_map(&mapQ, Q, R, s.Hkv, P.Rbox)) return JQ_ERR_CUDA;
 
     int sms = dev.sms;
-    if (2 * sms > kSlots) sms = kSlots / 2;
+    if (kGroups * sms > kSlots) sms = kSlots / kGroups;
     // KV heads are scored in groups whose keys fit in a share of the L2, so that pass 2 finds them there.
     // Among the admissible group sizes, take the one that wastes the fewest CTA-tile slots.
     const long long head_bytes = (long long)s.L * kD * 2;
