@@ -79,6 +79,19 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSlotCols = kTmemCols / kTSlots;
 constexpr long long kWaitCycles = 4000000000ll;  // about 2 s of SM clock per wait
 constexpr int kRing = 4;                         // grid counters per kind
+#ifndef JQ_SLEEP_LONG
+#define JQ_SLEEP_LONG 256
+#endif
+#ifndef JQ_SLEEP_SHORT
+#define JQ_SLEEP_SHORT 32
+#endif
+constexpr uint32_t kSleepLong = JQ_SLEEP_LONG;   // ns between polls of a waiter that runs ahead (producer, stager)
+constexpr uint32_t kSleepShort = JQ_SLEEP_SHORT; // ns between polls of a waiter on the critical path
+#ifndef JQ_CHUNK
+#define JQ_CHUNK 32
+#endif
+constexpr int kChunk = JQ_CHUNK;                 // accumulator columns per tensor-memory read (32 or 64)
+static_assert(kChunk == 32 || kChunk == 64, "kChunk");
 constexpr int kPolyOf8 = JQ_POLY_OF8;            // of every 8 pairs of exponentials, this many go to the FMA pipe
 // words of the workspace status block
 constexpr int kWStatus = 0, kWDone = 1, kWCnt1 = 8, kWCnt2 = 12;
@@ -139,16 +152,22 @@ __device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait.  false: the wait ran out (status recorded) or another thread of the CTA aborted.
-// The clock is only consulted after a few thousand failed polls, so a normal wait never pays for it.
-__device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, Ctl *ctl, int *status)
+// A waiter that can afford it sleeps `sleep_ns` between polls: a spinning warp takes issue slots and
+// queue entries of the shared-memory pipe away from the epilogue warps on its scheduler.  The clock is
+// only consulted after many failed polls, so a normal wait never pays for it.
+__device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, Ctl *ctl, int *status, uint32_t sleep_ns)
 {
     if (*(volatile int *)&ctl->abort_flag) return false;
-    for (int i = 0; i < 4096; ++i)
+    for (int i = 0; i < 2048; ++i) {
         if (mbar_try(bar, parity)) return true;
+        if (sleep_ns) __nanosleep(sleep_ns);
+    }
     const long long t0 = clock64();
     for (;;) {
-        for (int i = 0; i < 256; ++i)
+        for (int i = 0; i < 64; ++i) {
             if (mbar_try(bar, parity)) return true;
+            if (sleep_ns) __nanosleep(sleep_ns);
+        }
         if (*(volatile int *)&ctl->abort_flag) return false;
         if (clock64() - t0 > kWaitCycles) {
             *(volatile int *)&ctl->abort_flag = 1;
@@ -157,10 +176,10 @@ __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, Ctl 
         }
     }
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, Ctl *ctl, int *status)
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, Ctl *ctl, int *status, uint32_t sleep_ns = 0)
 {
     if (mbar_try(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, ctl, status);
+    return mbar_wait_slow(bar, parity, ctl, status, sleep_ns);
 }
 
 // Bounded wait for a grid-wide counter to reach `target` (acquire).
@@ -305,7 +324,7 @@ __device__ __forceinline__ void exp_acc2(float2 &acc, uint32_t v0, uint32_t v1, 
 // would waste registers: pass 1 passes a pointer to a 4-float broadcast instead, see STRIDE).
 // STRIDE = 1: bias[t]; STRIDE = 0: the same 4 floats for every quad.
 template <int STRIDE>
-__device__ __forceinline__ void exp_acc32(float2 &a0, float2 &a1, const uint32_t (&v)[32], float2 cc, const float4 *bias)
+__device__ __forceinline__ void exp_acc32(float2 &a0, float2 &a1, const uint32_t *v, float2 cc, const float4 *bias)
 {
 #pragma unroll
     for (int t = 0; t < 32; t += 16) {
@@ -322,11 +341,12 @@ __device__ __forceinline__ void exp_acc32(float2 &a0, float2 &a1, const uint32_t
     }
 }
 
-__device__ __forceinline__ float max32(const uint32_t (&v)[32])
+template <int N>
+__device__ __forceinline__ float max_of(const uint32_t (&v)[N])
 {
     float c0 = -INFINITY, c1 = -INFINITY;
 #pragma unroll
-    for (int t = 0; t < 32; t += 4) {
+    for (int t = 0; t < N; t += 4) {
         c0 = max3(c0, __uint_as_float(v[t + 0]), __uint_as_float(v[t + 1]));
         c1 = max3(c1, __uint_as_float(v[t + 2]), __uint_as_float(v[t + 3]));
     }
@@ -387,6 +407,8 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, stages = P.stages;
+    const int tph = P.tph, L = P.L, R = P.R, Rpad = P.Rpad;   // register copies: the loops below must not touch memory for them
+    int *const status = P.status;
     const int nblk = P.Rbox / 128;                            // accumulator blocks per tile, both passes
     const int nseg = 2 * P.ngroups;
 
@@ -413,31 +435,32 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             TR_DECL;
-            uint32_t it = 0, qn = 0;
+            uint32_t st = 0, ph = 0, qn = 0;                  // ring stage and its phase; query loads so far
             int prev_kv = -1;
             bool ok = true;
 #pragma unroll 1
             for (int s = 0; s < nseg && ok; ++s) {
                 const Seg sg = segment(s, P);
+                const int pass = sg.pass, ntiles = sg.ntiles;
                 int kv = sg.kv0, tt = sg.t0;
 #pragma unroll 1
-                for (int n = 0; n < sg.ntiles; ++n, ++it, walk(sg.pass, P.tph, kv, tt)) {
+                for (int n = 0; n < ntiles; ++n, walk(pass, tph, kv, tt)) {
                     TR_ADD(2);
                     if (kv != prev_kv) {
                         const uint32_t qb = qn & 1;
-                        if (!mbar_wait(&ctl->q_empty[qb], ((qn >> 1) & 1) ^ 1, ctl, P.status)) { ok = false; break; }
+                        if (!mbar_wait(&ctl->q_empty[qb], ((qn >> 1) & 1) ^ 1, ctl, status, kSleepLong)) { ok = false; break; }
                         mbar_expect_tx(&ctl->q_full[qb], q_bytes);
                         tma_load_3d(qbuf + (size_t)qb * q_bytes, &mapQ, &ctl->q_full[qb], 0, 0, kv);
                         tma_load_3d(qbuf + (size_t)qb * q_bytes + q_bytes / 2, &mapQ, &ctl->q_full[qb], 64, 0, kv);
                         prev_kv = kv; ++qn;
                         TR_ADD(0);
                     }
-                    const uint32_t st = it % stages;
-                    if (!mbar_wait(&ctl->empty[st], ((it / stages) & 1) ^ 1, ctl, P.status)) { ok = false; break; }
+                    if (!mbar_wait(&ctl->empty[st], ph ^ 1, ctl, status, kSleepLong)) { ok = false; break; }
                     TR_ADD(1);
                     mbar_expect_tx(&ctl->full[st], kStageBytes);
                     tma_load_3d(kbuf + (size_t)st * kStageBytes, &mapK, &ctl->full[st], 0, tt * kTile, kv);
                     tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, &mapK, &ctl->full[st], 64, tt * kTile, kv);
+                    if (++st == (uint32_t)stages) { st = 0; ph ^= 1; }
                 }
             }
             TR_DUMP;
@@ -448,190 +471,215 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             TR_DECL;
             const uint32_t idesc1 = instr_desc(128, kTile);
             // pass 2: a block's columns are the query rows it covers, rounded up to 16
-            const uint32_t idesc2a = instr_desc(kTile, min(128, P.Rpad)), idesc2b = instr_desc(kTile, max(16, P.Rpad - 128));
-            uint32_t it = 0, qn = 0, u = 0;                   // tiles, query loads, accumulator blocks so far
+            const uint32_t idesc2a = instr_desc(kTile, min(128, Rpad)), idesc2b = instr_desc(kTile, max(16, Rpad - 128));
+            uint32_t st = 0, ph = 0, qn = 0, u = 0;           // ring stage and phase, query loads, accumulator blocks so far
             int prev_kv = -1;
             bool ok = true;
 #pragma unroll 1
             for (int s = 0; s < nseg && ok; ++s) {
                 const Seg sg = segment(s, P);
+                const int pass = sg.pass, ntiles = sg.ntiles;
                 int kv = sg.kv0, tt = sg.t0;
 #pragma unroll 1
-                for (int n = 0; n < sg.ntiles && ok; ++n, ++it, walk(sg.pass, P.tph, kv, tt)) {
+                for (int n = 0; n < ntiles && ok; ++n, walk(pass, tph, kv, tt)) {
                     TR_ADD(4);
                     if (kv != prev_kv) {
                         if (qn > 0) tc_commit(&ctl->q_empty[(qn - 1) & 1]);   // the previous head's queries are free once its MMAs retire
-                        if (!mbar_wait(&ctl->q_full[qn & 1], (qn >> 1) & 1, ctl, P.status)) { ok = false; break; }
+                        if (!mbar_wait(&ctl->q_full[qn & 1], (qn >> 1) & 1, ctl, status, kSleepShort)) { ok = false; break; }
                         prev_kv = kv; ++qn;
                         TR_ADD(0);
                     }
-                    const uint32_t st = it % stages;
-                    if (!mbar_wait(&ctl->full[st], (it / stages) & 1, ctl, P.status)) { ok = false; break; }
+                    if (!mbar_wait(&ctl->full[st], ph, ctl, status, kSleepShort)) { ok = false; break; }
                     TR_ADD(1);
                     const uint32_t k_lo = desc_lo(smem_u32(kbuf) + st * kStageBytes);
                     const uint32_t q_lo = desc_lo(smem_u32(qbuf) + ((qn - 1) & 1) * q_bytes);
 #pragma unroll 1
                     for (int blk = 0; blk < nblk; ++blk, ++u) {
                         const uint32_t slot = u % kTSlots;
-                        if (!mbar_wait(&ctl->t_empty[slot], ((u / kTSlots) & 1) ^ 1, ctl, P.status)) { ok = false; break; }
+                        if (!mbar_wait(&ctl->t_empty[slot], ((u / kTSlots) & 1) ^ 1, ctl, status, kSleepShort)) { ok = false; break; }
                         TR_ADD(2);
                         tc_fence_after();
                         const uint32_t d = tmem + slot * kSlotCols;
                         const uint32_t qb_lo = q_lo + (uint32_t)blk * (kHalfBytes >> 4);   // query rows [128 blk, 128 blk + 128)
-                        if (sg.pass == 1) tc_mma_block(d, qb_lo, k_lo, q_bytes / 2, kHalfBytes, idesc1);
+                        if (pass == 1) tc_mma_block(d, qb_lo, k_lo, q_bytes / 2, kHalfBytes, idesc1);
                         else tc_mma_block(d, k_lo, qb_lo, kHalfBytes, q_bytes / 2, blk == 0 ? idesc2a : idesc2b);
                         tc_commit(&ctl->t_full[slot]);
                         TR_ADD(3);
                     }
                     if (ok) tc_commit(&ctl->empty[st]);
+                    if (++st == (uint32_t)stages) { st = 0; ph ^= 1; }
                 }
             }
             TR_DUMP;
         }
     } else if (warp < kMergeWarp) {
         // ---------------------------------------------------------------- epilogue groups
+        // A warp only visits the accumulator blocks of its own group (every kGroups-th block of the
+        // CTA's sequence) and moves its tile cursor by the tiles in between: the code outside the
+        // exponential stream is executed at a fraction of an instruction per clock, so there must be
+        // little of it.
         const int grp = (warp - 2) >> 2, quarter = warp & 3;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         const int row0 = quarter * 32 + lane;                   // TMEM lane: query row within its block (pass 1), key within its tile (pass 2)
+        const int blk_shift = nblk - 1;                         // blocks per tile is 1 or 2
         const float c = P.c;
         const float2 cc = make_float2(c, c);
-        uint32_t u = 0, hs = 0;                                 // accumulator blocks so far; pass-2 heads so far
+        float *const scores_out = P.scores;
+        float2 *const part_out = P.part + (size_t)(kGroups * blockIdx.x + grp) * R;
+        uint32_t u = 0;                                         // accumulator blocks of the CTA before this segment
+        int hs = 0;                                             // pass-2 heads of the CTA before this segment
         bool ok = true;
         TR_DECL;
 
 #pragma unroll 1
         for (int s = 0; s < nseg; ++s) {
             const Seg sg = segment(s, P);
-            int prev_kv = -1;
-            int kv = sg.kv0, tt = sg.t0;
+            const int ntiles = sg.ntiles, nunits = ntiles << blk_shift;
+            int kv = sg.kv0, tt = sg.t0, at = 0;                // tile cursor: head, tile in head, index in the segment
+            int k = (grp + kGroups - (int)(u % kGroups)) % kGroups;   // this group's first block of the segment
             if (sg.pass == 1) {
                 // Per block of 128 query rows: l = sum_j exp2(c (s_j - m)) against a REFERENCE m that need
-                // not be the row max: it is the max of the first 32 values seen and is only raised when later
-                // values would push the sum towards overflow (those 32 are then redone from their
-                // registers).  Any reference gives the same M_r = c m + log2(l) after the merge.
+                // not be the row max: it is the max of the first values seen and is only raised when later
+                // values would push the sum towards overflow (they are then redone from their registers).
+                // Any reference gives the same M_r = c m + log2(l) after the merge.
                 struct RowState { float m; float2 l01, l23; };
                 RowState st0 = {-INFINITY, make_float2(0.f, 0.f), make_float2(0.f, 0.f)}, st1 = st0;
+                int pub = sg.kv0;                               // next head whose partials this warp has to publish
+                // Every group publishes a partial for every head of the CTA's range, an empty one if it saw no block of it.
+                auto publish_upto = [&](int head_end) {
 #pragma unroll 1
-                for (int n = 0; n <= sg.ntiles; ++n, walk(1, P.tph, kv, tt)) {
-                    if (n == sg.ntiles || kv != prev_kv) {
-                        if (prev_kv >= 0) {
-                            // publish this warp's partials of the head just left
-                            float2 *dst = P.part + ((size_t)prev_kv * kSlots + kGroups * blockIdx.x + grp) * P.R;
-                            if (ok && row0 < P.R) dst[row0] = make_float2(st0.m, (st0.l01.x + st0.l01.y) + (st0.l23.x + st0.l23.y));
-                            if (ok && nblk == 2 && row0 + 128 < P.R)
-                                dst[row0 + 128] = make_float2(st1.m, (st1.l01.x + st1.l01.y) + (st1.l23.x + st1.l23.y));
-                            st0.m = st1.m = -INFINITY;
-                            st0.l01 = st0.l23 = st1.l01 = st1.l23 = make_float2(0.f, 0.f);
-                        }
-                        if (n == sg.ntiles) break;
-                        prev_kv = kv;
+                    for (; pub < head_end; ++pub) {
+                        float2 *dst = part_out + (size_t)pub * kSlots * R;
+                        if (row0 < R) dst[row0] = make_float2(st0.m, (st0.l01.x + st0.l01.y) + (st0.l23.x + st0.l23.y));
+                        if (nblk == 2 && row0 + 128 < R)
+                            dst[row0 + 128] = make_float2(st1.m, (st1.l01.x + st1.l01.y) + (st1.l23.x + st1.l23.y));
+                        st0.m = st1.m = -INFINITY;
+                        st0.l01 = st0.l23 = st1.l01 = st1.l23 = make_float2(0.f, 0.f);
                     }
-                    const int valid = min(kTile, P.L - tt * kTile);
+                };
 #pragma unroll 1
-                    for (int blk = 0; blk < nblk; ++blk, ++u) {
-                        if ((int)(u % kGroups) != grp) continue;
-                        const uint32_t slot = u % kTSlots;
-                        TR_ADD(8);
-                        if (ok) ok = mbar_wait(&ctl->t_full[slot], (u / kTSlots) & 1, ctl, P.status);
-                        if (!ok) continue;
-                        TR_ADD(0);
-                        tc_fence_after();
-                        const uint32_t taddr = lane_addr + slot * kSlotCols;
-                        // one copy of the block code: the second row block borrows the first one's registers
-                        if (blk == 1) { const RowState t = st0; st0 = st1; st1 = t; }
+                for (; k < nunits && ok; k += kGroups) {
+                    const int tl = k >> blk_shift, blk = k & blk_shift;
+                    for (; at < tl; ++at) walk(1, tph, kv, tt);
+                    publish_upto(kv);
+                    const uint32_t uu = u + (uint32_t)k, slot = uu % kTSlots;
+                    TR_ADD(8);
+                    ok = mbar_wait(&ctl->t_full[slot], (uu / kTSlots) & 1, ctl, status, kSleepShort);
+                    if (!ok) break;
+                    TR_ADD(0);
+                    tc_fence_after();
+                    const uint32_t taddr = lane_addr + slot * kSlotCols;
+                    const int valid = min(kTile, L - tt * kTile);
+                    // one copy of the block code: the second row block borrows the first one's registers
+                    if (blk == 1) { const RowState t = st0; st0 = st1; st1 = t; }
 #pragma unroll 1
-                        for (int c0 = 0; c0 < kTile; c0 += 32) {
-                            uint32_t v[32];
-                            JQ_TMEM_LD32(taddr + c0, v);
-                            tmem_ld_wait();
-                            TR_ADD(1);
-                            if (c0 + 32 == kTile) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], 1); }
-                            if (valid < c0 + 32) {
+                    for (int c0 = 0; c0 < kTile; c0 += kChunk) {
+                        uint32_t v[kChunk];
+                        if (kChunk == 64) JQ_TMEM_LD64(taddr + c0, v); else JQ_TMEM_LD32(taddr + c0, v);
+                        tmem_ld_wait();
+                        TR_ADD(1);
+                        if (c0 + kChunk == kTile) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], 1); }
+                        if (valid < c0 + kChunk) {
 #pragma unroll
-                                for (int t = 0; t < 32; ++t) if (c0 + t >= valid) v[t] = 0xff800000u;   // -inf: not a key
-                            }
-                            if (st0.m == -INFINITY) st0.m = max32(v);
-                            const float2 keep01 = st0.l01, keep23 = st0.l23;
-#pragma unroll 1
-                            for (int attempt = 0; attempt < 2; ++attempt) {
-                                const float nb = -st0.m * c;
-                                const float4 b4 = make_float4(nb, nb, nb, nb);
-                                exp_acc32<0>(st0.l01, st0.l23, v, cc, &b4);
-                                const float lsum = (st0.l01.x + st0.l01.y) + (st0.l23.x + st0.l23.y);
-                                if (lsum < 1.0e30f) break;
-                                // the reference is too far below these values: raise it to their max and redo them
-                                const float cm = fmaxf(max32(v), st0.m);
-                                const float f = ex2(c * (st0.m - cm));
-                                st0.l01 = make_float2(keep01.x * f, keep01.y * f);
-                                st0.l23 = make_float2(keep23.x * f, keep23.y * f);
-                                st0.m = cm;
-                            }
-                            TR_ADD(2);
+                            for (int t = 0; t < kChunk; ++t) if (c0 + t >= valid) v[t] = 0xff800000u;   // -inf: not a key
                         }
-                        if (blk == 1) { const RowState t = st0; st0 = st1; st1 = t; }
+                        if (st0.m == -INFINITY) st0.m = max_of<kChunk>(v);
+                        const float2 keep01 = st0.l01, keep23 = st0.l23;
+#pragma unroll 1
+                        for (int attempt = 0; attempt < 2; ++attempt) {
+                            const float nb = -st0.m * c;
+                            const float4 b4 = make_float4(nb, nb, nb, nb);
+#pragma unroll
+                            for (int h = 0; h < kChunk; h += 32) exp_acc32<0>(st0.l01, st0.l23, v + h, cc, &b4);
+                            const float lsum = (st0.l01.x + st0.l01.y) + (st0.l23.x + st0.l23.y);
+                            if (lsum < 1.0e30f) break;
+                            // the reference is too far below these values: raise it to their max and redo them
+                            const float cm = fmaxf(max_of<kChunk>(v), st0.m);
+                            const float f = ex2(c * (st0.m - cm));
+                            st0.l01 = make_float2(keep01.x * f, keep01.y * f);
+                            st0.l23 = make_float2(keep23.x * f, keep23.y * f);
+                            st0.m = cm;
+                        }
+                        TR_ADD(2);
                     }
+                    if (blk == 1) { const RowState t = st0; st0 = st1; st1 = t; }
                 }
                 TR_ADD(8);
+                if (ok && ntiles > 0) {
+                    for (; at < ntiles - 1; ++at) walk(1, tph, kv, tt);
+                    publish_upto(kv + 1);
+                }
                 // this warp's share of pass 1 of the group is published: count it in
                 __threadfence();
                 __syncwarp();
-                if (lane == 0) atomicAdd(P.status + kWCnt1 + (sg.g & (kRing - 1)), 1);
+                if (lane == 0) atomicAdd(status + kWCnt1 + (sg.g & (kRing - 1)), 1);
                 TR_ADD(6);
             } else {
-                const float *Ms = ctl->Ms[0];
+                // Heads of the segment are numbered hs, hs + 1, ... in walking order (descending KV head); the
+                // stage warp fills buffer (number & 1).  `held` is the number of the head whose normalisers
+                // this warp currently reads, hs - 1 before the first.
+                int held = hs - 1;
+                auto hold = [&](int want) {
 #pragma unroll 1
-                for (int n = 0; n < sg.ntiles; ++n, walk(2, P.tph, kv, tt)) {
-                    if (kv != prev_kv) {
-                        TR_ADD(10);
-                        // done with the previous head's normalisers; wait for this head's
-                        if (prev_kv >= 0) {
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(&ctl->ms_empty[(hs - 1) & 1], 1);
-                        }
-                        if (ok) ok = mbar_wait(&ctl->ms_full[hs & 1], (hs >> 1) & 1, ctl, P.status);
-                        Ms = ctl->Ms[hs & 1];
-                        ++hs;
-                        prev_kv = kv;
-                        TR_ADD(4);
+                    while (held < want && ok) {
+                        if (held >= hs) { __syncwarp(); if (lane == 0) mbar_arrive(&ctl->ms_empty[held & 1], 1); }
+                        ++held;
+                        ok = mbar_wait(&ctl->ms_full[held & 1], (held >> 1) & 1, ctl, status, kSleepShort);
                     }
+                };
 #pragma unroll 1
-                    for (int blk = 0; blk < nblk; ++blk, ++u) {
-                        if ((int)(u % kGroups) != grp) continue;
-                        const uint32_t slot = u % kTSlots;
-                        TR_ADD(10);
-                        if (ok) ok = mbar_wait(&ctl->t_full[slot], (u / kTSlots) & 1, ctl, P.status);
-                        if (!ok) continue;
-                        TR_ADD(3);
-                        tc_fence_after();
-                        const uint32_t taddr = lane_addr + slot * kSlotCols;
-                        const int ncols = min(128, P.Rpad - blk * 128);    // accumulator columns of this block
-                        const float *bias = Ms + blk * 128;                 // columns that are not query rows carry a bias of -inf
-                        float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
+                for (; k < nunits && ok; k += kGroups) {
+                    const int tl = k >> blk_shift, blk = k & blk_shift;
+                    for (; at < tl; ++at) walk(2, tph, kv, tt);
+                    TR_ADD(10);
+                    hold(hs + (sg.kv0 - kv));
+                    if (!ok) break;
+                    TR_ADD(4);
+                    const uint32_t uu = u + (uint32_t)k, slot = uu % kTSlots;
+                    ok = mbar_wait(&ctl->t_full[slot], (uu / kTSlots) & 1, ctl, status, kSleepShort);
+                    if (!ok) break;
+                    TR_ADD(3);
+                    tc_fence_after();
+                    const uint32_t taddr = lane_addr + slot * kSlotCols;
+                    const int ncols = min(128, Rpad - blk * 128);      // accumulator columns of this block
+                    const float *bias = ctl->Ms[held & 1] + blk * 128;  // columns that are not query rows carry a bias of -inf
+                    float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
 #pragma unroll 1
-                        for (int c0 = 0; c0 < ncols; c0 += 32) {
-                            uint32_t v[32];
-                            JQ_TMEM_LD32(taddr + c0, v);
-                            tmem_ld_wait();
-                            TR_ADD(1);
-                            if (c0 + 32 >= ncols) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], 1); }
-                            exp_acc32<1>(a01, a23, v, cc, (const float4 *)(bias + c0));
-                            TR_ADD(5);
+                    for (int c0 = 0; c0 < ncols; c0 += kChunk) {
+                        uint32_t v[kChunk];
+                        if (kChunk == 64) JQ_TMEM_LD64(taddr + c0, v); else JQ_TMEM_LD32(taddr + c0, v);
+                        tmem_ld_wait();
+                        TR_ADD(1);
+                        if (c0 + kChunk >= ncols) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], 1); }
+                        if (ncols < c0 + kChunk) {
+                            // columns the MMA did not write hold whatever tensor memory held: make them finite (their bias is -inf)
+#pragma unroll
+                            for (int t = 0; t < kChunk; ++t) if (c0 + t >= ncols) v[t] = 0u;
                         }
-                        const int key = tt * kTile + row0;
-                        if (key < P.L) {
-                            float *dst = P.scores + (size_t)kv * P.L + key;
-                            const float sum = (a01.x + a01.y) + (a23.x + a23.y);
-                            if (nblk == 1) *dst = sum;
-                            else atomicAdd(dst, sum);              // two blocks per key, onto a zero the stage warp wrote
-                        }
+#pragma unroll
+                        for (int h = 0; h < kChunk; h += 32) exp_acc32<1>(a01, a23, v + h, cc, (const float4 *)(bias + c0 + h));
+                        TR_ADD(5);
                     }
-                }
-                if (prev_kv >= 0) {
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&ctl->ms_empty[(hs - 1) & 1], 1);
+                    const int key = tt * kTile + row0;
+                    if (key < L) {
+                        float *dst = scores_out + (size_t)kv * L + key;
+                        const float sum = (a01.x + a01.y) + (a23.x + a23.y);
+                        if (nblk == 1) *dst = sum;
+                        else atomicAdd(dst, sum);              // two blocks per key, onto a zero the stage warp wrote
+                    }
                 }
                 TR_ADD(10);
+                // take part in the hand-over of every remaining head of the segment, then give the last one back
+                if (ntiles > 0) {
+                    for (; at < ntiles - 1; ++at) walk(2, tph, kv, tt);
+                    const int nheads = sg.kv0 - kv + 1;
+                    hold(hs + nheads - 1);
+                    if (ok) { __syncwarp(); if (lane == 0) mbar_arrive(&ctl->ms_empty[held & 1], 1); }
+                    hs += nheads;
+                }
+                TR_ADD(4);
             }
+            u += (uint32_t)nunits;
         }
         TR_DUMP;
     } else if (warp == kMergeWarp) {
@@ -716,7 +764,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             if (sg.pass != 2 || sg.ntiles == 0) continue;
             if (nblk == 2) {
                 int kv = sg.kv0, tt = sg.t0;
-                for (int n = 0; n < sg.ntiles; ++n, walk(2, P.tph, kv, tt)) {
+                for (int n = 0; n < sg.ntiles; ++n, walk(2, tph, kv, tt)) {
                     float *dst = P.scores + (size_t)kv * P.L + tt * kTile;
                     for (int t = lane; t < kTile && tt * kTile + t < P.L; t += 32) dst[t] = 0.f;
                 }
@@ -729,11 +777,11 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             int prev_kv = -1;
             int kv = sg.kv0, tt = sg.t0;
 #pragma unroll 1
-            for (int n = 0; n < sg.ntiles && ok; ++n, walk(2, P.tph, kv, tt)) {
+            for (int n = 0; n < sg.ntiles && ok; ++n, walk(2, tph, kv, tt)) {
                 if (kv == prev_kv) continue;
                 prev_kv = kv;
                 const uint32_t buf = hs & 1;
-                ok = mbar_wait(&ctl->ms_empty[buf], ((hs >> 1) & 1) ^ 1, ctl, P.status) ? 1 : 0;
+                ok = mbar_wait(&ctl->ms_empty[buf], ((hs >> 1) & 1) ^ 1, ctl, status, kSleepLong) ? 1 : 0;
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 for (int r = lane; r < kMaxR; r += 32)   // stored negated: x = c s + (-M_r); -inf silences a padding column
