@@ -117,8 +117,7 @@ jq_status jq_evict_layer(const void *K, const void *V, const void *Qwin, const j
     if ((rc = check_ws(s, ws, ws_bytes, &w)) != JQ_OK) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     if ((rc = launch_score_tc(K, Qwin, *s, w.scores, w, st)) != JQ_OK) return rc;
-    if ((rc = launch_select(w.scores, *s, kept_idx, nullptr, w, st)) != JQ_OK) return rc;
-    return launch_gather(K, V, kept_idx, *s, Kout, Vout, st);
+    return launch_select(w.scores, *s, kept_idx, nullptr, w, st, K, V, Kout, Vout);   // selects, then copies the kept rows
 }
 
 size_t jq_host_call_bytes(const jq_shape *s)

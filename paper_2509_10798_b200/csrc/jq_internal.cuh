@@ -58,8 +58,10 @@ jq_status launch_score_fma(const void *K, const void *Q, const jq_shape &s, floa
                            const Workspace &w, cudaStream_t st);
 jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float *scores,
                           const Workspace &w, cudaStream_t st);
+// With K, V, Kout, Vout given, the kernel also copies the kept rows (the fused layer path).
 jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, float *pooled,
-                        const Workspace &w, cudaStream_t st);
+                        const Workspace &w, cudaStream_t st, const void *K = nullptr, const void *V = nullptr,
+                        void *Kout = nullptr, void *Vout = nullptr);
 jq_status launch_gather(const void *K, const void *V, const int32_t *idx, const jq_shape &s,
                         void *Kout, void *Vout, cudaStream_t st);
 

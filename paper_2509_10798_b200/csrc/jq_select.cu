@@ -5,12 +5,16 @@
 //      the positions and keeps its keys in shared memory (in the workspace for very long prefixes).
 //   2. radix select, 3 rounds of 11/11/10 bits, most significant first: local integer histograms
 //      are summed into the leading CTA through distributed shared memory, which finds the digit
-//      holding the nkeep-th largest key and broadcasts it.  Result: the key tau of the nkeep-th
-//      largest element and how many elements equal to tau are kept.  Max-pooling copies every peak
+//      holding the nkeep-th largest key and broadcasts it.  After the first round the keys that
+//      share that digit are normally few: they are then copied into the leading CTA, which runs
+//      the two remaining rounds on them alone (no further pass over all keys, no further
+//      histogram traffic).  Result: the key tau of the nkeep-th largest element and how many
+//      elements equal to tau are kept.  Max-pooling copies every peak
 //      into up to `pool` neighbours, so ties at tau are the normal case: all keys > tau are kept,
 //      then the lowest-index keys == tau.
 //   3. ordered compaction: kept positions are written in ascending order (CTA rank, warp,
 //      iteration and lane order all follow the position order).
+//   4. (fused layer path only) the cluster copies the kept K and V rows of its head.
 // Everything is integer arithmetic on bit patterns, hence deterministic and exact.
 #include "jq_internal.cuh"
 #include <cooperative_groups.h>
@@ -23,14 +27,18 @@ namespace {
 constexpr int kCl = 8;             // CTAs per cluster (= per KV head)
 constexpr int kSelThreads = 1024;
 constexpr int kBins = 2048;
-constexpr int kRawTile = 4096;     // scores staged per pooling step
+constexpr int kRawTile = 20480;    // scores staged per pooling step (a CTA's whole share unless the prefix is very long)
 constexpr int kHalo = 32;          // >= pool radius
-constexpr int kKeysSmemMax = 36864; // keys a CTA can keep in shared memory
+constexpr int kKeysSmemMax = 24576; // keys a CTA can keep in shared memory
+constexpr int kCandMax = 8192;     // candidates the leading CTA finishes alone (they live in its staging buffer)
+static_assert(kCandMax <= kRawTile, "candidates are kept in the staging buffer");
 
 struct SelCtl {
     uint32_t prefix;
     int krem;
-    int found_prefix_digit, found_krem;
+    int found_prefix_digit, found_krem, found_count;
+    int cand_total;      // keys sharing the first-round digit (broadcast by the leading CTA)
+    int cand_count;      // leading CTA only: candidates appended so far
     int counts_gt[kCl], counts_eq[kCl];
     int warp_gt[32], warp_eq[32];
     int tot_gt, tot_eq;
@@ -71,10 +79,46 @@ __device__ __forceinline__ int block_excl_scan(int v, int *warp_sums)
     return excl;
 }
 
+// All 1024 threads of a CTA: in a histogram of kBins bins find, walking the bins from the top, the bin
+// that holds the krem-th element; leaves the bin, the rank within it and its population in ctl.
+__device__ __forceinline__ void find_digit(const uint32_t *g, int krem, SelCtl &ctl)
+{
+    // bins in descending order: thread t looks at bins 2047-2t and 2046-2t
+    const int hi = kBins - 1 - 2 * (int)threadIdx.x, lo = hi - 1;
+    const int h_hi = (int)g[hi], h_lo = (int)g[lo];
+    const int above = block_excl_scan(h_hi + h_lo, ctl.scan);
+    if (above < krem && krem <= above + h_hi) {
+        ctl.found_prefix_digit = hi; ctl.found_krem = krem - above; ctl.found_count = h_hi;
+    } else if (above + h_hi < krem && krem <= above + h_hi + h_lo) {
+        ctl.found_prefix_digit = lo; ctl.found_krem = krem - above - h_hi; ctl.found_count = h_lo;
+    }
+    __syncthreads();
+}
+
+// The cluster copies the kept K and V rows of its head (256 bytes each: 16 lanes x 16 bytes), CTA r the
+// r-th eighth of them, once every index of the head has been written.
+__device__ __forceinline__ void copy_kept_rows(cg::cluster_group &cluster, const int32_t *out, int kv, int L, int nkeep,
+                                               const uint4 *Kin, const uint4 *Vin, uint4 *Kout, uint4 *Vout)
+{
+    __threadfence();
+    cluster.sync();
+    const int rank = (int)cluster.block_rank();
+    const int r0 = (int)((long long)rank * nkeep / kCl), r1 = (int)((long long)(rank + 1) * nkeep / kCl);
+    const int lane16 = threadIdx.x & 15;
+    for (int t = r0 + (int)(threadIdx.x >> 4); t < r1; t += kSelThreads / 16) {
+        const int j = min(max(__ldcg(out + t), 0), L - 1);
+        const size_t src = ((size_t)kv * L + j) * 16 + lane16, dst = ((size_t)kv * nkeep + t) * 16 + lane16;
+        Kout[dst] = Kin[src];
+        Vout[dst] = Vin[src];
+    }
+}
+
 // grid (Hkv * 8), cluster 8, block 1024.
 __global__ void __cluster_dims__(kCl, 1, 1) __launch_bounds__(kSelThreads, 1)
 select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, int32_t *__restrict__ idx,
-               float *__restrict__ pooled, uint32_t *__restrict__ gkeys, int chunk, int keys_in_smem)
+               float *__restrict__ pooled, uint32_t *__restrict__ gkeys, int chunk, int keys_in_smem,
+               const uint4 *__restrict__ Kin, const uint4 *__restrict__ Vin, uint4 *__restrict__ Kout,
+               uint4 *__restrict__ Vout)
 {
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
@@ -110,10 +154,11 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     }
     if (nkeep >= L) {   // everything is kept (uniform over the cluster; no cluster traffic yet)
         for (int e = tid; e < n; e += kSelThreads) out[j0 + e] = j0 + e;
+        if (Kin) copy_kept_rows(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout);
         return;
     }
     for (int i = tid; i < 3 * kBins; i += kSelThreads) ghist[i] = 0;
-    if (tid == 0) { ctl.prefix = 0; ctl.krem = nkeep; }
+    if (tid == 0) { ctl.prefix = 0; ctl.krem = nkeep; ctl.cand_count = 0; ctl.cand_total = 0; }
     cluster.sync();
 
     // ---- 2. radix select
@@ -146,25 +191,61 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         }
         cluster.sync();
         if (rank == 0) {
-            // bins in descending order: thread t looks at bins 2047-2t and 2046-2t
-            const uint32_t *g = ghist + round * kBins;
-            const int hi = kBins - 1 - 2 * tid, lo = hi - 1;
-            const int h_hi = (int)g[hi], h_lo = (int)g[lo];
-            const int above = block_excl_scan(h_hi + h_lo, ctl.scan);
-            const int krem = ctl.krem;
-            if (above < krem && krem <= above + h_hi) {
-                ctl.found_prefix_digit = hi; ctl.found_krem = krem - above;
-            } else if (above + h_hi < krem && krem <= above + h_hi + h_lo) {
-                ctl.found_prefix_digit = lo; ctl.found_krem = krem - above - h_hi;
-            }
-            __syncthreads();
+            find_digit(ghist + round * kBins, ctl.krem, ctl);
             if (tid < kCl) {
                 SelCtl *rc = cluster.map_shared_rank(&ctl, tid);
                 rc->prefix = (prefix << width) | (uint32_t)ctl.found_prefix_digit;
                 rc->krem = ctl.found_krem;
+                rc->cand_total = ctl.found_count;
             }
         }
         cluster.sync();
+        if (round == 0 && ctl.cand_total <= kCandMax) {
+            // The keys with the winning first digit go to the leading CTA (order does not matter: only
+            // their values decide the threshold), which finishes the selection on them alone.
+            const uint32_t d0 = ctl.prefix;
+            uint32_t *cand = (uint32_t *)cluster.map_shared_rank(raw, 0);
+            int *cand_count = &cluster.map_shared_rank(&ctl, 0)->cand_count;
+            for (int base = 0; base < n_up; base += kSelThreads) {
+                const int e = base + tid;
+                const uint32_t k = (e < n) ? mykeys[e] : 0u;
+                const bool hit = e < n && (k >> 21) == d0;
+                const uint32_t votes = __ballot_sync(0xffffffffu, hit);
+                if (votes) {
+                    int at = 0;
+                    if (lane == 0) at = atomicAdd(cand_count, __popc(votes));
+                    at = __shfl_sync(0xffffffffu, at, 0);
+                    if (hit) cand[at + __popc(votes & ((1u << lane) - 1u))] = k;
+                }
+            }
+            cluster.sync();
+            if (rank == 0) {
+                const int nc = ctl.cand_total;
+                const uint32_t *mine = (const uint32_t *)raw;
+                uint32_t pre = d0;
+                for (int r2 = 1; r2 < 3; ++r2) {
+                    const int sh = (r2 == 1) ? 10 : 0, wd = (r2 == 2) ? 10 : 11;
+                    for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
+                    __syncthreads();
+                    for (int e = tid; e < nc; e += kSelThreads) {
+                        const uint32_t k = mine[e];
+                        if ((k >> (sh + wd)) == pre) atomicAdd(&hist[(k >> sh) & ((1u << wd) - 1u)], 1u);
+                    }
+                    __syncthreads();
+                    find_digit(hist, ctl.krem, ctl);
+                    pre = (pre << wd) | (uint32_t)ctl.found_prefix_digit;
+                    if (tid == 0) ctl.krem = ctl.found_krem;
+                    __syncthreads();
+                }
+                if (tid < kCl) {
+                    SelCtl *rc = cluster.map_shared_rank(&ctl, tid);
+                    rc->prefix = pre;
+                    rc->krem = ctl.found_krem;
+                }
+            }
+            cluster.sync();
+            break;
+        }
     }
     const uint32_t tau = ctl.prefix;
     const int need_eq = ctl.krem;   // how many of the keys == tau are kept (lowest positions first)
@@ -217,12 +298,13 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         gt_before += __popc(bg);
         eq_before += __popc(be);
     }
+    if (Kin) copy_kept_rows(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout);
 }
 
 }  // namespace
 
 jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, float *pooled,
-                        const Workspace &w, cudaStream_t st)
+                        const Workspace &w, cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout)
 {
     const int nkeep = s.budget < s.L ? s.budget : s.L;
     int chunk = (s.L + kCl - 1) / kCl;
@@ -239,7 +321,8 @@ jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, fl
         attr_done[dev] = true;
     }
     select_cluster<<<s.Hkv * kCl, kSelThreads, smem, st>>>(scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, w.keys,
-                                                          chunk, in_smem);
+                                                          chunk, in_smem, (const uint4 *)K, (const uint4 *)V,
+                                                          (uint4 *)Kout, (uint4 *)Vout);
     count_launch(1);
     return check_launch();
 }
