@@ -140,11 +140,20 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     for (int t0 = 0; t0 < n; t0 += kRawTile) {
         const int tile = min(kRawTile, n - t0);
         __syncthreads();
-        for (int i = tid; i < tile + 2 * radius; i += kSelThreads) {
-            const int j = j0 + t0 - radius + i;
-            raw[i] = (j >= 0 && j < L) ? s[j] : -INFINITY;
+        // eight loads in flight per thread: the scores come from L2, one round trip each
+        for (int i0 = tid; i0 < tile + 2 * radius; i0 += 8 * kSelThreads) {
+            float vals[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int j = j0 + t0 - radius + i0 + q * kSelThreads;
+                vals[q] = (i0 + q * kSelThreads < tile + 2 * radius && j >= 0 && j < L) ? __ldcg(s + j) : -INFINITY;
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (i0 + q * kSelThreads < tile + 2 * radius) raw[i0 + q * kSelThreads] = vals[q];
         }
         __syncthreads();
+#pragma unroll 4
         for (int e = tid; e < tile; e += kSelThreads) {
             float best = raw[e];
             for (int u = 1; u <= 2 * radius; ++u) best = fmaxf(best, raw[e + u]);
@@ -170,18 +179,27 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
         __syncthreads();
         const uint32_t prefix = ctl.prefix;
-        for (int base = 0; base < n_up; base += kSelThreads) {   // uniform trip count: whole warps reach the match
-            const int e = base + tid;
-            bool live = false;
-            uint32_t digit = 0;
-            if (e < n) {
+        // A thread takes a run of consecutive keys and adds equal neighbouring digits as one count: the
+        // max-pool leaves plateaus, so a few additions per thread replace one per key.
+        {
+            const int per = (n + kSelThreads - 1) / kSelThreads;
+            const int e0 = min(tid * per, n), e1 = min(e0 + per, n);
+            uint32_t cur = 0xffffffffu, cnt = 0;
+            int pos = per ? tid % per : 0;                      // rotated start: neighbouring threads hit different banks
+            for (int i = 0; i < per; ++i) {
+                const int e = e0 + pos;
+                if (++pos == per) pos = 0;
+                if (e >= e1) continue;
                 const uint32_t k = mykeys[e];
-                live = (round == 0) || ((k >> (shift + width)) == prefix);
-                digit = (k >> shift) & mask;
+                const bool live = (round == 0) || ((k >> (shift + width)) == prefix);
+                const uint32_t digit = live ? ((k >> shift) & mask) : 0xffffffffu;
+                if (digit != cur) {
+                    if (cnt && cur != 0xffffffffu) atomicAdd(&hist[cur], cnt);
+                    cur = digit; cnt = 0;
+                }
+                ++cnt;
             }
-            const uint32_t tag = live ? digit : 0xffffffffu;
-            const uint32_t peers = __match_any_sync(0xffffffffu, tag);
-            if (live && (__ffs(peers) - 1) == lane) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
+            if (cnt && cur != 0xffffffffu) atomicAdd(&hist[cur], cnt);
         }
         __syncthreads();
         uint32_t *g0 = cluster.map_shared_rank(ghist + round * kBins, 0);
