@@ -69,7 +69,9 @@ size_t jq_workspace_bytes(const jq_shape *shape);
 /*
  * Zeroes the status word at the head of a workspace.  Call once after allocating `ws` and before
  * its first use (on the stream that will use it); the status then accumulates over all later calls
- * until it is read with jq_last_device_status or cleared by calling this again.
+ * until it is read with jq_last_device_status or cleared by calling this again.  The block also holds
+ * the counters the scoring kernel's CTAs synchronise through; a call that ended in JQ_ERR_TIMEOUT
+ * leaves them undefined, so call this again before reusing the workspace after such an error.
  */
 jq_status jq_workspace_init(void *ws, size_t ws_bytes, jq_stream_t stream);
 

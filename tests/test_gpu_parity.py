@@ -243,3 +243,26 @@ def test_cfg5_full_size_sampled_heads():
         for kv in range(wl.Hkv):
             assert np.all(np.diff(gidx[kv]) > 0)
             assert np.array_equal(gKo[kv], K[kv][gidx[kv]]) and np.array_equal(gVo[kv], V[kv][gidx[kv]])
+
+
+# ------------------------------------------------------------------ bounded waits (failure is made on the host)
+
+def test_wait_that_nothing_ends_times_out_and_leaves_the_context_usable():
+    """A grid counter the kernel waits for is set, from the host, to a value it can never reach.  Every wait
+    in the kernel is bounded, so the call must come back with JQ_ERR_TIMEOUT in the status word (no trap,
+    no hang), and the same workspace must work again after jq_workspace_init."""
+    wl = small_wl(2, 4, 16, 700, 1)
+    K, _, Q, _ = W.make_layer(wl, with_v=False)
+    s = shape_of(wl)
+    ws = jq.new_workspace(s)
+    torch.cuda.synchronize()
+    ws.view(torch.int32)[8] = -(1 << 28)            # first pass-1 completion counter: unreachable
+    out = torch.zeros((s.Hkv, s.L), dtype=torch.float32, device="cuda")
+    jq.score(dev_bf16(K), dev_bf16(Q), s, out, ws)
+    assert jq.last_device_status(ws) == jq.JQ_ERR_TIMEOUT
+    lib = jq.lib()
+    import ctypes
+    assert lib.jq_workspace_init(ctypes.c_void_p(ws.data_ptr()), ws.numel(), ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)) == jq.JQ_OK
+    jq.score(dev_bf16(K), dev_bf16(Q), s, out, ws)
+    assert jq.last_device_status(ws) == jq.JQ_OK
+    assert_scores_close(out.cpu().numpy(), oracle.score(K, Q))
