@@ -538,10 +538,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             int kv = sg.kv0, tt = sg.t0, at = 0;                // tile cursor: head, tile in head, index in the segment
             int k = (grp + kGroups - (int)(u % kGroups)) % kGroups;   // this group's first block of the segment
             if (sg.pass == 1) {
-                // Per block of 128 query rows: l = sum_j exp2(c (s_j - m)) against a REFERENCE m that need
-                // not be the row max: it is the max of the first values seen and is only raised when later
-                // values would push the sum towards overflow (they are then redone from their registers).
-                // Any reference gives the same M_r = c m + log2(l) after the merge.
+                // Per block of 128 query rows: running max m and l = sum_j exp2(c (s_j - m)).
                 struct RowState { float m; float2 l01, l23; };
                 RowState st0 = {-INFINITY, make_float2(0.f, 0.f), make_float2(0.f, 0.f)}, st1 = st0;
                 int pub = sg.kv0;                               // next head whose partials this warp has to publish
@@ -583,23 +580,20 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll
                             for (int t = 0; t < kChunk; ++t) if (c0 + t >= valid) v[t] = 0xff800000u;   // -inf: not a key
                         }
-                        if (st0.m == -INFINITY) st0.m = max_of<kChunk>(v);
-                        const float2 keep01 = st0.l01, keep23 = st0.l23;
-#pragma unroll 1
-                        for (int attempt = 0; attempt < 2; ++attempt) {
-                            const float nb = -st0.m * c;
-                            const float4 b4 = make_float4(nb, nb, nb, nb);
-#pragma unroll
-                            for (int h = 0; h < kChunk; h += 32) exp_acc32<0>(st0.l01, st0.l23, v + h, cc, &b4);
-                            const float lsum = (st0.l01.x + st0.l01.y) + (st0.l23.x + st0.l23.y);
-                            if (lsum < 1.0e30f) break;
-                            // the reference is too far below these values: raise it to their max and redo them
-                            const float cm = fmaxf(max_of<kChunk>(v), st0.m);
-                            const float f = ex2(c * (st0.m - cm));
-                            st0.l01 = make_float2(keep01.x * f, keep01.y * f);
-                            st0.l23 = make_float2(keep23.x * f, keep23.y * f);
+                        // online softmax statistics: the reference is the running max, raised (and l rescaled) when
+                        // a piece brings a larger value; the max runs on the ALU pipe and, unlike a check of the
+                        // sum, does not wait for the exponentials in flight
+                        const float cm = max_of<kChunk>(v);
+                        if (cm > st0.m) {
+                            const float f = ex2(c * (st0.m - cm));   // 0 for the first piece (m = -inf)
+                            st0.l01 = make_float2(st0.l01.x * f, st0.l01.y * f);
+                            st0.l23 = make_float2(st0.l23.x * f, st0.l23.y * f);
                             st0.m = cm;
                         }
+                        const float nb = -st0.m * c;
+                        const float4 b4 = make_float4(nb, nb, nb, nb);
+#pragma unroll
+                        for (int h = 0; h < kChunk; h += 32) exp_acc32<0>(st0.l01, st0.l23, v + h, cc, &b4);
                         TR_ADD(2);
                     }
                     if (blk == 1) { const RowState t = st0; st0 = st1; st1 = t; }
