@@ -70,7 +70,8 @@ constexpr int kMaxStages = 5;                    // K ring depth (5 when R <= 12
 constexpr int kGroups = JQ_GROUPS;               // epilogue groups of 128 threads
 constexpr int kTSlots = 4;                       // accumulator slots in tensor memory
 constexpr int kEpiWarps = 4 * kGroups;
-constexpr int kMergeWarp = 2 + kEpiWarps, kStageWarp = kMergeWarp + 1;
+constexpr int kFirstEpiWarp = 3;                 // warps 1 and 2 issue the MMAs
+constexpr int kMergeWarp = kFirstEpiWarp + kEpiWarps, kStageWarp = kMergeWarp + 1;
 constexpr int kThreads = (kStageWarp + 1) * 32;
 constexpr uint32_t kHalfBytes = kTile * 128;     // one 64-column half of a K tile (128-byte rows)
 constexpr uint32_t kStageBytes = 2 * kHalfBytes; // 32 KiB
@@ -413,9 +414,9 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     const int nseg = 2 * P.ngroups;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], nblk); }   // one release per MMA issuer
         for (int s = 0; s < 2; ++s) {
-            mbar_init(&ctl->q_full[s], 1); mbar_init(&ctl->q_empty[s], 1);
+            mbar_init(&ctl->q_full[s], 1); mbar_init(&ctl->q_empty[s], nblk);
             mbar_init(&ctl->ms_full[s], 1); mbar_init(&ctl->ms_empty[s], kEpiWarps);
         }
         for (int s = 0; s < kTSlots; ++s) { mbar_init(&ctl->t_full[s], 1); mbar_init(&ctl->t_empty[s], 128); }
@@ -465,14 +466,18 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             }
             TR_DUMP;
         }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
+    } else if (warp < kFirstEpiWarp) {
+        // ---------------------------------------------------------------- MMA issuers
+        // Two threads (one per warp) share the issue work: with two accumulator blocks per tile, issuer b
+        // takes block b of every tile; with one, issuer 0 works alone.  One thread could not keep up:
+        // an accumulator block costs it about a thousand cycles of issue and loop time.
+        const int which = warp - 1;
+        if (lane == 0 && which < nblk) {
             TR_DECL;
             const uint32_t idesc1 = instr_desc(128, kTile);
             // pass 2: a block's columns are the query rows it covers, rounded up to 16
             const uint32_t idesc2a = instr_desc(kTile, min(128, Rpad)), idesc2b = instr_desc(kTile, max(16, Rpad - 128));
-            uint32_t st = 0, ph = 0, qn = 0, u = 0;           // ring stage and phase, query loads, accumulator blocks so far
+            uint32_t st = 0, ph = 0, qn = 0, u = (uint32_t)which;   // ring stage and phase, query loads, this issuer's next accumulator block
             int prev_kv = -1;
             bool ok = true;
 #pragma unroll 1
@@ -493,8 +498,8 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     TR_ADD(1);
                     const uint32_t k_lo = desc_lo(smem_u32(kbuf) + st * kStageBytes);
                     const uint32_t q_lo = desc_lo(smem_u32(qbuf) + ((qn - 1) & 1) * q_bytes);
-#pragma unroll 1
-                    for (int blk = 0; blk < nblk; ++blk, ++u) {
+                    {
+                        const int blk = which;
                         const uint32_t slot = u % kTSlots;
                         if (!mbar_wait(&ctl->t_empty[slot], ((u / kTSlots) & 1) ^ 1, ctl, status, kSleepShort)) { ok = false; break; }
                         TR_ADD(2);
@@ -505,6 +510,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                         else tc_mma_block(d, k_lo, qb_lo, kHalfBytes, q_bytes / 2, blk == 0 ? idesc2a : idesc2b);
                         tc_commit(&ctl->t_full[slot]);
                         TR_ADD(3);
+                        u += (uint32_t)nblk;
                     }
                     if (ok) tc_commit(&ctl->empty[st]);
                     if (++st == (uint32_t)stages) { st = 0; ph ^= 1; }
@@ -518,7 +524,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         // CTA's sequence) and moves its tile cursor by the tiles in between: the code outside the
         // exponential stream is executed at a fraction of an instruction per clock, so there must be
         // little of it.
-        const int grp = (warp - 2) >> 2, quarter = warp & 3;
+        const int grp = (warp - kFirstEpiWarp) >> 2, quarter = warp & 3;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         const int row0 = quarter * 32 + lane;                   // TMEM lane: query row within its block (pass 1), key within its tile (pass 2)
         const int blk_shift = nblk - 1;                         // blocks per tile is 1 or 2
