@@ -70,8 +70,7 @@ constexpr int kMaxStages = 5;                    // K ring depth (5 when R <= 12
 constexpr int kGroups = JQ_GROUPS;               // epilogue groups of 128 threads
 constexpr int kTSlots = 4;                       // accumulator slots in tensor memory
 constexpr int kEpiWarps = 4 * kGroups;
-constexpr int kFirstEpiWarp = 3;                 // warps 1 and 2 issue the MMAs
-constexpr int kMergeWarp = kFirstEpiWarp + kEpiWarps, kStageWarp = kMergeWarp + 1;
+constexpr int kMergeWarp = 2 + kEpiWarps, kStageWarp = kMergeWarp + 1;
 constexpr int kThreads = (kStageWarp + 1) * 32;
 constexpr uint32_t kHalfBytes = kTile * 128;     // one 64-column half of a K tile (128-byte rows)
 constexpr uint32_t kStageBytes = 2 * kHalfBytes; // 32 KiB
@@ -211,9 +210,16 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, u
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// Issued by ONE lane of a converged warp (the whole warp runs the issuing code so that its address
+// arithmetic stays warp-uniform; only the tensor-core instructions themselves are predicated).
 __device__ __forceinline__ void tc_commit(uint64_t *bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+    __syncwarp();
+    asm volatile(
+        "{\n\t.reg .pred pe;\n\t"
+        "elect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar)) : "memory");
 }
 
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, shape M x N.
@@ -221,8 +227,6 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
-
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ float ex2(float x)
 {
@@ -247,35 +251,38 @@ __device__ __forceinline__ uint32_t desc_lo(uint32_t addr) { return ((addr >> 4)
 
 // One accumulator block: D[tmem] = A[smem] * B[smem]^T over the whole head dimension (8 steps of 16),
 // both operands K-major bf16 in two 64-column halves `a_half` / `b_half` bytes apart, fp32 accumulate.
-// A single straight-line sequence: the issuing thread shares its scheduler with epilogue warps, so
-// every instruction it does not execute is time the tensor pipe does not wait.
+// A single straight-line sequence run by the whole (converged) warp with one elected lane issuing: the
+// warp shares its scheduler with epilogue warps, so every instruction it does not execute is time the
+// tensor pipe does not wait.
 __device__ __forceinline__ void tc_mma_block(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_half,
                                              uint32_t b_half, uint32_t idesc)
 {
     const uint32_t a1 = a_lo + (a_half >> 4), b1 = b_lo + (b_half >> 4);
+    __syncwarp();
     asm volatile(
         "{\n\t"
-        ".reg .pred pz, po;\n\t"
+        ".reg .pred pz, po, pe;\n\t"
         ".reg .b64 da, db;\n\t"
         ".reg .b32 ta, tb;\n\t"
         "setp.ne.u32 pz, %0, %0;\n\t"
         "setp.eq.u32 po, %0, %0;\n\t"
+        "elect.sync _|pe, 0xffffffff;\n\t"
         "mov.b64 da, {%1, %5};\n\t mov.b64 db, {%2, %5};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, pz;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, pz;\n\t"
         "add.u32 ta, %1, 2;\n\t add.u32 tb, %2, 2;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
         "add.u32 ta, %1, 4;\n\t add.u32 tb, %2, 4;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
         "add.u32 ta, %1, 6;\n\t add.u32 tb, %2, 6;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
         "mov.b64 da, {%3, %5};\n\t mov.b64 db, {%4, %5};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
         "add.u32 ta, %3, 2;\n\t add.u32 tb, %4, 2;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
         "add.u32 ta, %3, 4;\n\t add.u32 tb, %4, 4;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
         "add.u32 ta, %3, 6;\n\t add.u32 tb, %4, 6;\n\t mov.b64 da, {ta, %5};\n\t mov.b64 db, {tb, %5};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, po;\n\t"
         "}"
         ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(a1), "r"(b1), "r"(kDescHi), "r"(idesc) : "memory");
 }
@@ -414,9 +421,9 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     const int nseg = 2 * P.ngroups;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], nblk); }   // one release per MMA issuer
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(&ctl->q_full[s], 1); mbar_init(&ctl->q_empty[s], nblk);
+            mbar_init(&ctl->q_full[s], 1); mbar_init(&ctl->q_empty[s], 1);
             mbar_init(&ctl->ms_full[s], 1); mbar_init(&ctl->ms_empty[s], kEpiWarps);
         }
         for (int s = 0; s < kTSlots; ++s) { mbar_init(&ctl->t_full[s], 1); mbar_init(&ctl->t_empty[s], 128); }
@@ -466,18 +473,14 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             }
             TR_DUMP;
         }
-    } else if (warp < kFirstEpiWarp) {
-        // ---------------------------------------------------------------- MMA issuers
-        // Two threads (one per warp) share the issue work: with two accumulator blocks per tile, issuer b
-        // takes block b of every tile; with one, issuer 0 works alone.  One thread could not keep up:
-        // an accumulator block costs it about a thousand cycles of issue and loop time.
-        const int which = warp - 1;
-        if (lane == 0 && which < nblk) {
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer (all 32 lanes walk the loop)
+        {
             TR_DECL;
             const uint32_t idesc1 = instr_desc(128, kTile);
             // pass 2: a block's columns are the query rows it covers, rounded up to 16
             const uint32_t idesc2a = instr_desc(kTile, min(128, Rpad)), idesc2b = instr_desc(kTile, max(16, Rpad - 128));
-            uint32_t st = 0, ph = 0, qn = 0, u = (uint32_t)which;   // ring stage and phase, query loads, this issuer's next accumulator block
+            uint32_t st = 0, ph = 0, qn = 0, u = 0;           // ring stage and phase, query loads, accumulator blocks so far
             int prev_kv = -1;
             bool ok = true;
 #pragma unroll 1
@@ -498,8 +501,8 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     TR_ADD(1);
                     const uint32_t k_lo = desc_lo(smem_u32(kbuf) + st * kStageBytes);
                     const uint32_t q_lo = desc_lo(smem_u32(qbuf) + ((qn - 1) & 1) * q_bytes);
-                    {
-                        const int blk = which;
+#pragma unroll 1
+                    for (int blk = 0; blk < nblk; ++blk, ++u) {
                         const uint32_t slot = u % kTSlots;
                         if (!mbar_wait(&ctl->t_empty[slot], ((u / kTSlots) & 1) ^ 1, ctl, status, kSleepShort)) { ok = false; break; }
                         TR_ADD(2);
@@ -510,7 +513,6 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                         else tc_mma_block(d, k_lo, qb_lo, kHalfBytes, q_bytes / 2, blk == 0 ? idesc2a : idesc2b);
                         tc_commit(&ctl->t_full[slot]);
                         TR_ADD(3);
-                        u += (uint32_t)nblk;
                     }
                     if (ok) tc_commit(&ctl->empty[st]);
                     if (++st == (uint32_t)stages) { st = 0; ph ^= 1; }
@@ -524,7 +526,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         // CTA's sequence) and moves its tile cursor by the tiles in between: the code outside the
         // exponential stream is executed at a fraction of an instruction per clock, so there must be
         // little of it.
-        const int grp = (warp - kFirstEpiWarp) >> 2, quarter = warp & 3;
+        const int grp = (warp - 2) >> 2, quarter = warp & 3;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         const int row0 = quarter * 32 + lane;                   // TMEM lane: query row within its block (pass 1), key within its tile (pass 2)
         const int blk_shift = nblk - 1;                         // blocks per tile is 1 or 2
@@ -579,7 +581,6 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     for (int c0 = 0; c0 < kTile; c0 += kChunk) {
                         uint32_t v[kChunk];
                         if (kChunk == 64) JQ_TMEM_LD64(taddr + c0, v); else JQ_TMEM_LD32(taddr + c0, v);
-                        tmem_ld_wait();
                         TR_ADD(1);
                         if (c0 + kChunk == kTile) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], 1); }
                         if (valid < c0 + kChunk) {
@@ -648,7 +649,6 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     for (int c0 = 0; c0 < ncols; c0 += kChunk) {
                         uint32_t v[kChunk];
                         if (kChunk == 64) JQ_TMEM_LD64(taddr + c0, v); else JQ_TMEM_LD32(taddr + c0, v);
-                        tmem_ld_wait();
                         TR_ADD(1);
                         if (c0 + kChunk >= ncols) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], 1); }
                         if (ncols < c0 + kChunk) {

@@ -266,3 +266,20 @@ def test_wait_that_nothing_ends_times_out_and_leaves_the_context_usable():
     jq.score(dev_bf16(K), dev_bf16(Q), s, out, ws)
     assert jq.last_device_status(ws) == jq.JQ_OK
     assert_scores_close(out.cpu().numpy(), oracle.score(K, Q))
+
+
+def test_score_full_size_is_bitwise_repeatable():
+    """The 128K-key, 256-row workload three times in a row: every launch must give the same bits (all
+    reductions have a fixed order; the two additions per key of the wide mode commute)."""
+    wl = W.CFG5
+    K, _, Q, _ = W.make_layer(wl, with_v=False)
+    s = shape_of(wl)
+    ws = jq.new_workspace(s)
+    dK, dQ = dev_bf16(K), dev_bf16(Q)
+    outs = []
+    for _ in range(3):
+        out = torch.full((s.Hkv, s.L), -1.0, dtype=torch.float32, device="cuda")
+        jq.score(dK, dQ, s, out, ws)
+        assert jq.last_device_status(ws) == jq.JQ_OK
+        outs.append(out.cpu().numpy())
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
