@@ -96,7 +96,7 @@ jq_status jq_score(const void *K, const void *Qwin, const jq_shape *shape, float
  * free byte of the GPU to its KV-cache pool, a plug-in running inside somebody else's memory budget, a
  * call site that must not touch the allocator.  (The paper has no counterpart; this is a property of
  * the library.)  Same inputs, same output and the same kernel as jq_score, but no workspace argument:
- * the scratch the kernel needs sits in a device array built into the library, about 5.3 MB that every
+ * the scratch the kernel needs sits in a device array built into the library, about 10.5 MB that every
  * GPU using the library holds until the process exits.
  *  - Limit: Hkv * group * w <= 2048 query rows in total; a larger shape returns JQ_ERR_UNSUPPORTED and
  *    launches nothing.
