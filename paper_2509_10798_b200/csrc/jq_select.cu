@@ -131,6 +131,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     __shared__ SelCtl ctl;
 
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    cudaGridDependencySynchronize();   // everything above ran while the previous kernel of the stream was finishing
     const int j0 = min(rank * chunk, L), j1 = min(j0 + chunk, L), n = j1 - j0;
     const float *s = scores + (size_t)kv * L;
     uint32_t *mykeys = keys_in_smem ? keys_s : gkeys + (size_t)kv * L + j0;
@@ -338,9 +339,23 @@ jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, fl
             return JQ_ERR_CUDA;
         attr_done[dev] = true;
     }
-    select_cluster<<<s.Hkv * kCl, kSelThreads, smem, st>>>(scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, w.keys,
-                                                          chunk, in_smem, (const uint4 *)K, (const uint4 *)V,
-                                                          (uint4 *)Kout, (uint4 *)Vout);
+    // Launched with programmatic stream serialisation: the CTAs may be set up while the kernel before it in
+    // the stream (the scoring kernel) drains; the kernel waits for that kernel's memory before reading anything.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(s.Hkv * kCl));
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, select_cluster, scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, w.keys, chunk,
+                           in_smem, (const uint4 *)K, (const uint4 *)V, (uint4 *)Kout, (uint4 *)Vout) != cudaSuccess) {
+        cudaGetLastError();
+        return JQ_ERR_CUDA;
+    }
     count_launch(1);
     return check_launch();
 }
