@@ -438,6 +438,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *(volatile uint32_t *)&ctl->tmem_base;
+    cudaGridDependencySynchronize();   // no global memory has been touched so far
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
@@ -951,11 +952,14 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem_bytes(P.Rbox, P.stages);
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
+    // the CTAs may be set up (barriers, tensor-memory allocation) while the previous kernel of the stream drains
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, score_fused, mapK, mapQ, P) != cudaSuccess) {
         cudaGetLastError();
         return JQ_ERR_CUDA;
