@@ -102,6 +102,7 @@ struct Ctl {
     uint64_t q_full[2], q_empty[2];
     uint64_t t_full[kTSlots], t_empty[kTSlots];
     uint64_t ms_full[2], ms_empty[2];
+    uint64_t p1_done[2];               // all epilogue warps have published their pass-1 partials of a group
     uint32_t tmem_base;
     int abort_flag;
     alignas(16) float Ms[2][kMaxR];   // -M_r of the KV head being scored in pass 2, double-buffered; read as float4
@@ -425,6 +426,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         for (int s = 0; s < 2; ++s) {
             mbar_init(&ctl->q_full[s], 1); mbar_init(&ctl->q_empty[s], 1);
             mbar_init(&ctl->ms_full[s], 1); mbar_init(&ctl->ms_empty[s], kEpiWarps);
+            mbar_init(&ctl->p1_done[s], kEpiWarps);
         }
         for (int s = 0; s < kTSlots; ++s) { mbar_init(&ctl->t_full[s], 1); mbar_init(&ctl->t_empty[s], 128); }
         ctl->abort_flag = 0;
@@ -611,10 +613,10 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     for (; at < ntiles - 1; ++at) walk(1, tph, kv, tt);
                     publish_upto(kv + 1);
                 }
-                // this warp's share of pass 1 of the group is published: count it in
-                __threadfence();
+                // this warp's share of pass 1 of the group is published: tell the merge warp, which makes the
+                // stores visible to the grid and counts the CTA in (an epilogue warp does not wait for that)
                 __syncwarp();
-                if (lane == 0) atomicAdd(status + kWCnt1 + (sg.g & (kRing - 1)), 1);
+                if (lane == 0) mbar_arrive(&ctl->p1_done[sg.g & 1], 1);
                 TR_ADD(6);
             } else {
                 // Heads of the segment are numbered hs, hs + 1, ... in walking order (descending KV head); the
@@ -692,8 +694,15 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll 1
         for (int g = 0; g < P.ngroups; ++g) {
             int ok = 1;
-            if (lane == 0)
-                ok = wait_counter(P.status + kWCnt1 + (g & (kRing - 1)), (g / kRing + 1) * G * kEpiWarps, ctl, P.status) ? 1 : 0;
+            // this CTA's epilogue warps first (their partial stores happen-before the arrival), then the grid
+            ok = mbar_wait(&ctl->p1_done[g & 1], (g >> 1) & 1, ctl, P.status, kSleepLong) ? 1 : 0;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (lane == 0) {
+                __threadfence();
+                atomicAdd(P.status + kWCnt1 + (g & (kRing - 1)), 1);
+                ok = wait_counter(P.status + kWCnt1 + (g & (kRing - 1)), (g / kRing + 1) * G, ctl, P.status) ? 1 : 0;
+            }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             const int h0 = g * P.hpg, nh = min(P.hpg, P.Hkv - h0);
