@@ -102,7 +102,7 @@ struct Ctl {
     uint64_t q_full[2], q_empty[2];
     uint64_t t_full[kTSlots], t_empty[kTSlots];
     uint64_t ms_full[2], ms_empty[2];
-    uint64_t p1_done[2];               // all epilogue warps have published their pass-1 partials of a group
+    uint64_t p1_done[4];               // all epilogue warps have published their pass-1 partials of a group
     uint32_t tmem_base;
     int abort_flag;
     alignas(16) float Ms[2][kMaxR];   // -M_r of the KV head being scored in pass 2, double-buffered; read as float4
@@ -115,7 +115,7 @@ struct Params {
     int Hkv, tph;            // KV heads; tiles per head
     int hpg, ngroups;        // heads per group, groups
     int stages;              // K ring depth
-    int pipelined;           // 1: P1(0) P1(1) P2(0) P1(2) ... ; 0: P1(0) P2(0) P1(1) P2(1) ...
+    int depth;               // pass 2 of a group starts after pass 1 of `depth` groups: 1 = P1(0) P2(0) P1(1) ..., 2 = P1(0) P1(1) P2(0) P1(2) ..., 3 = P1(0) P1(1) P1(2) P2(0) ...
     float c;                 // log2(e) / sqrt(d)
     float2 *part;            // [Hkv][kSlots][R]
     float *Mrow;             // [Hkv][R]   c*m + log2(l) per query row
@@ -375,11 +375,10 @@ __device__ __noinline__ Seg segment(int s, const Params &P)
 {
     Seg sg;
     const int NG = P.ngroups;
-    if (!P.pipelined) { sg.g = s >> 1; sg.pass = 1 + (s & 1); }
-    else if (s == 0) { sg.pass = 1; sg.g = 0; }
-    else if (s == 2 * NG - 1) { sg.pass = 2; sg.g = NG - 1; }
-    else if (s & 1) { sg.pass = 1; sg.g = (s + 1) >> 1; }
-    else { sg.pass = 2; sg.g = (s >> 1) - 1; }
+    const int D = min(P.depth, NG), t = s - D;
+    if (s < D) { sg.pass = 1; sg.g = s; }                                  // lead-in: pass 1 of the first D groups
+    else if (t < 2 * (NG - D)) { sg.pass = (t & 1) ? 1 : 2; sg.g = (t & 1) ? D + (t >> 1) : (t >> 1); }
+    else { sg.pass = 2; sg.g = s - NG; }                                   // tail: the last D groups' pass 2
     sg.h0 = sg.g * P.hpg;
     const int nh = min(P.hpg, P.Hkv - sg.h0);
     const uint32_t T = (uint32_t)nh * P.tph, G = gridDim.x;
@@ -426,9 +425,9 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         for (int s = 0; s < 2; ++s) {
             mbar_init(&ctl->q_full[s], 1); mbar_init(&ctl->q_empty[s], 1);
             mbar_init(&ctl->ms_full[s], 1); mbar_init(&ctl->ms_empty[s], kEpiWarps);
-            mbar_init(&ctl->p1_done[s], kEpiWarps);
+
         }
-        for (int s = 0; s < kTSlots; ++s) { mbar_init(&ctl->t_full[s], 1); mbar_init(&ctl->t_empty[s], 128); }
+        for (int s = 0; s < kTSlots; ++s) { mbar_init(&ctl->t_full[s], 1); mbar_init(&ctl->t_empty[s], 128); mbar_init(&ctl->p1_done[s], kEpiWarps); }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -616,7 +615,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                 // this warp's share of pass 1 of the group is published: tell the merge warp, which makes the
                 // stores visible to the grid and counts the CTA in (an epilogue warp does not wait for that)
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->p1_done[sg.g & 1], 1);
+                if (lane == 0) mbar_arrive(&ctl->p1_done[sg.g & 3], 1);
                 TR_ADD(6);
             } else {
                 // Heads of the segment are numbered hs, hs + 1, ... in walking order (descending KV head); the
@@ -695,7 +694,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         for (int g = 0; g < P.ngroups; ++g) {
             int ok = 1;
             // this CTA's epilogue warps first (their partial stores happen-before the arrival), then the grid
-            ok = mbar_wait(&ctl->p1_done[g & 1], (g >> 1) & 1, ctl, P.status, kSleepLong) ? 1 : 0;
+            ok = mbar_wait(&ctl->p1_done[g & 3], (g >> 2) & 1, ctl, P.status, kSleepLong) ? 1 : 0;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             if (lane == 0) {
@@ -893,8 +892,8 @@ bool device_info(DeviceInfo *out)
     return true;
 }
 
-// Overrides for tuning runs (read once): JQ_SCORE_GROUP_MIB = K bytes per head group, JQ_SCORE_ORDER = 0
-// for the unpipelined segment order.
+// Overrides for tuning runs (read once): JQ_SCORE_GROUP_MIB = K bytes per head group, JQ_SCORE_DEPTH = 1..3,
+// the number of groups whose pass 1 precedes the first pass 2.
 long long env_ll(const char *name, long long dflt)
 {
     const char *v = getenv(name);
@@ -914,14 +913,14 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
     DeviceInfo dev;
     if (!device_info(&dev)) return JQ_ERR_CUDA;
     static const long long group_mib = env_ll("JQ_SCORE_GROUP_MIB", 32);
-    static const long long order = env_ll("JQ_SCORE_ORDER", 1);
+    static const long long order = env_ll("JQ_SCORE_DEPTH", 2);
     const int R = s.group * s.w;
     Params P;
     P.L = s.L; P.R = R; P.Rbox = R <= 128 ? 128 : 256; P.Rpad = (R + 15) & ~15;
     P.Hkv = s.Hkv;
     P.tph = (s.L + kTile - 1) / kTile;
     P.stages = P.Rbox == 128 ? 5 : 3;
-    P.pipelined = order != 0;
+    P.depth = order < 1 ? 1 : (order > 3 ? 3 : (int)order);
     P.c = 1.4426950408889634f / sqrtf((float)s.d);
     P.part = w.part; P.Mrow = w.Mrow; P.scores = scores; P.status = w.status;
 #ifdef JQ_TRACE
