@@ -138,6 +138,10 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     int32_t *out = idx + (size_t)kv * nkeep;
 
     // ---- 1. max-pool -> keys
+    // With the keys in shared memory and a window of at most 9, a thread pools four neighbouring
+    // positions from three 16-byte reads and the first-round histogram is built on the way.
+    const bool fast_pool = keys_in_smem && radius <= 4;
+    for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
     for (int t0 = 0; t0 < n; t0 += kRawTile) {
         const int tile = min(kRawTile, n - t0);
         __syncthreads();
@@ -153,7 +157,58 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
             for (int q = 0; q < 8; ++q)
                 if (i0 + q * kSelThreads < tile + 2 * radius) raw[i0 + q * kSelThreads] = vals[q];
         }
+        for (int i = tid; i < 8; i += kSelThreads) raw[tile + 2 * radius + i] = -INFINITY;   // the 16-byte reads run a little past the window
         __syncthreads();
+        if (fast_pool) {
+            const int nquads = (tile + 3) / 4;
+            const float4 *raw4 = (const float4 *)raw;
+            for (int base = 0; base < nquads; base += kSelThreads) {      // uniform trip count: whole warps reach the votes
+                const int g4 = base + tid;
+                const bool act = g4 < nquads;
+                float x[12];
+                {
+                    const float4 a = act ? raw4[g4] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    const float4 b = act ? raw4[g4 + 1] : a, c = act ? raw4[g4 + 2] : a;
+                    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+                    x[8] = c.x; x[9] = c.y; x[10] = c.z; x[11] = c.w;
+                }
+                uint32_t key[4];
+                float best[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float m = x[i];
+#pragma unroll
+                    for (int u = 1; u <= 8; ++u) if (u <= 2 * radius) m = fmaxf(m, x[i + u]);
+                    best[i] = m;
+                    key[i] = order_key(m);
+                }
+                const int nval = act ? min(4, tile - 4 * g4) : 0;          // positions of this quad inside the tile
+                if (act) {
+                    if (nval == 4) *(uint4 *)(mykeys + t0 + 4 * g4) = make_uint4(key[0], key[1], key[2], key[3]);
+                    else for (int i = 0; i < nval; ++i) mykeys[t0 + 4 * g4 + i] = key[i];
+                    if (pooled) for (int i = 0; i < nval; ++i) pooled[(size_t)kv * L + j0 + t0 + 4 * g4 + i] = best[i];
+                }
+                // first-round histogram: one addition per warp when all its positions share the digit (the usual
+                // case: 128 neighbouring positions of similar size), else runs of equal digits per thread
+                const uint32_t d0 = key[0] >> 21;
+                bool same = true;
+                for (int i = 1; i < 4; ++i) if (i < nval && (key[i] >> 21) != d0) same = false;
+                const uint32_t lead = __shfl_sync(0xffffffffu, d0, 0);
+                if (__all_sync(0xffffffffu, nval == 0 || (same && d0 == lead))) {
+                    const int tot = __reduce_add_sync(0xffffffffu, nval);
+                    if (lane == 0 && tot) atomicAdd(&hist[lead], (uint32_t)tot);
+                } else {
+                    uint32_t cur = 0, cnt = 0;
+                    for (int i = 0; i < nval; ++i) {
+                        const uint32_t d = key[i] >> 21;
+                        if (cnt && d != cur) { atomicAdd(&hist[cur], cnt); cnt = 0; }
+                        cur = d; ++cnt;
+                    }
+                    if (cnt) atomicAdd(&hist[cur], cnt);
+                }
+            }
+            continue;
+        }
 #pragma unroll 4
         for (int e = tid; e < tile; e += kSelThreads) {
             float best = raw[e];
@@ -177,12 +232,13 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         const int shift = (round == 0) ? 21 : (round == 1 ? 10 : 0);
         const int width = (round == 2) ? 10 : 11;
         const uint32_t mask = (1u << width) - 1u;
-        for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
+        const bool have_hist = round == 0 && fast_pool;          // built while pooling
+        if (!have_hist) for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
         __syncthreads();
         const uint32_t prefix = ctl.prefix;
         // A thread takes a run of consecutive keys and adds equal neighbouring digits as one count: the
         // max-pool leaves plateaus, so a few additions per thread replace one per key.
-        {
+        if (!have_hist) {
             const int per = (n + kSelThreads - 1) / kSelThreads;
             const int e0 = min(tid * per, n), e1 = min(e0 + per, n);
             uint32_t cur = 0xffffffffu, cnt = 0;
