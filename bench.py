@@ -4,7 +4,10 @@
     python bench.py --impl reference ...      # the fp64 CPU oracle, timed on the host cores
 
 One step = one pass of the whole hot path (scores -> pool -> top-k -> gather) over every layer of
-one synthetic cache: `layers` calls of jq_evict_layer on one stream.  Prints ONE JSON line.
+one synthetic cache, on one stream.  Every (layer, KV head) is an independent unit of the pass, so the
+layers of a cache are evicted by ONE jq_evict_layer call on tensors that stack the layers along the
+KV-head axis (`--call stacked`, the default: K, V [layers*Hkv, L, d], Qwin [layers*Hq, w, d]); the same
+work as `layers` separate calls (`--call per-layer`) is also timed and reported.  Prints ONE JSON line.
 With N > 1 (torchrun) every rank evicts a cache of its own (independent replicas, no collective on
 the data path); the value is the sum over ranks divided by the slowest rank's time.
 """
@@ -25,6 +28,8 @@ if ROOT not in sys.path:
 import jq_workloads as W  # noqa: E402
 
 METRIC = "prefix tokens evicted/sec per layer"
+# dram__bytes_read.sum + dram__bytes_write.sum of one score_fused launch on one layer (ncu, see profiles/)
+NCU_DRAM_BYTES_PER_LAYER = {}
 UNIT = "tokens/s"
 
 
@@ -37,6 +42,7 @@ def parse():
     ap.add_argument("--workload", default="cfg5", choices=["cfg2", "cfg3", "cfg5"])
     ap.add_argument("--budget", type=int, default=None)
     ap.add_argument("--layers", type=int, default=None, help="layer calls per step (default: the workload's)")
+    ap.add_argument("--call", default="stacked", choices=["stacked", "per-layer"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -51,9 +57,11 @@ def pick_workload(args):
     return wl
 
 
-def config_of(wl, layers, distinct):
+def config_of(wl, layers, distinct, call="per-layer"):
     return {"workload": wl.name, "L": wl.L, "Hkv": wl.Hkv, "Hq": wl.Hq, "d": wl.d, "w": wl.w,
             "budget": wl.budget, "pool": wl.pool, "layers_per_step": layers, "distinct_layers": distinct,
+            "call": ("one jq_evict_layer call per step, the layers stacked along the KV-head axis" if call == "stacked"
+                     else "one jq_evict_layer call per layer"),
             "l2": "inputs larger than L2 (K of one step: %.0f MiB)" % (distinct * wl.Hkv * wl.L * wl.d * 2 / 2**20)}
 
 
@@ -203,10 +211,28 @@ def run_ours(args):
     idx = torch.zeros((wl.Hkv, nkeep), dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()
 
-    def step():
+    def step_per_layer():
         for i in range(layers):
             j = i % distinct
             jq.evict_layer(Ks[j], Vs[j], Qs[j], s, Ko, Vo, idx, ws, stream=stream)
+
+    # the layers of the cache stacked along the KV-head axis (a layer repeated in the workload is copied, so
+    # that every layer of the step has memory of its own)
+    sS = jq.shape(wl.Hkv * layers, wl.Hq * layers, wl.L, wl.w, wl.budget, wl.pool, wl.d)
+    if args.call == "stacked":
+        order = [i % distinct for i in range(layers)]
+        KS = torch.cat([Ks[j] for j in order], 0)
+        VS = torch.cat([Vs[j] for j in order], 0)
+        QS = torch.cat([Qs[j] for j in order], 0)
+        wsS = jq.new_workspace(sS)
+        KoS = torch.zeros((sS.Hkv, nkeep, wl.d), dtype=torch.bfloat16, device="cuda")
+        VoS = torch.zeros_like(KoS)
+        idxS = torch.zeros((sS.Hkv, nkeep), dtype=torch.int32, device="cuda")
+
+    def step_stacked():
+        jq.evict_layer(KS, VS, QS, sS, KoS, VoS, idxS, wsS, stream=stream)
+
+    step = step_stacked if args.call == "stacked" else step_per_layer
 
     def barrier():
         if world > 1:
@@ -227,6 +253,24 @@ def run_ours(args):
     ms = e0.elapsed_time(e1)
     launches = jq.launch_count() - n0
     assert jq.last_device_status(ws) == jq.JQ_OK, "device status not ok"
+    if args.call == "stacked":
+        assert jq.last_device_status(wsS) == jq.JQ_OK, "device status not ok"
+        # the same work as one call per layer, for comparison (and its results must be the same bits)
+        for _ in range(3):
+            step_per_layer()
+        barrier()
+        e0.record(stream)
+        for _ in range(max(args.steps // 4, 3)):
+            step_per_layer()
+        e1.record(stream)
+        barrier()
+        ms_pl = e0.elapsed_time(e1) / max(args.steps // 4, 3)
+        jlast = (layers - 1) % distinct
+        assert torch.equal(idx, idxS[(layers - 1) * wl.Hkv:]) and torch.equal(Ko, KoS[(layers - 1) * wl.Hkv:]), \
+            "stacked call and per-layer call disagree"
+        per_layer_calls = {"ms_per_layer": ms_pl / layers, "value": world * wl.L / (ms_pl * 1e-3 / layers), "unit": UNIT}
+    else:
+        per_layer_calls = None
 
     # per-stage times through the stage entry points: batches of back-to-back calls between events on the
     # launching stream, so that host launch latency is not counted as device time
@@ -246,9 +290,16 @@ def run_ours(args):
         torch.cuda.synchronize()
         return ev[0].elapsed_time(ev[1]) / nb
 
-    stage_ms[0] = timed(lambda j: jq.score(Ks[j], Qs[j], s, scores[j % len(scores)], ws, stream=stream))
-    stage_ms[1] = timed(lambda j: jq.select_topk(scores[j % len(scores)], s, idx, ws, stream=stream))
-    stage_ms[2] = timed(lambda j: jq.compact_kv(Ks[j], Vs[j], idx, s, Ko, Vo, stream=stream))
+    if args.call == "stacked":
+        scoresS = torch.empty((sS.Hkv, wl.L), dtype=torch.float32, device="cuda")
+        nb = 4
+        stage_ms[0] = timed(lambda j: jq.score(KS, QS, sS, scoresS, wsS, stream=stream)) / layers
+        stage_ms[1] = timed(lambda j: jq.select_topk(scoresS, sS, idxS, wsS, stream=stream)) / layers
+        stage_ms[2] = timed(lambda j: jq.compact_kv(KS, VS, idxS, sS, KoS, VoS, stream=stream)) / layers
+    else:
+        stage_ms[0] = timed(lambda j: jq.score(Ks[j], Qs[j], s, scores[j % len(scores)], ws, stream=stream))
+        stage_ms[1] = timed(lambda j: jq.select_topk(scores[j % len(scores)], s, idx, ws, stream=stream))
+        stage_ms[2] = timed(lambda j: jq.compact_kv(Ks[j], Vs[j], idx, s, Ko, Vo, stream=stream))
     clocks = sampler.stop() if sampler else None
 
     t = torch.tensor([ms], dtype=torch.float64, device="cuda")
@@ -297,20 +348,33 @@ def run_ours(args):
             peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured"
     else:
         peak, peak_src = 6650.0, "fallback"
-    # dominant stage: the two scoring passes (jq_score); algorithmic bytes = two reads of K
-    score_bytes = 2 * wl.Hkv * wl.L * wl.d * 2
-    achieved = score_bytes / (stage_ms[0] * 1e-3) / 1e9
+    # dominant kernel: score_fused (jq_score, both passes); algorithmic bytes = two reads of K.  One launch
+    # covers one layer, or all stacked layers of the step.
+    per_launch = layers if args.call == "stacked" else 1
+    score_bytes = 2 * wl.Hkv * wl.L * wl.d * 2 * per_launch
+    ms_launch = float(stage_ms[0]) * per_launch
+    achieved = score_bytes / (ms_launch * 1e-3) / 1e9
     layer_gbs = W.formula_bytes(wl) / t_layer / 1e9
-    roofline = {"bound": "hbm", "kernel": "jq_score (pass 1 + pass 2)", "achieved": achieved, "peak": peak,
-                "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
-                "bytes_per_launch": score_bytes, "ms_per_launch": float(stage_ms[0]),
+    # DRAM bytes of one score_fused launch on ONE layer of this workload from an ncu capture of the kernel
+    # as it stands (profiles/), scaled to the launch by the layers it covers; None where no capture exists
+    traffic_one_layer = NCU_DRAM_BYTES_PER_LAYER.get(wl.name)
+    n_exp = 2.0 * wl.R * wl.L * wl.Hkv * per_launch                      # exponentials per launch
+    ex2_peak = 148 * 16 * 1965e6 / 1e9                                   # G/s: 16 results per clock per SM at the maximum SM clock
+    roofline = {"bound": "hbm", "kernel": "score_fused (jq_score, pass 1 + pass 2)", "achieved": achieved, "peak": peak,
+                "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None if traffic_one_layer is None else traffic_one_layer * per_launch,
+                "bytes_per_launch": score_bytes, "ms_per_launch": ms_launch,
                 "layer_formula_gbs": layer_gbs, "layer_frac_of_peak": layer_gbs / peak,
                 "layer_frac_of_8tbs": layer_gbs / 8000.0,
-                "stage_ms": {"score": float(stage_ms[0]), "select": float(stage_ms[1]), "compact": float(stage_ms[2])}}
+                "ex2_unit": {"note": "the unit that binds this kernel (DRAM is below a quarter of its peak under ncu)",
+                             "achieved": n_exp / (ms_launch * 1e-3) / 1e9, "peak": ex2_peak, "unit": "Gexp/s",
+                             "frac": n_exp / (ms_launch * 1e-3) / 1e9 / ex2_peak},
+                "stage_ms_per_layer": {"score": float(stage_ms[0]), "select": float(stage_ms[1]), "compact": float(stage_ms[2])}}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": config_of(wl, layers, distinct), "ms_per_layer": t_layer * 1e3,
+            "config": config_of(wl, layers, distinct, args.call), "ms_per_layer": t_layer * 1e3,
+            "per_layer_calls": per_layer_calls,
             "tokens_discarded_per_s": world * (wl.L - nkeep) / t_layer,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline}
     if not args.no_cpu_baseline and world == 1:

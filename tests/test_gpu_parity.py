@@ -283,3 +283,17 @@ def test_score_full_size_is_bitwise_repeatable():
         assert jq.last_device_status(ws) == jq.JQ_OK
         outs.append(out.cpu().numpy())
     assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+
+
+def test_layers_stacked_along_the_head_axis_equal_separate_calls():
+    """Every (layer, KV head) is an independent unit: one call on K, V, Qwin of several layers stacked along
+    the head axis must give, bit for bit, what one call per layer gives."""
+    wl = small_wl(2, 4, 32, 2500, 300)
+    layers = [W.make_layer(wl, layer=i) for i in range(3)]
+    K = np.concatenate([l[0] for l in layers]); V = np.concatenate([l[1] for l in layers]); Q = np.concatenate([l[2] for l in layers])
+    sS = jq.shape(wl.Hkv * 3, wl.Hq * 3, wl.L, wl.w, wl.budget, wl.pool, wl.d)
+    gKo, gVo, gidx = gpu_evict(K, V, Q, sS)
+    for i, (Ki, Vi, Qi, _) in enumerate(layers):
+        Ko, Vo, idx = gpu_evict(Ki, Vi, Qi, shape_of(wl))
+        sl = slice(i * wl.Hkv, (i + 1) * wl.Hkv)
+        assert np.array_equal(idx, gidx[sl]) and np.array_equal(Ko, gKo[sl]) and np.array_equal(Vo, gVo[sl])
