@@ -129,6 +129,24 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ----------------------------------------------------------------------------- N > 1: independent replicas
+
+def max_over_ranks(ms, world, device="cuda"):
+    """The job's time is the slowest rank's: all-reduce MAX of the rank-local milliseconds (no-op at N = 1)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(wl, world, t_layer):
+    """Whole-job throughput: every rank evicts a cache of its own (replicas, no data-path collective)."""
+    return world * wl.L / t_layer
+
+
 # ----------------------------------------------------------------------------- GPU arm
 
 class ClockSampler:
@@ -302,12 +320,9 @@ def run_ours(args):
         stage_ms[2] = timed(lambda j: jq.compact_kv(Ks[j], Vs[j], idx, s, Ko, Vo, stream=stream))
     clocks = sampler.stop() if sampler else None
 
-    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms = float(t.item())
+    ms = max_over_ranks(ms, world)
     t_layer = ms * 1e-3 / (args.steps * layers)
-    value = world * wl.L / t_layer
+    value = job_value(wl, world, t_layer)
 
     # end to end through the host-buffer entry point: pinned host tensors in, pinned host results out
     e2e = None
@@ -328,10 +343,7 @@ def run_ours(args):
             jq.evict_layer_host(hK, hV, hQ, s, hKo, hVo, hidx, buf, stream=stream)
         e1.record(stream)
         barrier()
-        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        t_e2e_layer = float(t.item()) * 1e-3 / (n_e2e * e2e_layers)
+        t_e2e_layer = max_over_ranks(e0.elapsed_time(e1), world) * 1e-3 / (n_e2e * e2e_layers)
         h2d = e2e_layers * (2 * hK.numel() + hQ.numel()) * 2
         d2h = e2e_layers * (2 * hKo.numel() * 2 + hidx.numel() * 4)
         e2e = {"value": world * wl.L / t_e2e_layer, "unit": UNIT, "h2d_bytes_per_step": h2d,
