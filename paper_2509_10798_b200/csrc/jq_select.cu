@@ -27,7 +27,7 @@ namespace {
 constexpr int kCl = 8;             // CTAs per cluster (= per KV head)
 constexpr int kSelThreads = 1024;
 constexpr int kBins = 2048;
-constexpr int kRawTile = 20480;    // scores staged per pooling step (a CTA's whole share unless the prefix is very long)
+constexpr int kRawTile = 20480;    // most scores staged per pooling step (a CTA's whole share unless the prefix is very long)
 constexpr int kHalo = 32;          // >= pool radius
 constexpr int kKeysSmemMax = 24576; // keys a CTA can keep in shared memory
 constexpr int kCandMax = 8192;     // candidates the leading CTA finishes alone (they live in its staging buffer)
@@ -114,9 +114,9 @@ __device__ __forceinline__ void copy_kept_rows(cg::cluster_group &cluster, const
 }
 
 // grid (Hkv * 8), cluster 8, block 1024.
-__global__ void __cluster_dims__(kCl, 1, 1) __launch_bounds__(kSelThreads, 1)
+__global__ void __cluster_dims__(kCl, 1, 1) __launch_bounds__(kSelThreads, 2)
 select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, int32_t *__restrict__ idx,
-               float *__restrict__ pooled, uint32_t *__restrict__ gkeys, int chunk, int keys_in_smem,
+               float *__restrict__ pooled, uint32_t *__restrict__ gkeys, int chunk, int keys_in_smem, int raw_tile,
                const uint4 *__restrict__ Kin, const uint4 *__restrict__ Vin, uint4 *__restrict__ Kout,
                uint4 *__restrict__ Vout)
 {
@@ -126,8 +126,8 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     extern __shared__ __align__(16) uint8_t sm[];
     uint32_t *ghist = (uint32_t *)sm;                       // [3][kBins]; the leading CTA's copy accumulates the cluster
     uint32_t *hist = ghist + 3 * kBins;                     // [kBins]
-    float *raw = (float *)(hist + kBins);                   // [kRawTile + 2*kHalo]
-    uint32_t *keys_s = (uint32_t *)(raw + kRawTile + 2 * kHalo);
+    float *raw = (float *)(hist + kBins);                   // [raw_tile + 2*kHalo]; later the candidate keys
+    uint32_t *keys_s = (uint32_t *)(raw + raw_tile + 2 * kHalo);
     __shared__ SelCtl ctl;
 
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -142,8 +142,8 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     // positions from three 16-byte reads and the first-round histogram is built on the way.
     const bool fast_pool = keys_in_smem && radius <= 4;
     for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
-    for (int t0 = 0; t0 < n; t0 += kRawTile) {
-        const int tile = min(kRawTile, n - t0);
+    for (int t0 = 0; t0 < n; t0 += raw_tile) {
+        const int tile = min(raw_tile, n - t0);
         __syncthreads();
         // eight loads in flight per thread: the scores come from L2, one round trip each
         for (int i0 = tid; i0 < tile + 2 * radius; i0 += 8 * kSelThreads) {
@@ -157,7 +157,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
             for (int q = 0; q < 8; ++q)
                 if (i0 + q * kSelThreads < tile + 2 * radius) raw[i0 + q * kSelThreads] = vals[q];
         }
-        for (int i = tid; i < 8; i += kSelThreads) raw[tile + 2 * radius + i] = -INFINITY;   // the 16-byte reads run a little past the window
+        if (fast_pool) for (int i = tid; i < 8; i += kSelThreads) raw[tile + 2 * radius + i] = -INFINITY;   // its 16-byte reads run a little past the window
         __syncthreads();
         if (fast_pool) {
             const int nquads = (tile + 3) / 4;
@@ -385,7 +385,11 @@ jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, fl
     int chunk = (s.L + kCl - 1) / kCl;
     chunk = (chunk + 31) / 32 * 32;
     const int in_smem = chunk <= kKeysSmemMax;
-    const size_t smem = (size_t)(4 * kBins + kRawTile + 2 * kHalo) * 4 + (in_smem ? (size_t)chunk * 4 : 0);
+    // the staging buffer holds a CTA's share of the scores (at most kRawTile) and later up to kCandMax candidates;
+    // sized to the shape so that two CTAs fit on an SM when the prefix is short
+    int raw_tile = chunk < kRawTile ? chunk : kRawTile;
+    if (raw_tile < kCandMax) raw_tile = kCandMax;
+    const size_t smem = (size_t)(4 * kBins + raw_tile + 2 * kHalo) * 4 + (in_smem ? (size_t)chunk * 4 : 0);
     static bool attr_done[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return JQ_ERR_CUDA;
@@ -408,7 +412,7 @@ jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, fl
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (cudaLaunchKernelEx(&cfg, select_cluster, scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, w.keys, chunk,
-                           in_smem, (const uint4 *)K, (const uint4 *)V, (uint4 *)Kout, (uint4 *)Vout) != cudaSuccess) {
+                           in_smem, raw_tile, (const uint4 *)K, (const uint4 *)V, (uint4 *)Kout, (uint4 *)Vout) != cudaSuccess) {
         cudaGetLastError();
         return JQ_ERR_CUDA;
     }
