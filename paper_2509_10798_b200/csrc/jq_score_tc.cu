@@ -4,14 +4,15 @@
 // another).  A CTA is warp-specialised:
 //   warp 0        TMA producer: K tiles of 128 keys (two 64-column halves, 128-byte swizzle) into a ring of
 //                 shared-memory stages; the query rows of a KV head into one of two stationary buffers;
-//   warp 1        issues tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory) and owns the TMEM allocation;
+//   warp 1        issues tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory; the warp stays converged, one
+//                 elected lane issues) and owns the TMEM allocation;
 //   warps 2..     kGroups epilogue groups of 128 threads.  Accumulator block u (128 TMEM lanes x 128
 //                 columns) sits in slot u % 4 and is taken by group u % kGroups, 32 columns at a time;
 //   then          one warp that merges the per-warp partial row statistics of pass 1 across the grid,
 //                 and one that stages the merged row normalisers of the next KV head of pass 2.
 // The operand roles are swapped between the passes so that no reduction crosses threads:
 //   pass 1  S[128 x 128] = Q K^T  (A = a block of 128 query rows): a thread owns a QUERY ROW and keeps
-//           l = sum_j exp2(c (s_j - m)) against a reference m; per-warp partial (m, l) go to the workspace;
+//           the running max m and l = sum_j exp2(c (s_j - m)); per-warp partial (m, l) go to the workspace;
 //   pass 2  S^T[128 x N] = K Q^T  (A = key tile, B = a block of up to 128 query rows): a thread owns a KEY
 //           and adds exp2(c s - M_r) over the rows, M_r = c m_r + log2(l_r) merged from the partials.
 //           With more than 128 query rows a key gets two blocks, added into the scores with red.add
@@ -33,9 +34,9 @@
 // roles then run out of their loops without touching data and leave through the common exit (which
 // frees the tensor memory).
 //
-// The code is kept small on purpose (rolled loops over 32-column pieces, one copy of each block routine,
-// 32-bit index arithmetic, no division per tile): the roles run different code on one SM, and what falls
-// out of the instruction cache costs hundreds of cycles at every turn of the outer loops.
+// The code outside the exponential stream is kept short (rolled loops over 32-column pieces, one copy of
+// each block routine, 32-bit index arithmetic, no division per tile, a warp visits only its own blocks):
+// a warp executes it at a fraction of an instruction per clock, and the ex2 unit idles meanwhile.
 #include "jq_internal.cuh"
 #include "jq_tmem_ld.cuh"
 #include <cuda.h>
