@@ -42,7 +42,7 @@ extern "C" {
 typedef enum {
     JQ_OK = 0,
     JQ_ERR_INVALID_ARG = 1, /* null or misaligned pointer, inconsistent shape                 */
-    JQ_ERR_UNSUPPORTED = 2, /* a legal shape this build has no kernel for (d != 128, ...)      */
+    JQ_ERR_UNSUPPORTED = 2, /* a legal shape the library has no kernel for (d != 128, ...)     */
     JQ_ERR_WORKSPACE = 3,   /* ws_bytes < jq_workspace_bytes(shape)                            */
     JQ_ERR_CUDA = 4,        /* a CUDA runtime / driver call or a launch failed                 */
     JQ_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (see jq_last_device_status)  */

@@ -49,7 +49,7 @@ def test_outlier_channels_and_planted_rows_are_heavy():
         assert sc[kv, pl].mean() > 2 * wl.R / wl.L
 
 
-def test_formula_bytes_matches_survey_numbers():
+def test_formula_bytes_matches_hand_computed_numbers():
     assert abs(W.formula_bytes(W.CFG2) / 1e6 - 39.9) < 0.1
     assert abs(W.formula_bytes(W.CFG3) / 1e6 - 137.4) < 0.1
     assert abs(W.formula_bytes(W.CFG5) / 1e6 - 543.2) < 0.1
