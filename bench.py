@@ -60,8 +60,9 @@ def pick_workload(args):
 def config_of(wl, layers, distinct, call="per-layer"):
     return {"workload": wl.name, "L": wl.L, "Hkv": wl.Hkv, "Hq": wl.Hq, "d": wl.d, "w": wl.w,
             "budget": wl.budget, "pool": wl.pool, "layers_per_step": layers, "distinct_layers": distinct,
-            "call": ("one jq_evict_layer call per step, the layers stacked along the KV-head axis" if call == "stacked"
-                     else "one jq_evict_layer call per layer"),
+            "call": {"stacked": "one jq_evict_layer call per step, the layers stacked along the KV-head axis",
+                     "per-layer": "one jq_evict_layer call per layer",
+                     "oracle": "the CPU oracle on a bounded sample of one layer"}[call],
             "l2": "inputs larger than L2 (K of one step: %.0f MiB)" % (distinct * wl.Hkv * wl.L * wl.d * 2 / 2**20)}
 
 
@@ -122,7 +123,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": config_of(wl, 1, 1),
+            "config": config_of(wl, 1, 1, "oracle"),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(n), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
