@@ -297,3 +297,55 @@ def test_layers_stacked_along_the_head_axis_equal_separate_calls():
         Ko, Vo, idx = gpu_evict(Ki, Vi, Qi, shape_of(wl))
         sl = slice(i * wl.Hkv, (i + 1) * wl.Hkv)
         assert np.array_equal(idx, gidx[sl]) and np.array_equal(Ko, gKo[sl]) and np.array_equal(Vo, gVo[sl])
+
+
+# ------------------------------------------------------------------ the benchmark's launch configuration
+
+def _stacked_call(K_layers, V_layers, Q_layers, wl):
+    """One jq_evict_layer call on layers stacked along the KV-head axis, tensors built on the device."""
+    n = len(K_layers)
+    dK = torch.cat([dev_bf16(k) for k in K_layers], 0)
+    dV = torch.cat([dev_bf16(v) for v in V_layers], 0)
+    dQ = torch.cat([dev_bf16(q) for q in Q_layers], 0)
+    s = jq.shape(wl.Hkv * n, wl.Hq * n, wl.L, wl.w, wl.budget, wl.pool, wl.d)
+    ws = jq.new_workspace(s)
+    Ko = torch.zeros((s.Hkv, wl.nkeep, s.d), dtype=torch.bfloat16, device="cuda")
+    Vo = torch.zeros_like(Ko)
+    idx = torch.full((s.Hkv, wl.nkeep), -1, dtype=torch.int32, device="cuda")
+    jq.evict_layer(dK, dV, dQ, s, Ko, Vo, idx, ws)
+    assert jq.last_device_status(ws) == jq.JQ_OK
+    return Ko, Vo, idx.cpu().numpy()
+
+
+def test_cfg3_all_32_layers_in_one_stacked_call_sampled_heads():
+    """The benchmark's call for the 32K workload: 32 distinct layers, 256 stacked KV heads, one launch of each
+    kernel.  The oracle recomputes sampled (layer, head) units in full; every unit's structure is checked."""
+    wl = W.CFG3
+    layers = [W.make_layer(wl, layer=i) for i in range(wl.layers)]
+    Ko, Vo, idx = _stacked_call([l[0] for l in layers], [l[1] for l in layers], [l[2] for l in layers], wl)
+    g = wl.group
+    for layer, kv in ((0, 0), (13, 5), (31, 7)):
+        K, V, Q, _ = layers[layer]
+        po = oracle.pool(oracle.score(K[kv:kv + 1], Q[kv * g:(kv + 1) * g]), wl.pool)
+        oidx = oracle.select(po, wl.budget)
+        u = layer * wl.Hkv + kv
+        assert_kept_sets_agree(idx[u:u + 1], oidx, po, wl.nkeep)
+        assert np.array_equal(host_bits(Ko[u]), K[kv][idx[u]]) and np.array_equal(host_bits(Vo[u]), V[kv][idx[u]])
+    assert np.all(np.diff(idx, axis=1) > 0) and idx.min() >= 0 and idx.max() < wl.L
+
+
+def test_cfg5_32_copies_in_one_stacked_call_sampled_heads():
+    """The benchmark's call for the 128K workload: one layer copied 32 times (16 GiB of K and V), 256 stacked
+    KV heads.  Copies must agree with one another bit for bit and a sampled head with the oracle."""
+    wl = W.CFG5
+    K, V, Q, _ = W.make_layer(wl)
+    Ko, Vo, idx = _stacked_call([K] * wl.layers, [V] * wl.layers, [Q] * wl.layers, wl)
+    for c in range(1, wl.layers):
+        assert np.array_equal(idx[:wl.Hkv], idx[c * wl.Hkv:(c + 1) * wl.Hkv])
+    kv, g = 3, wl.group
+    po = oracle.pool(oracle.score(K[kv:kv + 1], Q[kv * g:(kv + 1) * g]), wl.pool)
+    oidx = oracle.select(po, wl.budget)
+    for c in (0, 17, 31):
+        u = c * wl.Hkv + kv
+        assert_kept_sets_agree(idx[u:u + 1], oidx, po, wl.nkeep)
+        assert np.array_equal(host_bits(Ko[u]), K[kv][idx[u]]) and np.array_equal(host_bits(Vo[u]), V[kv][idx[u]])
