@@ -1,6 +1,6 @@
 """Benchmark of the per-layer KV-cache eviction pass (prefix tokens evicted per second per layer).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg3|cfg2] [--budget B]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg4|cfg3|cfg2] [--budget B]
     python bench.py --impl reference ...      # the fp64 CPU oracle, timed on the host cores
 
 One step = one pass of the whole hot path (scores -> pool -> top-k -> gather) over every layer of
@@ -39,7 +39,8 @@ def parse():
     ap.add_argument("--steps", type=int, default=60)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg5", choices=["cfg2", "cfg3", "cfg5"])
+    ap.add_argument("--workload", default="cfg5", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--seq", type=int, default=1, help="cfg4 only: which sequence of the ragged batch (0..3)")
     ap.add_argument("--budget", type=int, default=None)
     ap.add_argument("--layers", type=int, default=None, help="layer calls per step (default: the workload's)")
     ap.add_argument("--call", default="stacked", choices=["stacked", "per-layer"])
@@ -49,7 +50,7 @@ def parse():
 
 
 def pick_workload(args):
-    wl = {"cfg2": W.CFG2, "cfg3": W.CFG3, "cfg5": W.CFG5}[args.workload]
+    wl = {"cfg2": W.CFG2, "cfg3": W.CFG3, "cfg4": W.CFG4[args.seq % 4], "cfg5": W.CFG5}[args.workload]
     if args.workload == "cfg2":
         wl = W.Workload(wl.name, 2, wl.Hkv, wl.Hq, wl.L, wl.w, wl.budget, layers=32, distinct_layers=32)
     if args.budget:
