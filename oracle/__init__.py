@@ -25,6 +25,8 @@ def _load():
         lib.jq_oracle_threads.restype = c_int
         lib.jq_oracle_score_f64.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
         lib.jq_oracle_score.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
+        lib.jq_oracle_score_windowed_f64.argtypes = [vp, vp, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
+        lib.jq_oracle_score_windowed.argtypes = [vp, vp, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
         lib.jq_oracle_pool.argtypes = [vp, c_int, c_int, c_int, vp]
         lib.jq_oracle_select.argtypes = [vp, c_int, c_int, c_int, vp]
         lib.jq_oracle_select_f32.argtypes = [vp, c_int, c_int, c_int, c_int, vp, vp]
@@ -68,6 +70,28 @@ def score(K, Q, return_probs=False):
         rc = lib.jq_oracle_score_f64(_p(K), _p(Q), Hkv, Hq, L, d, w, _p(out), _p(probs))
     if rc:
         raise ValueError("jq_oracle_score: bad arguments")
+    return (out, probs) if return_probs else out
+
+
+def score_windowed(K, Q, Kw, return_probs=False):
+    """Window-inclusive scores: query i also attends, causally, to the window keys Kw[kv, i' <= i]; only the
+    mass on the prefix keys is scored.  K [Hkv,L,d], Q [Hq,w,d], Kw [Hkv,w,d], all uint16 (bf16 bits) or all
+    float64.  Returns score [Hkv,L] float64 (and the prefix part of the softmax rows [Hq,w,L] if asked)."""
+    lib = _load()
+    Hkv, L, d = K.shape
+    Hq, w, _ = Q.shape
+    if Kw.shape != (Hkv, w, d) or Q.shape[2] != d:
+        raise ValueError("shapes of K, Q, Kw do not fit")
+    out = np.empty((Hkv, L), np.float64)
+    probs = np.empty((Hq, w, L), np.float64) if return_probs else None
+    if K.dtype == np.uint16:
+        K, Q, Kw = _chk(K, np.uint16), _chk(Q, np.uint16), _chk(Kw, np.uint16)
+        rc = lib.jq_oracle_score_windowed(_p(K), _p(Q), _p(Kw), Hkv, Hq, L, d, w, _p(out), _p(probs))
+    else:
+        K, Q, Kw = _chk(K, np.float64), _chk(Q, np.float64), _chk(Kw, np.float64)
+        rc = lib.jq_oracle_score_windowed_f64(_p(K), _p(Q), _p(Kw), Hkv, Hq, L, d, w, _p(out), _p(probs))
+    if rc:
+        raise ValueError("jq_oracle_score_windowed: bad arguments")
     return (out, probs) if return_probs else out
 
 

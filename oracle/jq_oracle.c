@@ -28,6 +28,10 @@
  *   compact Inference section (the pruned cache is what decoding continues
  *           with): rows K[kv,idx,:], V[kv,idx,:] copied bit for bit.
  *
+ * (jq_oracle_score_windowed is the window-inclusive variant of the scores; its pins are a library
+ * softmax over the concatenated, causally masked logits, the Q = 0 closed form and the limit of a
+ * window that attracts no mass.)
+ *
  * Parity pins (tests/test_oracle_pins.py): softmax rows sum to 1; per-head
  * score mass equals w*group; g=w=1 equals a library softmax; key-shift
  * invariance; Q=0 and one-hot closed forms; pooling against an independent
@@ -135,6 +139,83 @@ int jq_oracle_score(const uint16_t *K, const uint16_t *Q, int Hkv, int Hq, int L
     int rc = jq_oracle_score_f64(Kd, Qd, Hkv, Hq, L, d, w, score, probs);
     free(Kd);
     free(Qd);
+    return rc;
+}
+
+/*
+ * Window-inclusive variant of the scores (the other reading of Eq. 3, and the way last-window methods of
+ * the experimental section score): query i of a head also attends, causally, to the keys Kw[kv, i'] of
+ * the query positions i' <= i themselves, as it does inside the model.  Those columns only enter the
+ * softmax denominator; the score is still the probability mass on the L prefix keys:
+ *     P_j = exp(s_j - m) / ( sum_{j<L} exp(s_j - m) + sum_{i'<=i} exp(t_i' - m) ),  t_i' = Q[h,i,:].Kw[kv,i',:]/sqrt(d)
+ * with m the max over both kinds of logit.  K [Hkv,L,d], Q [Hq,w,d], Kw [Hkv,w,d], doubles.
+ * probs, when not NULL, receives the prefix part of every softmax row: [Hq,w,L].
+ */
+int jq_oracle_score_windowed_f64(const double *K, const double *Q, const double *Kw, int Hkv, int Hq, int L, int d,
+                                 int w, double *score, double *probs)
+{
+    if (Hkv < 1 || Hq < 1 || L < 1 || d < 1 || w < 1 || Hq % Hkv != 0) return 1;
+    const int g = Hq / Hkv;
+    const double inv_sqrt_d = 1.0 / sqrt((double)d);
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int kv = 0; kv < Hkv; ++kv) {
+        double *e = (double *)malloc((size_t)(L + w) * sizeof(double));
+        if (!e) {
+#pragma omp atomic write
+            failed = 1;
+            continue;
+        }
+        double *sc = score + (size_t)kv * L;
+        for (int j = 0; j < L; ++j) sc[j] = 0.0;
+        for (int h = kv * g; h < kv * g + g; ++h) {
+            for (int i = 0; i < w; ++i) {
+                const double *q = Q + ((size_t)h * w + i) * d;
+                double m = -INFINITY;
+                for (int j = 0; j < L + i + 1; ++j) {      /* the L prefix keys, then window keys 0..i */
+                    const double *k = (j < L) ? K + ((size_t)kv * L + j) * d : Kw + ((size_t)kv * w + (j - L)) * d;
+                    double dot = 0.0;
+                    for (int c = 0; c < d; ++c) dot += q[c] * k[c];
+                    e[j] = dot * inv_sqrt_d;
+                    if (e[j] > m) m = e[j];
+                }
+                double l = 0.0;
+                for (int j = 0; j < L + i + 1; ++j) {
+                    e[j] = exp(e[j] - m);
+                    l += e[j];
+                }
+                double *pr = probs ? probs + ((size_t)h * w + i) * L : NULL;
+                for (int j = 0; j < L; ++j) {
+                    double p = e[j] / l;
+                    sc[j] += p;
+                    if (pr) pr[j] = p;
+                }
+            }
+        }
+        free(e);
+    }
+    return failed;
+}
+
+/* Same, from bf16 bit patterns (converted exactly to double first). */
+int jq_oracle_score_windowed(const uint16_t *K, const uint16_t *Q, const uint16_t *Kw, int Hkv, int Hq, int L, int d,
+                             int w, double *score, double *probs)
+{
+    if (Hkv < 1 || Hq < 1 || L < 1 || d < 1 || w < 1) return 1;
+    size_t nk = (size_t)Hkv * L * d, nq = (size_t)Hq * w * d, nw = (size_t)Hkv * w * d;
+    double *Kd = (double *)malloc(nk * sizeof(double));
+    double *Qd = (double *)malloc(nq * sizeof(double));
+    double *Wd = (double *)malloc(nw * sizeof(double));
+    int rc = 1;
+    if (Kd && Qd && Wd) {
+        for (size_t t = 0; t < nk; ++t) Kd[t] = bf16_to_double(K[t]);
+        for (size_t t = 0; t < nq; ++t) Qd[t] = bf16_to_double(Q[t]);
+        for (size_t t = 0; t < nw; ++t) Wd[t] = bf16_to_double(Kw[t]);
+        rc = jq_oracle_score_windowed_f64(Kd, Qd, Wd, Hkv, Hq, L, d, w, score, probs);
+    }
+    free(Kd);
+    free(Qd);
+    free(Wd);
     return rc;
 }
 

@@ -283,3 +283,58 @@ def test_config1_planted_and_duplicates():
         kept = set(idx[kv].tolist())
         hit = sum(int(j) in kept for j in info["planted"][kv])
         assert hit >= 20, hit                     # 24 planted heavy keys, budget 256
+
+
+# ---------------------------------------------------------------- window-inclusive scores
+
+def _rand_kqw(Hkv, g, w, L, d=16, seed=0):
+    rng = np.random.default_rng(seed)
+    return (rng.standard_normal((Hkv, L, d)), rng.standard_normal((Hkv * g, w, d)), rng.standard_normal((Hkv, w, d)))
+
+
+def test_windowed_equals_library_softmax_over_masked_concatenation():
+    """Each row against torch.softmax over [prefix logits, window logits] with the causal mask, prefix part kept."""
+    import torch
+    Hkv, g, w, L, d = 2, 3, 5, 37, 16
+    K, Q, Kw = _rand_kqw(Hkv, g, w, L, d, seed=3)
+    score, probs = oracle.score_windowed(K, Q, Kw, return_probs=True)
+    want = np.zeros((Hkv, L))
+    for h in range(Hkv * g):
+        kv = h // g
+        keys = torch.from_numpy(np.concatenate([K[kv], Kw[kv]], 0))                     # [L+w, d]
+        logits = torch.from_numpy(Q[h]) @ keys.T / np.sqrt(d)                            # [w, L+w]
+        mask = torch.zeros((w, L + w), dtype=torch.bool)
+        for i in range(w):
+            mask[i, L + i + 1:] = True                                                   # window keys after the query
+        p = torch.softmax(logits.masked_fill(mask, float("-inf")), dim=-1).numpy()
+        np.testing.assert_allclose(probs[h], p[:, :L], rtol=1e-12, atol=1e-15)
+        want[kv] += p[:, :L].sum(0)
+    np.testing.assert_allclose(score, want, rtol=1e-12)
+    assert np.all(score.sum(-1) < g * w)          # some mass went to the window
+
+
+def test_windowed_zero_queries_closed_form_pins_the_mask_direction():
+    Hkv, g, w, L, d = 1, 2, 6, 50, 8
+    K, Q, Kw = _rand_kqw(Hkv, g, w, L, d, seed=4)
+    _, probs = oracle.score_windowed(K, np.zeros_like(Q), Kw, return_probs=True)
+    for i in range(w):      # query i sees L prefix keys and i + 1 window keys, all with logit 0
+        np.testing.assert_allclose(probs[:, i, :], 1.0 / (L + i + 1), rtol=1e-13)
+
+
+def test_window_that_attracts_no_mass_gives_the_plain_scores():
+    Hkv, g, w, L, d = 2, 2, 4, 64, 16
+    K, Q, _ = _rand_kqw(Hkv, g, w, L, d, seed=5)
+    u = np.ones(d) / np.sqrt(d)
+    Q = Q * 0.1 + 3.0 * u                      # every query has a large component along u ...
+    Kw = np.tile(-200.0 * u, (Hkv, w, 1))      # ... and every window key points the other way: logits near -150
+    np.testing.assert_allclose(oracle.score_windowed(K, Q, Kw), oracle.score(K, Q), rtol=1e-12)
+
+
+def test_windowed_bf16_entry_matches_double_entry():
+    Hkv, g, w, L = 2, 2, 3, 40
+    rng = np.random.default_rng(6)
+    K = W.bf16_bits(rng.standard_normal((Hkv, L, 128), dtype=np.float32))
+    Q = W.bf16_bits(rng.standard_normal((Hkv * g, w, 128), dtype=np.float32))
+    Kw = W.bf16_bits(rng.standard_normal((Hkv, w, 128), dtype=np.float32))
+    f = lambda b: W.bf16_to_f32(b).astype(np.float64)
+    np.testing.assert_allclose(oracle.score_windowed(K, Q, Kw), oracle.score_windowed(f(K), f(Q), f(Kw)), rtol=1e-14)
