@@ -92,6 +92,21 @@ jq_status jq_score(const void *K, const void *Qwin, const jq_shape *shape, float
                    void *ws, size_t ws_bytes, jq_stream_t stream);
 
 /*
+ * Window-inclusive variants.  Eq. 3 can also be read as the attention the model itself computes for a soft
+ * token: its softmax then runs over the prefix AND, causally, over the soft tokens up to itself; the same
+ * holds for the last-window queries that the compared methods of the experimental section score with.
+ * Kwin [Hkv, w, d] bf16 holds the keys of the w query positions; query i of every head of the group sees
+ * Kwin[kv, 0..i] besides the L prefix keys.  These columns only enter the denominator: scores, pooling,
+ * selection and compaction still run over the L prefix positions (a caller that wants the window kept
+ * keeps it itself).  Everything else as in jq_score / jq_evict_layer.
+ */
+jq_status jq_score_windowed(const void *K, const void *Qwin, const void *Kwin, const jq_shape *shape,
+                            float *scores, void *ws, size_t ws_bytes, jq_stream_t stream);
+jq_status jq_evict_layer_windowed(const void *K, const void *V, const void *Qwin, const void *Kwin,
+                                  const jq_shape *shape, void *Kout, void *Vout, int32_t *kept_idx,
+                                  void *ws, size_t ws_bytes, jq_stream_t stream);
+
+/*
  * jq_score for callers that cannot allocate device memory: an inference server that has handed every
  * free byte of the GPU to its KV-cache pool, a plug-in running inside somebody else's memory budget, a
  * call site that must not touch the allocator.  (The paper has no counterpart; this is a property of

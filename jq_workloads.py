@@ -200,6 +200,15 @@ def make_layer(wl, layer=0, seq=0, with_v=True):
     return K, V, Q, info
 
 
+def make_window_keys(wl, Q, layer=0, seq=0):
+    """Keys of the w query positions themselves, [Hkv, w, d] bf16 bits, for the window-inclusive mode:
+    N(0,1) plus 0.3 x the mean query of the position over the GQA group (a token's key resembles its
+    query a little, so that the window takes a visible but not dominant share of the attention)."""
+    rng = _rng(seed_of(wl, layer, seq), 3)
+    Qf = bf16_to_f32(Q).reshape(wl.Hkv, wl.group, wl.w, wl.d)
+    return bf16_bits(_normal(rng, (wl.Hkv, wl.w, wl.d)) + 0.3 * Qf.mean(axis=1))
+
+
 def formula_bytes(wl):
     """Algorithmic HBM bytes of one layer call: two reads of K, one read of the kept V rows, the
     writes of the compacted K and V and of the int32 indices."""

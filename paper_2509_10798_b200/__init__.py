@@ -17,7 +17,7 @@ EXPORTS = (
     "jq_workspace_bytes", "jq_workspace_init", "jq_num_kept", "jq_check_shape", "jq_score",
     "jq_score_fma", "jq_select_topk", "jq_compact_kv", "jq_evict_layer", "jq_host_call_bytes",
     "jq_evict_layer_host", "jq_last_device_status", "jq_launch_count", "jq_status_string",
-    "jq_score_static",
+    "jq_score_static", "jq_score_windowed", "jq_evict_layer_windowed",
 )
 
 
@@ -56,6 +56,8 @@ def lib():
         L.jq_score.argtypes = [vp, vp, sp, vp, vp, sz, vp]
         L.jq_score_fma.argtypes = [vp, vp, sp, vp, vp, sz, vp]
         L.jq_score_static.argtypes = [vp, vp, sp, vp, vp]
+        L.jq_score_windowed.argtypes = [vp, vp, vp, sp, vp, vp, sz, vp]
+        L.jq_evict_layer_windowed.argtypes = [vp, vp, vp, vp, sp, vp, vp, vp, vp, sz, vp]
         L.jq_select_topk.argtypes = [vp, sp, vp, vp, vp, sz, vp]
         L.jq_compact_kv.argtypes = [vp, vp, vp, sp, vp, vp, vp]
         L.jq_evict_layer.argtypes = [vp, vp, vp, sp, vp, vp, vp, vp, sz, vp]
@@ -145,6 +147,18 @@ def score_static(K, Qwin, s, scores, stream=None):
     them on one stream)."""
     _raise("jq_score_static",
            lib().jq_score_static(_ptr(K), _ptr(Qwin), ctypes.byref(s), _ptr(scores), _stream(stream)))
+
+
+def score_windowed(K, Qwin, Kwin, s, scores, ws, stream=None):
+    """jq_score with the causal window keys Kwin [Hkv, w, d] in the softmax denominator."""
+    _raise("jq_score_windowed", lib().jq_score_windowed(_ptr(K), _ptr(Qwin), _ptr(Kwin), ctypes.byref(s), _ptr(scores),
+                                                        _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def evict_layer_windowed(K, V, Qwin, Kwin, s, Kout, Vout, kept_idx, ws, stream=None):
+    _raise("jq_evict_layer_windowed",
+           lib().jq_evict_layer_windowed(_ptr(K), _ptr(V), _ptr(Qwin), _ptr(Kwin), ctypes.byref(s), _ptr(Kout), _ptr(Vout),
+                                         _ptr(kept_idx), _ptr(ws), ws.numel(), _stream(stream)))
 
 
 def select_topk(scores, s, kept_idx, ws, pooled=None, stream=None):

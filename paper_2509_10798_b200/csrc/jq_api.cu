@@ -72,6 +72,33 @@ jq_status jq_score(const void *K, const void *Qwin, const jq_shape *s, float *sc
     return launch_score_tc(K, Qwin, *s, scores, w, (cudaStream_t)stream);
 }
 
+jq_status jq_score_windowed(const void *K, const void *Qwin, const void *Kwin, const jq_shape *s, float *scores,
+                            void *ws, size_t ws_bytes, jq_stream_t stream)
+{
+    jq_status rc = check_shape(s);
+    if (rc != JQ_OK) return rc;
+    if (!aligned16(K) || !aligned16(Qwin) || !aligned16(Kwin) || !aligned16(scores)) return JQ_ERR_INVALID_ARG;
+    Workspace w;
+    if ((rc = check_ws(s, ws, ws_bytes, &w)) != JQ_OK) return rc;
+    return launch_score_tc(K, Qwin, *s, scores, w, (cudaStream_t)stream, Kwin);
+}
+
+jq_status jq_evict_layer_windowed(const void *K, const void *V, const void *Qwin, const void *Kwin, const jq_shape *s,
+                                  void *Kout, void *Vout, int32_t *kept_idx, void *ws, size_t ws_bytes,
+                                  jq_stream_t stream)
+{
+    jq_status rc = check_shape(s);
+    if (rc != JQ_OK) return rc;
+    if (!aligned16(K) || !aligned16(V) || !aligned16(Qwin) || !aligned16(Kwin) || !aligned16(Kout) || !aligned16(Vout) ||
+        !aligned16(kept_idx))
+        return JQ_ERR_INVALID_ARG;
+    Workspace w;
+    if ((rc = check_ws(s, ws, ws_bytes, &w)) != JQ_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if ((rc = launch_score_tc(K, Qwin, *s, w.scores, w, st, Kwin)) != JQ_OK) return rc;
+    return launch_select(w.scores, *s, kept_idx, nullptr, w, st, K, V, Kout, Vout);
+}
+
 jq_status jq_score_fma(const void *K, const void *Qwin, const jq_shape *s, float *scores, void *ws,
                        size_t ws_bytes, jq_stream_t stream)
 {

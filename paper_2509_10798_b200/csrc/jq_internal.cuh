@@ -56,8 +56,9 @@ jq_status check_launch();   // cudaGetLastError -> JQ_OK / JQ_ERR_CUDA
 // Stage launchers (arguments already validated).
 jq_status launch_score_fma(const void *K, const void *Q, const jq_shape &s, float *scores,
                            const Workspace &w, cudaStream_t st);
+// Kwin, when not null: keys [Hkv][w][128] of the query positions themselves (window-inclusive softmax).
 jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float *scores,
-                          const Workspace &w, cudaStream_t st);
+                          const Workspace &w, cudaStream_t st, const void *Kwin = nullptr);
 // With K, V, Kout, Vout given, the kernel also copies the kept rows (the fused layer path).
 jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, float *pooled,
                         const Workspace &w, cudaStream_t st, const void *K = nullptr, const void *V = nullptr,

@@ -122,6 +122,9 @@ struct Params {
     float *Mrow;             // [Hkv][R]   c*m + log2(l) per query row
     float *scores;           // [Hkv][L]
     int *status;             // status block (kStatusWords ints)
+    const uint16_t *Q;       // query rows [Hkv][R][128] as raw bf16 (window-inclusive mode only)
+    const uint16_t *Kwin;    // [Hkv][w][128] keys of the query positions themselves, or null
+    int w;                   // soft-token queries per query head
 #ifdef JQ_TRACE
     long long *trace;
 #endif
@@ -397,6 +400,33 @@ __device__ __forceinline__ void walk(int pass, int tph, int &kv, int &t)
 {
     if (pass == 1) { if (++t == tph) { t = 0; ++kv; } }
     else { if (--t < 0) { t = tph - 1; --kv; } }
+}
+
+// Window-inclusive mode: log2-domain logits c * (q . kw_i') of one query row against the window keys
+// i' = first, first + step, ... <= last, folded into a running (max, sum of 2^(b - max)).
+__device__ __forceinline__ void window_terms(const uint16_t *qrow, const uint16_t *kw, int first, int step, int last,
+                                             float c, float &bm, float &bl)
+{
+    bm = -INFINITY; bl = 0.f;
+    const uint4 *q4 = (const uint4 *)qrow;
+    for (int i = first; i <= last; i += step) {
+        const uint4 *k4 = (const uint4 *)(kw + (size_t)i * kD);
+        float dot = 0.f;
+#pragma unroll 4
+        for (int v = 0; v < kD / 8; ++v) {
+            const uint4 a = __ldg(q4 + v), b = __ldg(k4 + v);
+            const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                dot = fmaf(__uint_as_float(aw[t] << 16), __uint_as_float(bw[t] << 16), dot);
+                dot = fmaf(__uint_as_float(aw[t] & 0xffff0000u), __uint_as_float(bw[t] & 0xffff0000u), dot);
+            }
+        }
+        const float b = c * dot;
+        const float mn = fmaxf(bm, b);
+        bl = bl * ex2(bm - mn) + ex2(b - mn);      // bm = -inf the first time: ex2(-inf) = 0
+        bm = mn;
+    }
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -753,7 +783,20 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                 for (int o = lpr >> 1; o >= 1; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, o));
                 l = (l > 0.f) ? l * ex2(c * (m - mw)) : 0.f;
                 for (int o = lpr >> 1; o >= 1; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-                if (have && sub == 0) P.Mrow[(size_t)kv * P.R + r] = c * mw + log2f(l);
+                float M = c * mw + log2f(l);                       // log2 of the row's sum of exponentials over the prefix
+                if (P.Kwin) {
+                    // window-inclusive softmax: the causal window keys of the row's own query position join the denominator
+                    float bm, bl;
+                    window_terms(P.Q + ((size_t)kv * P.R + r) * kD, P.Kwin + (size_t)kv * P.w * kD, sub, lpr,
+                                 have ? r % P.w : -1, c, bm, bl);
+                    float wm = bm;
+                    for (int o = lpr >> 1; o >= 1; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
+                    bl = (bl > 0.f) ? bl * ex2(bm - wm) : 0.f;
+                    for (int o = lpr >> 1; o >= 1; o >>= 1) bl += __shfl_xor_sync(0xffffffffu, bl, o);
+                    const float mx = fmaxf(M, wm);
+                    M = mx + log2f(ex2(M - mx) + bl * ex2(wm - mx));
+                }
+                if (have && sub == 0) P.Mrow[(size_t)kv * P.R + r] = M;
             }
             __syncwarp();
             if (lane == 0) {
@@ -909,7 +952,7 @@ extern "C" void jq_debug_set_trace(long long *p) { g_trace = p; }   // [grid][32
 #endif
 
 jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float *scores, const Workspace &w,
-                          cudaStream_t st)
+                          cudaStream_t st, const void *Kwin)
 {
     DeviceInfo dev;
     if (!device_info(&dev)) return JQ_ERR_CUDA;
@@ -924,6 +967,7 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
     P.depth = order < 1 ? 1 : (order > 3 ? 3 : (int)order);
     P.c = 1.4426950408889634f / sqrtf((float)s.d);
     P.part = w.part; P.Mrow = w.Mrow; P.scores = scores; P.status = w.status;
+    P.Q = (const uint16_t *)Q; P.Kwin = (const uint16_t *)Kwin; P.w = s.w;
 #ifdef JQ_TRACE
     P.trace = g_trace;
 #endif

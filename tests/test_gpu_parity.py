@@ -349,3 +349,56 @@ def test_cfg5_32_copies_in_one_stacked_call_sampled_heads():
         u = c * wl.Hkv + kv
         assert_kept_sets_agree(idx[u:u + 1], oidx, po, wl.nkeep)
         assert np.array_equal(host_bits(Ko[u]), K[kv][idx[u]]) and np.array_equal(host_bits(Vo[u]), V[kv][idx[u]])
+
+
+# ------------------------------------------------------------------ window-inclusive mode
+
+def gpu_score_windowed(K, Q, Kw, s):
+    ws = jq.new_workspace(s)
+    out = torch.full((s.Hkv, s.L), -1.0, dtype=torch.float32, device="cuda")
+    jq.score_windowed(dev_bf16(K), dev_bf16(Q), dev_bf16(Kw), s, out, ws)
+    assert jq.last_device_status(ws) == jq.JQ_OK
+    return out.cpu().numpy()
+
+
+@pytest.mark.parametrize("Hkv,g,w,L", [(1, 1, 1, 5), (2, 4, 16, 129), (3, 4, 32, 1000), (2, 4, 64, 2049), (1, 3, 11, 4000),
+                                       (8, 4, 32, 8192)])
+def test_score_windowed_matches_oracle(Hkv, g, w, L):
+    wl = small_wl(Hkv, g, w, L, 1)
+    K, _, Q, _ = W.make_layer(wl, with_v=False)
+    Kw = W.make_window_keys(wl, Q)
+    want = oracle.score_windowed(K, Q, Kw)
+    got = gpu_score_windowed(K, Q, Kw, shape_of(wl))
+    assert_scores_close(got, want)
+    plain = oracle.score(K, Q)
+    assert np.all(want.sum(-1) < plain.sum(-1))           # the window did take mass (the case is not vacuous)
+
+
+def test_score_windowed_with_dominant_window_keys():
+    """Window keys far more attractive than any prefix key: nearly all mass leaves the prefix; still exact."""
+    wl = small_wl(2, 2, 8, 700, 1)
+    K, _, Q, _ = W.make_layer(wl, with_v=False)
+    Kw = W.bf16_bits(3.0 * W.bf16_to_f32(Q).reshape(2, 2, 8, 128).mean(axis=1))
+    want = oracle.score_windowed(K, Q, Kw)
+    got = gpu_score_windowed(K, Q, Kw, shape_of(wl))
+    assert_scores_close(got, want)
+    assert want.sum() < 0.5 * wl.R * wl.Hkv
+
+
+def test_evict_layer_windowed_end_to_end():
+    wl = W.CFG2.with_L(5000)
+    K, V, Q, _ = W.make_layer(wl)
+    Kw = W.make_window_keys(wl, Q)
+    s = shape_of(wl)
+    ws = jq.new_workspace(s)
+    Ko = torch.zeros((s.Hkv, wl.nkeep, s.d), dtype=torch.bfloat16, device="cuda")
+    Vo = torch.zeros_like(Ko)
+    idx = torch.full((s.Hkv, wl.nkeep), -1, dtype=torch.int32, device="cuda")
+    jq.evict_layer_windowed(dev_bf16(K), dev_bf16(V), dev_bf16(Q), dev_bf16(Kw), s, Ko, Vo, idx, ws)
+    assert jq.last_device_status(ws) == jq.JQ_OK
+    gidx = idx.cpu().numpy()
+    pooled = oracle.pool(oracle.score_windowed(K, Q, Kw), wl.pool)
+    assert_kept_sets_agree(gidx, oracle.select(pooled, wl.budget), pooled, wl.nkeep)
+    gK, gV = host_bits(Ko), host_bits(Vo)
+    for kv in range(wl.Hkv):
+        assert np.array_equal(gK[kv], K[kv][gidx[kv]]) and np.array_equal(gV[kv], V[kv][gidx[kv]])
