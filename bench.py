@@ -44,6 +44,8 @@ def parse():
     ap.add_argument("--budget", type=int, default=None)
     ap.add_argument("--layers", type=int, default=None, help="layer calls per step (default: the workload's)")
     ap.add_argument("--call", default="stacked", choices=["stacked", "per-layer"])
+    ap.add_argument("--windowed", action="store_true",
+                    help="window-inclusive scoring (jq_evict_layer_windowed): the causal keys of the query positions join the softmax")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -219,12 +221,14 @@ def run_ours(args):
         return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
 
     host0 = None
-    Ks, Vs, Qs = [], [], []
+    Ks, Vs, Qs, Kws = [], [], [], []
     for i in range(distinct):
         K, V, Q, _ = W.make_layer(wl, layer=i, seq=rank)
         if i == 0:
             host0 = (K, V, Q)
         Ks.append(dev(K)); Vs.append(dev(V)); Qs.append(dev(Q))
+        if args.windowed:
+            Kws.append(dev(W.make_window_keys(wl, Q, layer=i, seq=rank)))
     ws = jq.new_workspace(s)
     Ko = torch.zeros((wl.Hkv, nkeep, wl.d), dtype=torch.bfloat16, device="cuda")
     Vo = torch.zeros_like(Ko)
@@ -234,7 +238,10 @@ def run_ours(args):
     def step_per_layer():
         for i in range(layers):
             j = i % distinct
-            jq.evict_layer(Ks[j], Vs[j], Qs[j], s, Ko, Vo, idx, ws, stream=stream)
+            if args.windowed:
+                jq.evict_layer_windowed(Ks[j], Vs[j], Qs[j], Kws[j], s, Ko, Vo, idx, ws, stream=stream)
+            else:
+                jq.evict_layer(Ks[j], Vs[j], Qs[j], s, Ko, Vo, idx, ws, stream=stream)
 
     # the layers of the cache stacked along the KV-head axis (a layer repeated in the workload is copied, so
     # that every layer of the step has memory of its own)
@@ -244,13 +251,17 @@ def run_ours(args):
         KS = torch.cat([Ks[j] for j in order], 0)
         VS = torch.cat([Vs[j] for j in order], 0)
         QS = torch.cat([Qs[j] for j in order], 0)
+        KwS = torch.cat([Kws[j] for j in order], 0) if args.windowed else None
         wsS = jq.new_workspace(sS)
         KoS = torch.zeros((sS.Hkv, nkeep, wl.d), dtype=torch.bfloat16, device="cuda")
         VoS = torch.zeros_like(KoS)
         idxS = torch.zeros((sS.Hkv, nkeep), dtype=torch.int32, device="cuda")
 
     def step_stacked():
-        jq.evict_layer(KS, VS, QS, sS, KoS, VoS, idxS, wsS, stream=stream)
+        if args.windowed:
+            jq.evict_layer_windowed(KS, VS, QS, KwS, sS, KoS, VoS, idxS, wsS, stream=stream)
+        else:
+            jq.evict_layer(KS, VS, QS, sS, KoS, VoS, idxS, wsS, stream=stream)
 
     step = step_stacked if args.call == "stacked" else step_per_layer
 
@@ -313,11 +324,17 @@ def run_ours(args):
     if args.call == "stacked":
         scoresS = torch.empty((sS.Hkv, wl.L), dtype=torch.float32, device="cuda")
         nb = 4
-        stage_ms[0] = timed(lambda j: jq.score(KS, QS, sS, scoresS, wsS, stream=stream)) / layers
+        if args.windowed:
+            stage_ms[0] = timed(lambda j: jq.score_windowed(KS, QS, KwS, sS, scoresS, wsS, stream=stream)) / layers
+        else:
+            stage_ms[0] = timed(lambda j: jq.score(KS, QS, sS, scoresS, wsS, stream=stream)) / layers
         stage_ms[1] = timed(lambda j: jq.select_topk(scoresS, sS, idxS, wsS, stream=stream)) / layers
         stage_ms[2] = timed(lambda j: jq.compact_kv(KS, VS, idxS, sS, KoS, VoS, stream=stream)) / layers
     else:
-        stage_ms[0] = timed(lambda j: jq.score(Ks[j], Qs[j], s, scores[j % len(scores)], ws, stream=stream))
+        if args.windowed:
+            stage_ms[0] = timed(lambda j: jq.score_windowed(Ks[j], Qs[j], Kws[j], s, scores[j % len(scores)], ws, stream=stream))
+        else:
+            stage_ms[0] = timed(lambda j: jq.score(Ks[j], Qs[j], s, scores[j % len(scores)], ws, stream=stream))
         stage_ms[1] = timed(lambda j: jq.select_topk(scores[j % len(scores)], s, idx, ws, stream=stream))
         stage_ms[2] = timed(lambda j: jq.compact_kv(Ks[j], Vs[j], idx, s, Ko, Vo, stream=stream))
     clocks = sampler.stop() if sampler else None
@@ -387,7 +404,9 @@ def run_ours(args):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": config_of(wl, layers, distinct, args.call), "ms_per_layer": t_layer * 1e3,
+            "config": dict(config_of(wl, layers, distinct, args.call),
+                           softmax=("prefix keys and the causal window keys" if args.windowed else "prefix keys only")),
+            "ms_per_layer": t_layer * 1e3,
             "per_layer_calls": per_layer_calls,
             "tokens_discarded_per_s": world * (wl.L - nkeep) / t_layer,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline}

@@ -98,7 +98,8 @@ jq_status jq_score(const void *K, const void *Qwin, const jq_shape *shape, float
  * Kwin [Hkv, w, d] bf16 holds the keys of the w query positions; query i of every head of the group sees
  * Kwin[kv, 0..i] besides the L prefix keys.  These columns only enter the denominator: scores, pooling,
  * selection and compaction still run over the L prefix positions (a caller that wants the window kept
- * keeps it itself).  Everything else as in jq_score / jq_evict_layer.
+ * keeps it itself).  Needs w <= 128 (JQ_ERR_UNSUPPORTED otherwise).  Everything else as in jq_score /
+ * jq_evict_layer.  The window keys are scored as one more tile of each head in pass 1, masked causally.
  */
 jq_status jq_score_windowed(const void *K, const void *Qwin, const void *Kwin, const jq_shape *shape,
                             float *scores, void *ws, size_t ws_bytes, jq_stream_t stream);

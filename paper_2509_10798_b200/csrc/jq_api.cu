@@ -77,6 +77,7 @@ jq_status jq_score_windowed(const void *K, const void *Qwin, const void *Kwin, c
 {
     jq_status rc = check_shape(s);
     if (rc != JQ_OK) return rc;
+    if (s->w > 128) return JQ_ERR_UNSUPPORTED;   // the window keys of a head must fit one tile
     if (!aligned16(K) || !aligned16(Qwin) || !aligned16(Kwin) || !aligned16(scores)) return JQ_ERR_INVALID_ARG;
     Workspace w;
     if ((rc = check_ws(s, ws, ws_bytes, &w)) != JQ_OK) return rc;
@@ -89,6 +90,7 @@ jq_status jq_evict_layer_windowed(const void *K, const void *V, const void *Qwin
 {
     jq_status rc = check_shape(s);
     if (rc != JQ_OK) return rc;
+    if (s->w > 128) return JQ_ERR_UNSUPPORTED;   // the window keys of a head must fit one tile
     if (!aligned16(K) || !aligned16(V) || !aligned16(Qwin) || !aligned16(Kwin) || !aligned16(Kout) || !aligned16(Vout) ||
         !aligned16(kept_idx))
         return JQ_ERR_INVALID_ARG;

@@ -113,7 +113,7 @@ static_assert(sizeof(Ctl) <= kCtlBytes, "control block too large");
 
 struct Params {
     int L, R, Rbox, Rpad;    // Rbox = 128 or 256: query rows staged per KV head (rows >= R are zero)
-    int Hkv, tph;            // KV heads; tiles per head
+    int Hkv, tph;            // KV heads; tiles per head (the window tile included)
     int hpg, ngroups;        // heads per group, groups
     int stages;              // K ring depth
     int depth;               // pass 2 of a group starts after pass 1 of `depth` groups: 1 = P1(0) P2(0) P1(1) ..., 2 = P1(0) P1(1) P2(0) P1(2) ..., 3 = P1(0) P1(1) P1(2) P2(0) ...
@@ -122,8 +122,7 @@ struct Params {
     float *Mrow;             // [Hkv][R]   c*m + log2(l) per query row
     float *scores;           // [Hkv][L]
     int *status;             // status block (kStatusWords ints)
-    const uint16_t *Q;       // query rows [Hkv][R][128] as raw bf16 (window-inclusive mode only)
-    const uint16_t *Kwin;    // [Hkv][w][128] keys of the query positions themselves, or null
+    int wtile;               // 1 in window-inclusive mode: every head has one more tile, the last, holding the w window keys
     int w;                   // soft-token queries per query head
 #ifdef JQ_TRACE
     long long *trace;
@@ -402,37 +401,11 @@ __device__ __forceinline__ void walk(int pass, int tph, int &kv, int &t)
     else { if (--t < 0) { t = tph - 1; --kv; } }
 }
 
-// Window-inclusive mode: log2-domain logits c * (q . kw_i') of one query row against the window keys
-// i' = first, first + step, ... <= last, folded into a running (max, sum of 2^(b - max)).
-__device__ __forceinline__ void window_terms(const uint16_t *qrow, const uint16_t *kw, int first, int step, int last,
-                                             float c, float &bm, float &bl)
-{
-    bm = -INFINITY; bl = 0.f;
-    const uint4 *q4 = (const uint4 *)qrow;
-    for (int i = first; i <= last; i += step) {
-        const uint4 *k4 = (const uint4 *)(kw + (size_t)i * kD);
-        float dot = 0.f;
-#pragma unroll 4
-        for (int v = 0; v < kD / 8; ++v) {
-            const uint4 a = __ldg(q4 + v), b = __ldg(k4 + v);
-            const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                dot = fmaf(__uint_as_float(aw[t] << 16), __uint_as_float(bw[t] << 16), dot);
-                dot = fmaf(__uint_as_float(aw[t] & 0xffff0000u), __uint_as_float(bw[t] & 0xffff0000u), dot);
-            }
-        }
-        const float b = c * dot;
-        const float mn = fmaxf(bm, b);
-        bl = bl * ex2(bm - mn) + ex2(b - mn);      // bm = -inf the first time: ex2(-inf) = 0
-        bm = mn;
-    }
-}
-
 // ------------------------------------------------------------------ the kernel
 
 __global__ void __launch_bounds__(kThreads, 1)
-score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ, const Params P)
+score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ,
+            const __grid_constant__ CUtensorMap mapW, const Params P)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     if (smem_u32(smem_raw) & 1023u) {   // the swizzled tiles need 1024-byte alignment; nothing has been started yet
@@ -499,8 +472,13 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     if (!mbar_wait(&ctl->empty[st], ph ^ 1, ctl, status, kSleepLong)) { ok = false; break; }
                     TR_ADD(1);
                     mbar_expect_tx(&ctl->full[st], kStageBytes);
-                    tma_load_3d(kbuf + (size_t)st * kStageBytes, &mapK, &ctl->full[st], 0, tt * kTile, kv);
-                    tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, &mapK, &ctl->full[st], 64, tt * kTile, kv);
+                    // window-inclusive mode: in pass 1 the last tile of a head is its window keys (rows past w read as
+                    // zero); in pass 2 that tile lies past the prefix, reads as zero and its scores are never stored
+                    const bool wt = P.wtile && pass == 1 && tt == tph - 1;
+                    const CUtensorMap *map = wt ? &mapW : &mapK;
+                    const int j0 = wt ? 0 : tt * kTile;
+                    tma_load_3d(kbuf + (size_t)st * kStageBytes, map, &ctl->full[st], 0, j0, kv);
+                    tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, map, &ctl->full[st], 64, j0, kv);
                     if (++st == (uint32_t)stages) { st = 0; ph ^= 1; }
                 }
             }
@@ -567,6 +545,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         const float2 cc = make_float2(c, c);
         float *const scores_out = P.scores;
         float2 *const part_out = P.part + (size_t)(kGroups * blockIdx.x + grp) * R;
+        const int win_i0 = row0 % P.w, win_i1 = (row0 + 128) % P.w;   // soft-token index of this thread's row in block 0 / block 1
         uint32_t u = 0;                                         // accumulator blocks of the CTA before this segment
         int hs = 0;                                             // pass-2 heads of the CTA before this segment
         bool ok = true;
@@ -607,7 +586,9 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     TR_ADD(0);
                     tc_fence_after();
                     const uint32_t taddr = lane_addr + slot * kSlotCols;
-                    const int valid = min(kTile, L - tt * kTile);
+                    // keys of this block that count for this thread's row: the prefix keys of the tile, or, in the window
+                    // tile, the window keys up to the row's own position (causal)
+                    const int valid = (P.wtile && tt == tph - 1) ? min(P.w, (blk ? win_i1 : win_i0) + 1) : min(kTile, L - tt * kTile);
                     // one copy of the block code: the second row block borrows the first one's registers
                     if (blk == 1) { const RowState t = st0; st0 = st1; st1 = t; }
 #pragma unroll 1
@@ -783,19 +764,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                 for (int o = lpr >> 1; o >= 1; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, o));
                 l = (l > 0.f) ? l * ex2(c * (m - mw)) : 0.f;
                 for (int o = lpr >> 1; o >= 1; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-                float M = c * mw + log2f(l);                       // log2 of the row's sum of exponentials over the prefix
-                if (P.Kwin) {
-                    // window-inclusive softmax: the causal window keys of the row's own query position join the denominator
-                    float bm, bl;
-                    window_terms(P.Q + ((size_t)kv * P.R + r) * kD, P.Kwin + (size_t)kv * P.w * kD, sub, lpr,
-                                 have ? r % P.w : -1, c, bm, bl);
-                    float wm = bm;
-                    for (int o = lpr >> 1; o >= 1; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
-                    bl = (bl > 0.f) ? bl * ex2(bm - wm) : 0.f;
-                    for (int o = lpr >> 1; o >= 1; o >>= 1) bl += __shfl_xor_sync(0xffffffffu, bl, o);
-                    const float mx = fmaxf(M, wm);
-                    M = mx + log2f(ex2(M - mx) + bl * ex2(wm - mx));
-                }
+                const float M = c * mw + log2f(l);
                 if (have && sub == 0) P.Mrow[(size_t)kv * P.R + r] = M;
             }
             __syncwarp();
@@ -962,17 +931,19 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
     Params P;
     P.L = s.L; P.R = R; P.Rbox = R <= 128 ? 128 : 256; P.Rpad = (R + 15) & ~15;
     P.Hkv = s.Hkv;
-    P.tph = (s.L + kTile - 1) / kTile;
+    P.wtile = Kwin ? 1 : 0;
+    P.tph = (s.L + kTile - 1) / kTile + P.wtile;
     P.stages = P.Rbox == 128 ? 5 : 3;
     P.depth = order < 1 ? 1 : (order > 3 ? 3 : (int)order);
     P.c = 1.4426950408889634f / sqrtf((float)s.d);
     P.part = w.part; P.Mrow = w.Mrow; P.scores = scores; P.status = w.status;
-    P.Q = (const uint16_t *)Q; P.Kwin = (const uint16_t *)Kwin; P.w = s.w;
+    P.w = s.w;
 #ifdef JQ_TRACE
     P.trace = g_trace;
 #endif
-    CUtensorMap mapK, mapQ;
+    CUtensorMap mapK, mapQ, mapW;
     if (!make_map(&mapK, K, s.L, s.Hkv, kTile) || !make_map(&mapQ, Q, R, s.Hkv, P.Rbox)) return JQ_ERR_CUDA;
+    if (Kwin) { if (!make_map(&mapW, Kwin, s.w, s.Hkv, kTile)) return JQ_ERR_CUDA; } else mapW = mapK;
 
     int sms = dev.sms;
     if (kGroups * sms > kSlots) sms = kSlots / kGroups;
@@ -1013,7 +984,7 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (cudaLaunchKernelEx(&cfg, score_fused, mapK, mapQ, P) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, score_fused, mapK, mapQ, mapW, P) != cudaSuccess) {
         cudaGetLastError();
         return JQ_ERR_CUDA;
     }
