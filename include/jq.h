@@ -175,6 +175,15 @@ jq_status jq_evict_layer_host(const void *hK, const void *hV, const void *hQwin,
                               void *dev_buf, size_t dev_buf_bytes, jq_stream_t stream);
 
 /*
+ * Eq. 6, the critical key-value hit rate: rate[kv] = |cur[kv] ^ ref[kv]| / nref, the share of a reference
+ * kept set (in the paper: the one chosen with the queries of the actually decoded tokens) that another kept
+ * set of the same head also holds.  cur [Hkv, ncur], ref [Hkv, nref] int32 device arrays whose rows are
+ * strictly ascending (as jq_select_topk writes them); rate [Hkv] fp32 device array.
+ */
+jq_status jq_hit_rate(const int32_t *cur, const int32_t *ref, int Hkv, int ncur, int nref, float *rate,
+                      jq_stream_t stream);
+
+/*
  * Synchronises `stream` and reads the status word kernels of earlier calls left in the workspace:
  * JQ_OK, JQ_ERR_TIMEOUT (a bounded wait inside a kernel gave up; outputs are invalid),
  * JQ_ERR_INVALID_ARG (an out-of-range index was met), or JQ_ERR_CUDA.

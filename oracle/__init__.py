@@ -27,6 +27,7 @@ def _load():
         lib.jq_oracle_score.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
         lib.jq_oracle_score_windowed_f64.argtypes = [vp, vp, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
         lib.jq_oracle_score_windowed.argtypes = [vp, vp, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
+        lib.jq_oracle_hit_rate.argtypes = [vp, vp, c_int, c_int, c_int, vp]
         lib.jq_oracle_pool.argtypes = [vp, c_int, c_int, c_int, vp]
         lib.jq_oracle_select.argtypes = [vp, c_int, c_int, c_int, vp]
         lib.jq_oracle_select_f32.argtypes = [vp, c_int, c_int, c_int, c_int, vp, vp]
@@ -126,6 +127,15 @@ def select_f32(scores_f32, budget, p):
     if _load().jq_oracle_select_f32(_p(s), Hkv, L, int(budget), int(p), _p(idx), _p(pooled)):
         raise ValueError("jq_oracle_select_f32: bad arguments")
     return idx, pooled
+
+
+def hit_rate(cur, ref):
+    """Eq. 6: per KV head, the share of the reference kept set `ref` [Hkv,nref] that `cur` [Hkv,ncur] also keeps."""
+    cur, ref = _chk(cur, np.int32), _chk(ref, np.int32)
+    out = np.empty(cur.shape[0], np.float64)
+    if _load().jq_oracle_hit_rate(_p(cur), _p(ref), cur.shape[0], cur.shape[1], ref.shape[1], _p(out)):
+        raise ValueError("jq_oracle_hit_rate: bad arguments")
+    return out
 
 
 def compact(K, V, idx):

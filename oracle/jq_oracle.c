@@ -351,3 +351,22 @@ int jq_oracle_evict_layer(const uint16_t *K, const uint16_t *V, const uint16_t *
     free(q);
     return rc;
 }
+
+/*
+ * Eq. 6, the critical key-value hit rate: |I_cur ^ I_ref| / |I_ref| per KV head, for two kept-index sets of
+ * the same budget regime (each row strictly ascending).  cur [Hkv,ncur], ref [Hkv,nref] -> rate [Hkv].
+ */
+int jq_oracle_hit_rate(const int32_t *cur, const int32_t *ref, int Hkv, int ncur, int nref, double *rate)
+{
+    if (Hkv < 1 || ncur < 1 || nref < 1) return 1;
+    for (int kv = 0; kv < Hkv; ++kv) {
+        const int32_t *a = cur + (size_t)kv * ncur, *b = ref + (size_t)kv * nref;
+        int hits = 0;
+        for (int i = 0; i < nref; ++i)            /* plain double loop: the definition, not a merge */
+            for (int j = 0; j < ncur; ++j)
+                if (a[j] == b[i]) { ++hits; break; }
+        rate[kv] = (double)hits / (double)nref;
+    }
+    return 0;
+}
+

@@ -17,7 +17,7 @@ EXPORTS = (
     "jq_workspace_bytes", "jq_workspace_init", "jq_num_kept", "jq_check_shape", "jq_score",
     "jq_score_fma", "jq_select_topk", "jq_compact_kv", "jq_evict_layer", "jq_host_call_bytes",
     "jq_evict_layer_host", "jq_last_device_status", "jq_launch_count", "jq_status_string",
-    "jq_score_static", "jq_score_windowed", "jq_evict_layer_windowed",
+    "jq_score_static", "jq_score_windowed", "jq_evict_layer_windowed", "jq_hit_rate",
 )
 
 
@@ -56,6 +56,7 @@ def lib():
         L.jq_score.argtypes = [vp, vp, sp, vp, vp, sz, vp]
         L.jq_score_fma.argtypes = [vp, vp, sp, vp, vp, sz, vp]
         L.jq_score_static.argtypes = [vp, vp, sp, vp, vp]
+        L.jq_hit_rate.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         L.jq_score_windowed.argtypes = [vp, vp, vp, sp, vp, vp, sz, vp]
         L.jq_evict_layer_windowed.argtypes = [vp, vp, vp, vp, sp, vp, vp, vp, vp, sz, vp]
         L.jq_select_topk.argtypes = [vp, sp, vp, vp, vp, sz, vp]
@@ -182,6 +183,12 @@ def evict_layer_host(hK, hV, hQwin, s, hKout, hVout, hkept_idx, dev_buf, stream=
     _raise("jq_evict_layer_host",
            lib().jq_evict_layer_host(_ptr(hK), _ptr(hV), _ptr(hQwin), ctypes.byref(s), _ptr(hKout), _ptr(hVout),
                                      _ptr(hkept_idx), _ptr(dev_buf), dev_buf.numel(), _stream(stream)))
+
+
+def hit_rate(cur_idx, ref_idx, rate, stream=None):
+    """Eq. 6 per KV head: the share of ref_idx's rows that cur_idx's rows also hold (rows ascending)."""
+    _raise("jq_hit_rate", lib().jq_hit_rate(_ptr(cur_idx), _ptr(ref_idx), int(cur_idx.shape[0]), int(cur_idx.shape[1]),
+                                            int(ref_idx.shape[1]), _ptr(rate), _stream(stream)))
 
 
 def last_device_status(ws, stream=None):

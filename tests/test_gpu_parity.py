@@ -402,3 +402,15 @@ def test_evict_layer_windowed_end_to_end():
     gK, gV = host_bits(Ko), host_bits(Vo)
     for kv in range(wl.Hkv):
         assert np.array_equal(gK[kv], K[kv][gidx[kv]]) and np.array_equal(gV[kv], V[kv][gidx[kv]])
+
+
+# ------------------------------------------------------------------ Eq. 6
+
+@pytest.mark.parametrize("Hkv,L,na,nb", [(1, 10, 3, 3), (8, 8192, 1024, 1024), (3, 70000, 4096, 512), (2, 300, 300, 1)])
+def test_hit_rate_matches_oracle(Hkv, L, na, nb):
+    rng = np.random.default_rng(L + na)
+    a = np.stack([np.sort(rng.choice(L, na, replace=False)) for _ in range(Hkv)]).astype(np.int32)
+    b = np.stack([np.sort(rng.choice(L, nb, replace=False)) for _ in range(Hkv)]).astype(np.int32)
+    out = torch.full((Hkv,), -1.0, dtype=torch.float32, device="cuda")
+    jq.hit_rate(torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda(), out)
+    np.testing.assert_allclose(out.cpu().numpy(), oracle.hit_rate(a, b), rtol=1e-7)

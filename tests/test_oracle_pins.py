@@ -338,3 +338,17 @@ def test_windowed_bf16_entry_matches_double_entry():
     Kw = W.bf16_bits(rng.standard_normal((Hkv, w, 128), dtype=np.float32))
     f = lambda b: W.bf16_to_f32(b).astype(np.float64)
     np.testing.assert_allclose(oracle.score_windowed(K, Q, Kw), oracle.score_windowed(f(K), f(Q), f(Kw)), rtol=1e-14)
+
+
+# ---------------------------------------------------------------- Eq. 6, hit rate
+
+def test_hit_rate_special_cases_and_library_intersection():
+    rng = np.random.default_rng(8)
+    a = np.stack([np.sort(rng.choice(500, 64, replace=False)) for _ in range(3)]).astype(np.int32)
+    np.testing.assert_array_equal(oracle.hit_rate(a, a), 1.0)                        # a set against itself
+    np.testing.assert_array_equal(oracle.hit_rate(a, a + 1000), 0.0)                  # disjoint sets
+    b = np.stack([np.sort(rng.choice(500, 40, replace=False)) for _ in range(3)]).astype(np.int32)
+    want = [len(np.intersect1d(a[k], b[k])) / 40.0 for k in range(3)]                 # library set intersection
+    np.testing.assert_allclose(oracle.hit_rate(a, b), want, rtol=0, atol=0)
+    half = np.concatenate([a[:, :32], a[:, 32:] + 1000], axis=1).astype(np.int32)    # exactly half shared
+    np.testing.assert_array_equal(oracle.hit_rate(half, a), 0.5)
