@@ -405,7 +405,7 @@ __device__ __forceinline__ void walk(int pass, int tph, int &kv, int &t)
 
 __global__ void __launch_bounds__(kThreads, 1)
 score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ,
-            const __grid_constant__ CUtensorMap mapW, const Params P)
+            const __grid_constant__ CUtensorMap mapW, const __grid_constant__ Params P)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     if (smem_u32(smem_raw) & 1023u) {   // the swizzled tiles need 1024-byte alignment; nothing has been started yet
@@ -577,7 +577,9 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll 1
                 for (; k < nunits && ok; k += kGroups) {
                     const int tl = k >> blk_shift, blk = k & blk_shift;
-                    for (; at < tl; ++at) walk(1, tph, kv, tt);
+                    // at most kGroups tiles ahead: predicated steps, no loop (taken backward branches are dear here)
+#pragma unroll
+                    for (int i_ = 0; i_ < kGroups; ++i_) if (at < tl) { walk(1, tph, kv, tt); ++at; }
                     publish_upto(kv);
                     const uint32_t uu = u + (uint32_t)k, slot = uu % kTSlots;
                     TR_ADD(8);
@@ -645,7 +647,8 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll 1
                 for (; k < nunits && ok; k += kGroups) {
                     const int tl = k >> blk_shift, blk = k & blk_shift;
-                    for (; at < tl; ++at) walk(2, tph, kv, tt);
+#pragma unroll
+                    for (int i_ = 0; i_ < kGroups; ++i_) if (at < tl) { walk(2, tph, kv, tt); ++at; }
                     TR_ADD(10);
                     hold(hs + (sg.kv0 - kv));
                     if (!ok) break;
