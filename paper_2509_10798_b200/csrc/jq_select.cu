@@ -1,7 +1,8 @@
-// Max-pool + exact top-k selection per KV head, one thread-block cluster of 8 CTAs per head.
+// Max-pool + exact top-k selection per KV head, one thread-block cluster per head: 8 CTAs when the call
+// has few heads, 4 or 2 when it has more heads than clusters fit on the GPU at a time (see choose_plan).
 //
 //   1. pool: pooled[j] = max of the centred window (edges clipped), turned into an order-preserving
-//      32-bit integer key (float order == unsigned order).  Each CTA owns a contiguous eighth of
+//      32-bit integer key (float order == unsigned order).  Each CTA owns a contiguous share of
 //      the positions and keeps its keys in shared memory (in the workspace for very long prefixes).
 //   2. radix select, 3 rounds of 11/11/10 bits, most significant first: local integer histograms
 //      are summed into the leading CTA through distributed shared memory, which finds the digit
@@ -24,7 +25,7 @@ namespace cg = cooperative_groups;
 namespace jq {
 namespace {
 
-constexpr int kCl = 8;             // CTAs per cluster (= per KV head)
+constexpr int kClMax = 8;          // most CTAs per cluster (= per KV head); the kernel also exists for 4 and 2
 constexpr int kSelThreads = 1024;
 constexpr int kBins = 2048;
 constexpr int kRawTile = 20480;    // most scores staged per pooling step (a CTA's whole share unless the prefix is very long)
@@ -39,7 +40,7 @@ struct SelCtl {
     int found_prefix_digit, found_krem, found_count;
     int cand_total;      // keys sharing the first-round digit (broadcast by the leading CTA)
     int cand_count;      // leading CTA only: candidates appended so far
-    int counts_gt[kCl], counts_eq[kCl];
+    int counts_gt[kClMax], counts_eq[kClMax];
     int warp_gt[32], warp_eq[32];
     int tot_gt, tot_eq;
     int scan[33];
@@ -96,14 +97,15 @@ __device__ __forceinline__ void find_digit(const uint32_t *g, int krem, SelCtl &
 }
 
 // The cluster copies the kept K and V rows of its head (256 bytes each: 16 lanes x 16 bytes), CTA r the
-// r-th eighth of them, once every index of the head has been written.
+// r-th share of them, once every index of the head has been written.
+template <int CL>
 __device__ __forceinline__ void copy_kept_rows(cg::cluster_group &cluster, const int32_t *out, int kv, int L, int nkeep,
                                                const uint4 *Kin, const uint4 *Vin, uint4 *Kout, uint4 *Vout)
 {
     __threadfence();
     cluster.sync();
     const int rank = (int)cluster.block_rank();
-    const int r0 = (int)((long long)rank * nkeep / kCl), r1 = (int)((long long)(rank + 1) * nkeep / kCl);
+    const int r0 = (int)((long long)rank * nkeep / CL), r1 = (int)((long long)(rank + 1) * nkeep / CL);
     const int lane16 = threadIdx.x & 15;
     for (int t = r0 + (int)(threadIdx.x >> 4); t < r1; t += kSelThreads / 16) {
         const int j = min(max(__ldcg(out + t), 0), L - 1);
@@ -113,8 +115,9 @@ __device__ __forceinline__ void copy_kept_rows(cg::cluster_group &cluster, const
     }
 }
 
-// grid (Hkv * 8), cluster 8, block 1024.
-__global__ void __cluster_dims__(kCl, 1, 1) __launch_bounds__(kSelThreads, 2)
+// grid (Hkv * CL), cluster CL, block 1024.
+template <int CL>
+__global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(kSelThreads, 2)
 select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, int32_t *__restrict__ idx,
                float *__restrict__ pooled, uint32_t *__restrict__ gkeys, int chunk, int keys_in_smem, int raw_tile,
                const uint4 *__restrict__ Kin, const uint4 *__restrict__ Vin, uint4 *__restrict__ Kout,
@@ -122,7 +125,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
 {
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
-    const int kv = blockIdx.x / kCl;
+    const int kv = blockIdx.x / CL;
     extern __shared__ __align__(16) uint8_t sm[];
     uint32_t *ghist = (uint32_t *)sm;                       // [3][kBins]; the leading CTA's copy accumulates the cluster
     uint32_t *hist = ghist + 3 * kBins;                     // [kBins]
@@ -219,7 +222,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     }
     if (nkeep >= L) {   // everything is kept (uniform over the cluster; no cluster traffic yet)
         for (int e = tid; e < n; e += kSelThreads) out[j0 + e] = j0 + e;
-        if (Kin) copy_kept_rows(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout);
+        if (Kin) copy_kept_rows<CL>(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout);
         return;
     }
     for (int i = tid; i < 3 * kBins; i += kSelThreads) ghist[i] = 0;
@@ -267,7 +270,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         cluster.sync();
         if (rank == 0) {
             find_digit(ghist + round * kBins, ctl.krem, ctl);
-            if (tid < kCl) {
+            if (tid < CL) {
                 SelCtl *rc = cluster.map_shared_rank(&ctl, tid);
                 rc->prefix = (prefix << width) | (uint32_t)ctl.found_prefix_digit;
                 rc->krem = ctl.found_krem;
@@ -312,7 +315,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
                     if (tid == 0) ctl.krem = ctl.found_krem;
                     __syncthreads();
                 }
-                if (tid < kCl) {
+                if (tid < CL) {
                     SelCtl *rc = cluster.map_shared_rank(&ctl, tid);
                     rc->prefix = pre;
                     rc->krem = ctl.found_krem;
@@ -350,7 +353,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         if (lane == 31) { ctl.tot_gt = gi; ctl.tot_eq = qi; }
     }
     __syncthreads();
-    if (tid < kCl) {
+    if (tid < CL) {
         SelCtl *rc = cluster.map_shared_rank(&ctl, tid);
         rc->counts_gt[rank] = ctl.tot_gt;
         rc->counts_eq[rank] = ctl.tot_eq;
@@ -373,7 +376,76 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         gt_before += __popc(bg);
         eq_before += __popc(be);
     }
-    if (Kin) copy_kept_rows(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout);
+    if (Kin) copy_kept_rows<CL>(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout);
+}
+
+// Shared memory of a CTA whose cluster has `cl` CTAs, the share of the head it holds, and whether its keys stay on chip.
+struct SelPlan { int cl, chunk, in_smem, raw_tile; size_t smem; };
+
+SelPlan plan_for(int L, int cl)
+{
+    SelPlan p;
+    p.cl = cl;
+    p.chunk = ((L + cl - 1) / cl + 31) / 32 * 32;
+    p.in_smem = p.chunk <= kKeysSmemMax;
+    // the staging buffer holds a CTA's share of the scores (at most kRawTile) and later up to kCandMax candidates;
+    // sized to the shape so that two CTAs fit on an SM when the share is short
+    p.raw_tile = p.chunk < kRawTile ? p.chunk : kRawTile;
+    if (p.raw_tile < kCandMax) p.raw_tile = kCandMax;
+    p.smem = (size_t)(4 * kBins + p.raw_tile + 2 * kHalo) * 4 + (p.in_smem ? (size_t)p.chunk * 4 : 0);
+    return p;
+}
+
+// Cluster size for Hkv heads of L keys.  The kernel is a chain of short phases between cluster barriers
+// (about 20 k cycles of them) plus work in proportion to a CTA's share (about 1.7 cycles per key); few heads
+// want the largest cluster (shortest chain per head), many heads want smaller ones (more heads at a time,
+// and the chain is paid once per head either way).  Estimated as rounds of resident clusters times the
+// time of one.
+SelPlan choose_plan(int Hkv, int L, int sms)
+{
+    SelPlan best = plan_for(L, kClMax);
+    double best_cost = 0;
+    for (int cl = kClMax; cl >= 2; cl >>= 1) {
+        const SelPlan p = plan_for(L, cl);
+        if (cl != kClMax && !p.in_smem) break;
+        const int per_sm = p.smem <= 113 * 1024 ? 2 : 1;
+        const int resident = sms * per_sm / cl > 0 ? sms * per_sm / cl : 1;
+        const double cost = (double)((Hkv + resident - 1) / resident) * (20000.0 + 1.7 * p.chunk);
+        if (cl == kClMax || cost < best_cost) { best = p; best_cost = cost; }
+    }
+    return best;
+}
+
+template <int CL>
+jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape &s, int nkeep, int32_t *idx, float *pooled,
+                           const Workspace &w, cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout, int dev)
+{
+    static bool attr_done[64] = {};
+    if (!attr_done[dev]) {
+        const int max_smem = (4 * kBins + kRawTile + 2 * kHalo + kKeysSmemMax) * 4;
+        if (cudaFuncSetAttribute(select_cluster<CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
+            return JQ_ERR_CUDA;
+        attr_done[dev] = true;
+    }
+    // Launched with programmatic stream serialisation: the CTAs may be set up while the kernel before it in
+    // the stream (the scoring kernel) drains; the kernel waits for that kernel's memory before reading anything.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(s.Hkv * CL));
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.dynamicSmemBytes = p.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, select_cluster<CL>, scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, w.keys, p.chunk,
+                           p.in_smem, p.raw_tile, (const uint4 *)K, (const uint4 *)V, (uint4 *)Kout, (uint4 *)Vout) != cudaSuccess) {
+        cudaGetLastError();
+        return JQ_ERR_CUDA;
+    }
+    count_launch(1);
+    return check_launch();
 }
 
 }  // namespace
@@ -382,42 +454,16 @@ jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, fl
                         const Workspace &w, cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout)
 {
     const int nkeep = s.budget < s.L ? s.budget : s.L;
-    int chunk = (s.L + kCl - 1) / kCl;
-    chunk = (chunk + 31) / 32 * 32;
-    const int in_smem = chunk <= kKeysSmemMax;
-    // the staging buffer holds a CTA's share of the scores (at most kRawTile) and later up to kCandMax candidates;
-    // sized to the shape so that two CTAs fit on an SM when the prefix is short
-    int raw_tile = chunk < kRawTile ? chunk : kRawTile;
-    if (raw_tile < kCandMax) raw_tile = kCandMax;
-    const size_t smem = (size_t)(4 * kBins + raw_tile + 2 * kHalo) * 4 + (in_smem ? (size_t)chunk * 4 : 0);
-    static bool attr_done[64] = {};
+    static int sms[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return JQ_ERR_CUDA;
-    if (!attr_done[dev]) {
-        const int max_smem = (4 * kBins + kRawTile + 2 * kHalo + kKeysSmemMax) * 4;
-        if (cudaFuncSetAttribute(select_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
-            return JQ_ERR_CUDA;
-        attr_done[dev] = true;
+    if (!sms[dev] && cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return JQ_ERR_CUDA;
+    const SelPlan p = choose_plan(s.Hkv, s.L, sms[dev]);
+    switch (p.cl) {
+    case 2: return launch_select_cl<2>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev);
+    case 4: return launch_select_cl<4>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev);
+    default: return launch_select_cl<8>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev);
     }
-    // Launched with programmatic stream serialisation: the CTAs may be set up while the kernel before it in
-    // the stream (the scoring kernel) drains; the kernel waits for that kernel's memory before reading anything.
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(s.Hkv * kCl));
-    cfg.blockDim = dim3(kSelThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, select_cluster, scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, w.keys, chunk,
-                           in_smem, raw_tile, (const uint4 *)K, (const uint4 *)V, (uint4 *)Kout, (uint4 *)Vout) != cudaSuccess) {
-        cudaGetLastError();
-        return JQ_ERR_CUDA;
-    }
-    count_launch(1);
-    return check_launch();
 }
 
 }  // namespace jq

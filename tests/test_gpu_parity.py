@@ -115,6 +115,21 @@ def test_select_bit_exact(Hkv, L, B, p, kind):
     assert np.array_equal(got_idx, want_idx)
 
 
+# With many heads the selection kernel runs smaller clusters (4 or 2 CTAs per head instead of 8): same results.
+@pytest.mark.parametrize("Hkv,L,B,p", [(64, 4096, 512, 7), (160, 5000, 700, 7), (300, 1000, 100, 5), (148, 40000, 2048, 7)])
+@pytest.mark.parametrize("kind", ["random", "ties"])
+def test_select_many_heads_bit_exact(Hkv, L, B, p, kind):
+    rng = np.random.default_rng(Hkv * 7 + L)
+    if kind == "random":
+        s32 = rng.random((Hkv, L), dtype=np.float32)
+    else:
+        s32 = (rng.integers(0, 5, size=(Hkv, L)) / 4.0).astype(np.float32)
+    want_idx, want_pooled = oracle.select_f32(s32, B, p)
+    got_idx, got_pooled = gpu_select(s32, jq.shape(Hkv, Hkv, L, 1, B, p))
+    assert np.array_equal(got_pooled.view(np.uint32), want_pooled.view(np.uint32))
+    assert np.array_equal(got_idx, want_idx)
+
+
 def test_select_all_equal_keeps_lowest_indices():
     s32 = np.full((2, 5000), 0.25, np.float32)
     idx, _ = gpu_select(s32, jq.shape(2, 2, 5000, 1, 777, 7))
@@ -155,7 +170,7 @@ def run_e2e(wl, K, V, Q, pooled=None):
 
 
 @pytest.mark.parametrize("wl", [W.CFG1, W.CFG2, W.CFG2.with_budget(100000), W.CFG4[0], W.CFG4[1],
-                                small_wl(2, 4, 16, 5, 3), small_wl(1, 4, 64, 1, 1)],
+                                small_wl(2, 4, 16, 5, 3), small_wl(1, 4, 64, 1, 1), small_wl(160, 1, 4, 5000, 700)],
                          ids=lambda w: "%s-L%d-B%d" % (w.name, w.L, w.budget))
 def test_evict_layer_end_to_end(wl):
     K, V, Q, _ = W.make_layer(wl)
