@@ -28,6 +28,7 @@ def _load():
         lib.jq_oracle_score_windowed_f64.argtypes = [vp, vp, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
         lib.jq_oracle_score_windowed.argtypes = [vp, vp, vp, c_int, c_int, c_int, c_int, c_int, vp, vp]
         lib.jq_oracle_hit_rate.argtypes = [vp, vp, c_int, c_int, c_int, vp]
+        lib.jq_oracle_decode_attention.argtypes = [vp, vp, vp, c_int, c_int, c_int, c_int, vp]
         lib.jq_oracle_pool.argtypes = [vp, c_int, c_int, c_int, vp]
         lib.jq_oracle_select.argtypes = [vp, c_int, c_int, c_int, vp]
         lib.jq_oracle_select_f32.argtypes = [vp, c_int, c_int, c_int, c_int, vp, vp]
@@ -135,6 +136,16 @@ def hit_rate(cur, ref):
     out = np.empty(cur.shape[0], np.float64)
     if _load().jq_oracle_hit_rate(_p(cur), _p(ref), cur.shape[0], cur.shape[1], ref.shape[1], _p(out)):
         raise ValueError("jq_oracle_hit_rate: bad arguments")
+    return out
+
+
+def decode_attention(Kc, Vc, q):
+    """One decoding step over the pruned cache: Kc, Vc [Hkv,n,d], q [Hq,d] bf16 bits -> out [Hq,d] float64."""
+    Kc, Vc, q = _chk(Kc, np.uint16), _chk(Vc, np.uint16, Kc.shape), _chk(q, np.uint16)
+    Hkv, n, d = Kc.shape
+    out = np.empty((q.shape[0], d), np.float64)
+    if q.shape[1] != d or _load().jq_oracle_decode_attention(_p(Kc), _p(Vc), _p(q), Hkv, q.shape[0], n, d, _p(out)):
+        raise ValueError("jq_oracle_decode_attention: bad arguments")
     return out
 
 

@@ -28,6 +28,10 @@
  *   compact Inference section (the pruned cache is what decoding continues
  *           with): rows K[kv,idx,:], V[kv,idx,:] copied bit for bit.
  *
+ * (jq_oracle_decode_attention is the step after the pass: one decoding step's attention over the pruned
+ * cache, the inference section's "decoding continues with the retained pairs"; pinned against a library
+ * softmax and matrix product, the q = 0 mean, a dominant key and n = 1.)
+ *
  * (jq_oracle_score_windowed is the window-inclusive variant of the scores; its pins are a library
  * softmax over the concatenated, causally masked logits, the Q = 0 closed form and the limit of a
  * window that attracts no mass.)
@@ -367,6 +371,41 @@ int jq_oracle_hit_rate(const int32_t *cur, const int32_t *ref, int Hkv, int ncur
                 if (a[j] == b[i]) { ++hits; break; }
         rate[kv] = (double)hits / (double)nref;
     }
+    return 0;
+}
+
+/*
+ * One decoding step over the pruned cache (inference section: after the eviction, decoding continues from the
+ * end of the input with the retained pairs only).  For query head h of KV head kv = h / group:
+ *     s_j = (q[h,:] . Kc[kv,j,:]) / sqrt(d),  P = softmax_j(s),  out[h,:] = sum_j P_j Vc[kv,j,:]
+ * Kc, Vc [Hkv,n,d] and q [Hq,d] are bf16 bit patterns; out [Hq,d] is fp64.
+ */
+int jq_oracle_decode_attention(const uint16_t *Kc, const uint16_t *Vc, const uint16_t *q, int Hkv, int Hq, int n, int d,
+                               double *out)
+{
+    if (Hkv < 1 || Hq < 1 || Hq % Hkv || n < 1 || d < 1) return 1;
+    const int group = Hq / Hkv;
+    double *s = (double *)malloc((size_t)n * sizeof(double));
+    if (!s) return 2;
+    for (int h = 0; h < Hq; ++h) {
+        const int kv = h / group;
+        double m = -INFINITY;
+        for (int j = 0; j < n; ++j) {
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c)
+                acc += bf16_to_double(q[(size_t)h * d + c]) * bf16_to_double(Kc[((size_t)kv * n + j) * d + c]);
+            s[j] = acc / sqrt((double)d);
+            if (s[j] > m) m = s[j];
+        }
+        double z = 0.0;
+        for (int j = 0; j < n; ++j) { s[j] = exp(s[j] - m); z += s[j]; }
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int j = 0; j < n; ++j) acc += s[j] * bf16_to_double(Vc[((size_t)kv * n + j) * d + c]);
+            out[(size_t)h * d + c] = acc / z;
+        }
+    }
+    free(s);
     return 0;
 }
 

@@ -352,3 +352,51 @@ def test_hit_rate_special_cases_and_library_intersection():
     np.testing.assert_allclose(oracle.hit_rate(a, b), want, rtol=0, atol=0)
     half = np.concatenate([a[:, :32], a[:, 32:] + 1000], axis=1).astype(np.int32)    # exactly half shared
     np.testing.assert_array_equal(oracle.hit_rate(half, a), 0.5)
+
+
+# ---------------------------------------------------------------- decoding step over the pruned cache
+
+def _decode_case(Hkv, group, n, seed, d=128):
+    rng = np.random.default_rng(seed)
+    Kc = W.bf16_bits(rng.standard_normal((Hkv, n, d)).astype(np.float32))
+    Vc = W.bf16_bits(rng.standard_normal((Hkv, n, d)).astype(np.float32))
+    q = W.bf16_bits((2.0 * rng.standard_normal((Hkv * group, d))).astype(np.float32))
+    return Kc, Vc, q
+
+
+def test_decode_attention_matches_library_softmax_and_matmul():
+    Kc, Vc, q = _decode_case(3, 4, 257, 5)
+    got = oracle.decode_attention(Kc, Vc, q)
+    Kf, Vf, qf = (torch.from_numpy(W.bf16_to_f32(x).astype(np.float64)) for x in (Kc, Vc, q))
+    for h in range(q.shape[0]):
+        kv = h // 4
+        p = torch.softmax(Kf[kv] @ qf[h] / math.sqrt(128.0), dim=0)
+        np.testing.assert_allclose(got[h], (p @ Vf[kv]).numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_decode_attention_closed_forms():
+    Kc, Vc, q = _decode_case(2, 2, 64, 6)
+    Vf = W.bf16_to_f32(Vc).astype(np.float64)
+    # q = 0: uniform weights, the mean of the head's V rows (and of the RIGHT head: GQA mapping h -> h // group)
+    got = oracle.decode_attention(Kc, Vc, np.zeros_like(q))
+    for h in range(4):
+        np.testing.assert_allclose(got[h], Vf[h // 2].mean(0), rtol=1e-13, atol=1e-15)
+    # one key aligned with the query and scaled up takes all the mass: the output is its V row
+    Kf = W.bf16_to_f32(Kc).copy()
+    qf = W.bf16_to_f32(q)
+    Kf[1, 17] = 64.0 * qf[3]                       # head 3 -> KV head 1
+    got = oracle.decode_attention(W.bf16_bits(Kf), Vc, q)
+    np.testing.assert_allclose(got[3], Vf[1, 17], rtol=0, atol=1e-9)
+    # n = 1: the single V row, whatever the logits
+    got = oracle.decode_attention(Kc[:, :1], Vc[:, :1], q)
+    for h in range(4):
+        np.testing.assert_array_equal(got[h], Vf[h // 2, 0])
+    # the order of the keys does not matter when V is permuted alike
+    perm = np.random.default_rng(0).permutation(64)
+    np.testing.assert_allclose(oracle.decode_attention(Kc[:, perm], Vc[:, perm], q), oracle.decode_attention(Kc, Vc, q),
+                               rtol=1e-12, atol=1e-14)
+    # scaling: logits are divided by sqrt(d) (a query scaled by 4 with d = 128 is not the same as one with d = 8)
+    Kc8, Vc8, q8 = _decode_case(1, 1, 9, 7, d=8)
+    s = W.bf16_to_f32(Kc8)[0].astype(np.float64) @ W.bf16_to_f32(q8)[0].astype(np.float64) / math.sqrt(8.0)
+    p = np.exp(s - s.max()); p /= p.sum()
+    np.testing.assert_allclose(oracle.decode_attention(Kc8, Vc8, q8)[0], p @ W.bf16_to_f32(Vc8)[0].astype(np.float64), rtol=1e-12)
