@@ -36,6 +36,7 @@ UNIT = "tokens/s"
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--decode", action="store_true", help="also time one decoding step over a layer's pruned cache")
     ap.add_argument("--steps", type=int, default=60)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -343,6 +344,17 @@ def run_ours(args):
     t_layer = ms * 1e-3 / (args.steps * layers)
     value = job_value(wl, world, t_layer)
 
+    # the step after the pass (optional, outside the metric): one decoding position over the pruned cache of a layer
+    decode = None
+    if args.decode:
+        qd = Qs[0][:, -1, :].contiguous()                       # [Hq, d]: the last soft token's queries as a decoding step
+        od = torch.empty((wl.Hq, wl.d), dtype=torch.float32, device="cuda")
+        wsd = torch.empty(jq.decode_workspace_bytes(wl.Hkv, wl.Hq, nkeep), dtype=torch.uint8, device="cuda")
+        nb = 32
+        t_dec = timed(lambda j: jq.decode_attention(Ko, Vo, qd, od, wsd, stream=stream))
+        decode = {"what": "jq_decode_attention over one layer's pruned cache (2 launches)", "n": nkeep, "ms_per_layer": float(t_dec),
+                  "cache_gbs": 2.0 * wl.Hkv * nkeep * wl.d * 2 / (t_dec * 1e-3) / 1e9}
+
     # end to end through the host-buffer entry point: pinned host tensors in, pinned host results out
     e2e = None
     if not args.no_e2e:
@@ -410,6 +422,8 @@ def run_ours(args):
             "per_layer_calls": per_layer_calls,
             "tokens_discarded_per_s": world * (wl.L - nkeep) / t_layer,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline}
+    if decode is not None:
+        line["decode_step"] = decode
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(wl, *host0)
     if world > 1:

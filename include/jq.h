@@ -184,6 +184,19 @@ jq_status jq_hit_rate(const int32_t *cur, const int32_t *ref, int Hkv, int ncur,
                       jq_stream_t stream);
 
 /*
+ * The step after the pass (inference section: decoding continues from the end of the input with the retained
+ * pairs only): attention of one new query position over the pruned cache,
+ *     out[h,:] = softmax_j( q[h,:] . Kc[kv,j,:] / sqrt(d) ) Vc[kv,:,:],   kv = h / (Hq / Hkv),  d = 128.
+ * Kc, Vc: device, bf16 [Hkv, n, 128] (what jq_evict_layer wrote), 16-byte aligned.  q: device, bf16 [Hq, 128].
+ * out: device, fp32 [Hq, 128], 16-byte aligned.  workspace: device, 16-byte aligned, at least
+ * jq_decode_workspace_bytes(Hkv, Hq, n) bytes (0 for arguments the call would reject); no initialisation
+ * needed, contents undefined afterwards.  Hq / Hkv <= 8.  Asynchronous on `stream`; two launches.
+ */
+size_t jq_decode_workspace_bytes(int Hkv, int Hq, int n);
+jq_status jq_decode_attention(const void *Kc, const void *Vc, const void *q, int Hkv, int Hq, int n, float *out,
+                              void *workspace, size_t workspace_bytes, jq_stream_t stream);
+
+/*
  * Synchronises `stream` and reads the status word kernels of earlier calls left in the workspace:
  * JQ_OK, JQ_ERR_TIMEOUT (a bounded wait inside a kernel gave up; outputs are invalid),
  * JQ_ERR_INVALID_ARG (an out-of-range index was met), or JQ_ERR_CUDA.

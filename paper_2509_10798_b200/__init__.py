@@ -18,6 +18,7 @@ EXPORTS = (
     "jq_score_fma", "jq_select_topk", "jq_compact_kv", "jq_evict_layer", "jq_host_call_bytes",
     "jq_evict_layer_host", "jq_last_device_status", "jq_launch_count", "jq_status_string",
     "jq_score_static", "jq_score_windowed", "jq_evict_layer_windowed", "jq_hit_rate",
+    "jq_decode_workspace_bytes", "jq_decode_attention",
 )
 
 
@@ -56,6 +57,9 @@ def lib():
         L.jq_score.argtypes = [vp, vp, sp, vp, vp, sz, vp]
         L.jq_score_fma.argtypes = [vp, vp, sp, vp, vp, sz, vp]
         L.jq_score_static.argtypes = [vp, vp, sp, vp, vp]
+        L.jq_decode_workspace_bytes.argtypes = [ci, ci, ci]
+        L.jq_decode_workspace_bytes.restype = ctypes.c_size_t
+        L.jq_decode_attention.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, ctypes.c_size_t, vp]
         L.jq_hit_rate.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         L.jq_score_windowed.argtypes = [vp, vp, vp, sp, vp, vp, sz, vp]
         L.jq_evict_layer_windowed.argtypes = [vp, vp, vp, vp, sp, vp, vp, vp, vp, sz, vp]
@@ -183,6 +187,16 @@ def evict_layer_host(hK, hV, hQwin, s, hKout, hVout, hkept_idx, dev_buf, stream=
     _raise("jq_evict_layer_host",
            lib().jq_evict_layer_host(_ptr(hK), _ptr(hV), _ptr(hQwin), ctypes.byref(s), _ptr(hKout), _ptr(hVout),
                                      _ptr(hkept_idx), _ptr(dev_buf), dev_buf.numel(), _stream(stream)))
+
+
+def decode_workspace_bytes(Hkv, Hq, n):
+    return int(lib().jq_decode_workspace_bytes(int(Hkv), int(Hq), int(n)))
+
+
+def decode_attention(Kc, Vc, q, out, ws, stream=None):
+    """One decoding step over the pruned cache: Kc, Vc [Hkv,n,128] bf16, q [Hq,128] bf16 -> out [Hq,128] fp32."""
+    _raise("jq_decode_attention", lib().jq_decode_attention(_ptr(Kc), _ptr(Vc), _ptr(q), int(Kc.shape[0]), int(q.shape[0]),
+                                                            int(Kc.shape[1]), _ptr(out), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
 
 
 def hit_rate(cur_idx, ref_idx, rate, stream=None):

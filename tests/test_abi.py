@@ -76,6 +76,12 @@ def test_pointer_errors_are_caught_on_the_host():
     assert lib.jq_evict_layer(a, a, a, ref, a, a, a, a, 16, None) == jq.JQ_ERR_WORKSPACE
     assert lib.jq_evict_layer_host(a, a, a, ref, a, a, a, a, 16, None) == jq.JQ_ERR_WORKSPACE
     assert lib.jq_evict_layer(a, a, a, None, a, a, a, a, n, None) == jq.JQ_ERR_INVALID_ARG
+    assert lib.jq_decode_attention(a, a, a, 2, 8, 100, None, a, 1 << 20, None) == jq.JQ_ERR_INVALID_ARG
+    assert lib.jq_decode_attention(a, a, a, 2, 7, 100, a, a, 1 << 20, None) == jq.JQ_ERR_INVALID_ARG      # Hq % Hkv
+    assert lib.jq_decode_attention(a, a, a, 1, 16, 100, a, a, 1 << 20, None) == jq.JQ_ERR_UNSUPPORTED     # group > 8
+    assert lib.jq_decode_attention(a, a, a, 2, 8, 100, a, a, 16, None) == jq.JQ_ERR_WORKSPACE
+    assert jq.decode_workspace_bytes(2, 8, 100) >= 8 * 2 * 130 * 4 and jq.decode_workspace_bytes(2, 7, 100) == 0
+    assert lib.jq_hit_rate(a, a, 0, 4, 4, a, None) == jq.JQ_ERR_INVALID_ARG
     assert lib.jq_last_device_status(None, None) == jq.JQ_ERR_INVALID_ARG
     assert jq.status_string(jq.JQ_ERR_TIMEOUT) and jq.status_string(99)
     assert jq.launch_count() == 0      # nothing above reached a launch

@@ -429,3 +429,51 @@ def test_hit_rate_matches_oracle(Hkv, L, na, nb):
     out = torch.full((Hkv,), -1.0, dtype=torch.float32, device="cuda")
     jq.hit_rate(torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda(), out)
     np.testing.assert_allclose(out.cpu().numpy(), oracle.hit_rate(a, b), rtol=1e-7)
+
+
+# ------------------------------------------------------------------ the step after the pass: decoding over the pruned cache
+
+def gpu_decode(Kc, Vc, q):
+    dKc, dVc, dq = dev_bf16(Kc), dev_bf16(Vc), dev_bf16(q)
+    out = torch.full((q.shape[0], 128), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(jq.decode_workspace_bytes(Kc.shape[0], q.shape[0], Kc.shape[1]), dtype=torch.uint8, device="cuda")
+    jq.decode_attention(dKc, dVc, dq, out, ws)
+    torch.cuda.synchronize()
+    return out.cpu().numpy()
+
+
+# fp32 sums of at most a few thousand products of bf16 values of unit size, weights from exp2f: absolute error of the
+# output (a convex combination of V values of size ~1) stays below 2e-5
+@pytest.mark.parametrize("Hkv,group,n", [(1, 1, 1), (2, 4, 63), (2, 4, 64), (3, 8, 65), (8, 4, 512), (8, 4, 1024), (2, 2, 5000),
+                                         (8, 4, 4096)])
+def test_decode_attention_matches_oracle(Hkv, group, n):
+    rng = np.random.default_rng(n * 13 + group)
+    Kc = W.bf16_bits(rng.standard_normal((Hkv, n, 128)).astype(np.float32))
+    Vc = W.bf16_bits(rng.standard_normal((Hkv, n, 128)).astype(np.float32))
+    q = W.bf16_bits((3.0 * rng.standard_normal((Hkv * group, 128))).astype(np.float32))
+    np.testing.assert_allclose(gpu_decode(Kc, Vc, q), oracle.decode_attention(Kc, Vc, q), rtol=1e-4, atol=2e-5)
+
+
+def test_decode_attention_large_logits_stay_finite():
+    rng = np.random.default_rng(3)
+    u = rng.standard_normal(128).astype(np.float32)
+    Kc = W.bf16_bits((30.0 * u[None, None, :] * rng.standard_normal((2, 300, 1))).astype(np.float32))
+    Vc = W.bf16_bits(rng.standard_normal((2, 300, 128)).astype(np.float32))
+    q = W.bf16_bits(np.tile(30.0 * u, (8, 1)).astype(np.float32))
+    got = gpu_decode(Kc, Vc, q)
+    assert np.all(np.isfinite(got))
+    np.testing.assert_allclose(got, oracle.decode_attention(Kc, Vc, q), rtol=1e-4, atol=2e-5)
+
+
+def test_evict_then_decode_then_evict_again():
+    """Streaming use: evict, decode over the pruned cache, append new rows, evict again - every step against the oracle."""
+    wl = small_wl(2, 4, 16, 3000, 400)
+    K, V, Q, _ = W.make_layer(wl)
+    run_e2e(wl, K, V, Q)
+    Kc, Vc, _ = gpu_evict(K, V, Q, shape_of(wl))
+    q = np.ascontiguousarray(Q[:, -1, :])                    # the last soft token's queries stand in for a decoding step
+    np.testing.assert_allclose(gpu_decode(Kc, Vc, q), oracle.decode_attention(Kc, Vc, q), rtol=1e-4, atol=2e-5)
+    # 200 newly decoded positions join the pruned cache, which is evicted again to the budget
+    K2, V2, Q2, _ = W.make_layer(small_wl(2, 4, 16, 200, 400), layer=1)
+    Kn, Vn = np.concatenate([Kc, K2], axis=1), np.concatenate([Vc, V2], axis=1)
+    run_e2e(small_wl(2, 4, 16, Kn.shape[1], 400), Kn, Vn, Q2)
