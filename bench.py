@@ -375,7 +375,8 @@ def run_ours(args):
         e1.record(stream)
         barrier()
         t_e2e_layer = max_over_ranks(e0.elapsed_time(e1), world) * 1e-3 / (n_e2e * e2e_layers)
-        h2d = e2e_layers * (2 * hK.numel() + hQ.numel()) * 2
+        # K and the queries are copied whole; of V (page-locked) only the kept rows cross, read in place by the kernel
+        h2d = e2e_layers * (hK.numel() + hQ.numel() + hVo.numel()) * 2
         d2h = e2e_layers * (2 * hKo.numel() * 2 + hidx.numel() * 4)
         e2e = {"value": world * wl.L / t_e2e_layer, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "layers_per_step": e2e_layers, "ms_per_layer": t_e2e_layer * 1e3}

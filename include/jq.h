@@ -165,7 +165,9 @@ jq_status jq_evict_layer(const void *K, const void *V, const void *Qwin, const j
 /*
  * jq_evict_layer for callers whose tensors live in HOST memory (pinned memory gives asynchronous
  * copies).  hK, hV, hQwin are copied to the device, the layer is evicted, and hKout, hVout,
- * hkept_idx are copied back, all on `stream`; the call returns without synchronising.
+ * hkept_idx are copied back, all on `stream`; the call returns without synchronising.  When hV is
+ * page-locked memory only its kept rows cross to the device (the kernel reads them in place); hV must
+ * then stay unchanged until the stream has passed the call, like every other host buffer.
  * dev_buf is a device buffer of at least jq_host_call_bytes(shape) bytes (it holds the device
  * copies and the workspace).
  */

@@ -189,8 +189,18 @@ jq_status jq_evict_layer_host(const void *hK, const void *hV, const void *hQwin,
     if (cudaMemsetAsync(ws, 0, 256, st) != cudaSuccess) return JQ_ERR_CUDA;
     if (cudaMemcpyAsync(dQ, hQwin, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
     if (cudaMemcpyAsync(dK, hK, kvb, cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
-    if (cudaMemcpyAsync(dV, hV, kvb, cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
-    rc = jq_evict_layer(dK, dV, dQ, s, dKo, dVo, (int32_t *)dI, ws, wsb, stream);
+    // V is read at the kept rows only.  A page-locked host buffer is mapped into the device's address space: the
+    // selection kernel then fetches those rows from it directly and the copy of all of V is skipped.
+    const void *v_src = dV;
+    cudaPointerAttributes pa;
+    if (cudaPointerGetAttributes(&pa, hV) == cudaSuccess && pa.type == cudaMemoryTypeHost && pa.devicePointer &&
+        !((uintptr_t)pa.devicePointer & 15u)) {
+        v_src = pa.devicePointer;
+    } else {
+        cudaGetLastError();
+        if (cudaMemcpyAsync(dV, hV, kvb, cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
+    }
+    rc = jq_evict_layer(dK, v_src, dQ, s, dKo, dVo, (int32_t *)dI, ws, wsb, stream);
     if (rc != JQ_OK) return rc;
     if (cudaMemcpyAsync(hkept_idx, dI, ib, cudaMemcpyDeviceToHost, st) != cudaSuccess) return JQ_ERR_CUDA;
     if (cudaMemcpyAsync(hKout, dKo, ob, cudaMemcpyDeviceToHost, st) != cudaSuccess) return JQ_ERR_CUDA;

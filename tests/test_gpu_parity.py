@@ -215,10 +215,13 @@ def test_host_entry_matches_device_entry():
     hVo = torch.zeros_like(hKo).pin_memory()
     hidx = torch.zeros((s.Hkv, wl.nkeep), dtype=torch.int32).pin_memory()
     buf = torch.empty(jq.host_call_bytes(s), dtype=torch.uint8, device="cuda")
-    jq.evict_layer_host(hK, hV, hQ, s, hKo, hVo, hidx, buf)
-    torch.cuda.synchronize()
-    assert np.array_equal(hidx.numpy(), gidx)
-    assert np.array_equal(hKo.numpy().view(np.uint16), gKo) and np.array_equal(hVo.numpy().view(np.uint16), gVo)
+    # page-locked V (only the kept rows cross to the device) and pageable V (copied whole): same results
+    for v_in in (hV, torch.from_numpy(V.view(np.int16).copy())):
+        hKo.zero_(); hVo.zero_(); hidx.zero_()
+        jq.evict_layer_host(hK, v_in, hQ, s, hKo, hVo, hidx, buf)
+        torch.cuda.synchronize()
+        assert np.array_equal(hidx.numpy(), gidx)
+        assert np.array_equal(hKo.numpy().view(np.uint16), gKo) and np.array_equal(hVo.numpy().view(np.uint16), gVo)
 
 
 # ------------------------------------------------------------------ full-size workloads (bench launch configuration)
