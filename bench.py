@@ -36,6 +36,7 @@ UNIT = "tokens/s"
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--fma-compare", action="store_true", help="also time the CUDA-core comparator of the scoring step")
     ap.add_argument("--decode", action="store_true", help="also time one decoding step over a layer's pruned cache")
     ap.add_argument("--steps", type=int, default=60)
     ap.add_argument("--warmup", type=int, default=3)
@@ -344,6 +345,15 @@ def run_ours(args):
     t_layer = ms * 1e-3 / (args.steps * layers)
     value = job_value(wl, world, t_layer)
 
+    # the CUDA-core comparator of the scoring step (optional, outside the metric): same two passes with fp32 FMAs
+    fma_cmp = None
+    if args.fma_compare:
+        nb = 8
+        t_tc = timed(lambda j: jq.score(Ks[j], Qs[j], s, scores[j % len(scores)], ws, stream=stream))
+        t_fma = timed(lambda j: jq.score(Ks[j], Qs[j], s, scores[j % len(scores)], ws, fma=True, stream=stream))
+        fma_cmp = {"what": "jq_score (tcgen05) against jq_score_fma (CUDA cores), one layer per call",
+                   "ms_per_layer_tensor": float(t_tc), "ms_per_layer_fma": float(t_fma), "ratio": float(t_fma / t_tc)}
+
     # the step after the pass (optional, outside the metric): one decoding position over the pruned cache of a layer
     decode = None
     if args.decode:
@@ -425,6 +435,8 @@ def run_ours(args):
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline}
     if decode is not None:
         line["decode_step"] = decode
+    if fma_cmp is not None:
+        line["fma_comparator"] = fma_cmp
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(wl, *host0)
     if world > 1:

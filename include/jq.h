@@ -155,8 +155,10 @@ jq_status jq_compact_kv(const void *K, const void *V, const int32_t *kept_idx,
                         const jq_shape *shape, void *Kout, void *Vout, jq_stream_t stream);
 
 /*
- * The whole pass for one layer: jq_score -> jq_select_topk -> jq_compact_kv on one stream, with
- * the scores kept in the workspace.
+ * The whole pass for one layer, with the results of jq_score -> jq_select_topk -> jq_compact_kv, on one
+ * stream in two launches (the selection kernel also copies the kept rows); the scores stay in the
+ * workspace.  K may hold several layers of equal shape stacked along the KV-head axis (Hkv = layers x
+ * heads per layer, Qwin stacked alike): heads are independent, so one call evicts them all.
  */
 jq_status jq_evict_layer(const void *K, const void *V, const void *Qwin, const jq_shape *shape,
                          void *Kout, void *Vout, int32_t *kept_idx, void *ws, size_t ws_bytes,
