@@ -6,8 +6,9 @@
 //                 shared-memory stages; the query rows of a KV head into one of two stationary buffers;
 //   warp 1        issues tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory; the warp stays converged, one
 //                 elected lane issues) and owns the TMEM allocation;
-//   warps 2..     kGroups epilogue groups of 128 threads.  Accumulator block u (128 TMEM lanes x 128
-//                 columns) sits in slot u % 4 and is taken by group u % kGroups, 32 columns at a time;
+//   warps 2..     kGroups epilogue groups of 128 threads (3 for up to 128 query rows per KV head, 4 above).
+//                 Accumulator block u (128 TMEM lanes x 128 columns) sits in slot u % 4 and is taken by
+//                 group u % kGroups, 32 columns at a time;
 //   then          one warp that merges the per-warp partial row statistics of pass 1 across the grid,
 //                 and one that stages the merged row normalisers of the next KV head of pass 2.
 // The operand roles are swapped between the passes so that no reduction crosses threads:
@@ -59,20 +60,17 @@ namespace {
 #define TR_DUMP
 #endif
 
-#ifndef JQ_GROUPS
-#define JQ_GROUPS 3
-#endif
 #ifndef JQ_POLY_OF8
 #define JQ_POLY_OF8 2
 #endif
 
 constexpr int kTile = 128;                       // keys per tile
 constexpr int kMaxStages = 5;                    // K ring depth (5 when R <= 128, 3 above)
-constexpr int kGroups = JQ_GROUPS;               // epilogue groups of 128 threads
+// Epilogue groups of 128 threads: the kernel is built for 3 (R <= 128) and for 4 (R > 128, where the fourth
+// group is worth more than the slot it takes from the MMA's lead: config 5 runs 3 % faster, config 3 4 % slower)
+constexpr int kGroupsNarrow = 3, kGroupsWide = 4;
 constexpr int kTSlots = 4;                       // accumulator slots in tensor memory
-constexpr int kEpiWarps = 4 * kGroups;
-constexpr int kMergeWarp = 2 + kEpiWarps, kStageWarp = kMergeWarp + 1;
-constexpr int kThreads = (kStageWarp + 1) * 32;
+constexpr int threads_for(int groups) { return (4 * groups + 4) * 32; }   // producer, MMA, 4 warps per group, merge, stage
 constexpr uint32_t kHalfBytes = kTile * 128;     // one 64-column half of a K tile (128-byte rows)
 constexpr uint32_t kStageBytes = 2 * kHalfBytes; // 32 KiB
 constexpr uint32_t kCtlBytes = 3072;             // barriers, flags, M_r
@@ -96,7 +94,7 @@ static_assert(kChunk == 32 || kChunk == 64, "kChunk");
 constexpr int kPolyOf8 = JQ_POLY_OF8;            // of every 8 pairs of exponentials, this many go to the FMA pipe
 // words of the workspace status block
 constexpr int kWStatus = 0, kWDone = 1, kWCnt1 = 8, kWCnt2 = 12;
-static_assert(kSlots >= kGroups * 148, "one partial slot per epilogue group and CTA");
+static_assert(kSlots >= kGroupsWide * 148 && kSlots >= kGroupsNarrow * 148, "one partial slot per epilogue group and CTA");
 
 struct Ctl {
     uint64_t full[kMaxStages], empty[kMaxStages];
@@ -403,10 +401,12 @@ __device__ __forceinline__ void walk(int pass, int tph, int &kv, int &t)
 
 // ------------------------------------------------------------------ the kernel
 
-__global__ void __launch_bounds__(kThreads, 1)
+template <int kGroups>
+__global__ void __launch_bounds__(threads_for(kGroups), 1)
 score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ,
             const __grid_constant__ CUtensorMap mapW, const __grid_constant__ Params P)
 {
+    constexpr int kEpiWarps = 4 * kGroups, kMergeWarp = 2 + kEpiWarps, kStageWarp = kMergeWarp + 1;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     if (smem_u32(smem_raw) & 1023u) {   // the swizzled tiles need 1024-byte alignment; nothing has been started yet
         if (threadIdx.x == 0) atomicMax(P.status + kWStatus, (int)JQ_ERR_CUDA);
@@ -897,8 +897,11 @@ bool device_info(DeviceInfo *out)
         if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess) return false;
         if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return false;
         const size_t smem = smem_bytes(256, 3) > smem_bytes(128, 5) ? smem_bytes(256, 3) : smem_bytes(128, 5);
-        if (cudaFuncSetAttribute(score_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, score_fused, kThreads, smem) != cudaSuccess || per_sm < 1)
+        if (cudaFuncSetAttribute(score_fused<kGroupsNarrow>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(score_fused<kGroupsWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, score_fused<kGroupsNarrow>, threads_for(kGroupsNarrow), smem) != cudaSuccess || per_sm < 1)
+            return false;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, score_fused<kGroupsWide>, threads_for(kGroupsWide), smem) != cudaSuccess || per_sm < 1)
             return false;
         d.sms = sms;
         d.l2 = l2;
@@ -948,8 +951,9 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
     if (!make_map(&mapK, K, s.L, s.Hkv, kTile) || !make_map(&mapQ, Q, R, s.Hkv, P.Rbox)) return JQ_ERR_CUDA;
     if (Kwin) { if (!make_map(&mapW, Kwin, s.w, s.Hkv, kTile)) return JQ_ERR_CUDA; } else mapW = mapK;
 
+    const int groups = R > 128 ? kGroupsWide : kGroupsNarrow;
     int sms = dev.sms;
-    if (kGroups * sms > kSlots) sms = kSlots / kGroups;
+    if (groups * sms > kSlots) sms = kSlots / groups;
     // KV heads are scored in groups whose keys fit in a share of the L2, so that pass 2 finds them there.
     // Among the admissible group sizes, take the one that wastes the fewest CTA-tile slots.
     const long long head_bytes = (long long)s.L * kD * 2;
@@ -976,7 +980,7 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3((unsigned)threads_for(groups));
     cfg.dynamicSmemBytes = smem_bytes(P.Rbox, P.stages);
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
@@ -987,7 +991,9 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (cudaLaunchKernelEx(&cfg, score_fused, mapK, mapQ, mapW, P) != cudaSuccess) {
+    const cudaError_t err = groups == kGroupsWide ? cudaLaunchKernelEx(&cfg, score_fused<kGroupsWide>, mapK, mapQ, mapW, P)
+                                                  : cudaLaunchKernelEx(&cfg, score_fused<kGroupsNarrow>, mapK, mapQ, mapW, P);
+    if (err != cudaSuccess) {
         cudaGetLastError();
         return JQ_ERR_CUDA;
     }
