@@ -116,7 +116,8 @@ def test_select_bit_exact(Hkv, L, B, p, kind):
 
 
 # With many heads the selection kernel runs smaller clusters (4 or 2 CTAs per head instead of 8): same results.
-@pytest.mark.parametrize("Hkv,L,B,p", [(64, 4096, 512, 7), (160, 5000, 700, 7), (300, 1000, 100, 5), (148, 40000, 2048, 7)])
+@pytest.mark.parametrize("Hkv,L,B,p", [(64, 4096, 512, 7), (160, 5000, 700, 7), (300, 1000, 100, 5), (148, 40000, 2048, 7),
+                                       (200, 1, 1, 7), (200, 5, 9, 7), (100, 33, 10, 3), (256, 70001, 300, 1)])
 @pytest.mark.parametrize("kind", ["random", "ties"])
 def test_select_many_heads_bit_exact(Hkv, L, B, p, kind):
     rng = np.random.default_rng(Hkv * 7 + L)
