@@ -105,19 +105,20 @@ def run_reference(args):
     wl = pick_workload(args)
     K, V, Q, _ = W.make_layer(wl, 0)
     cores = os.cpu_count() or 1
-    # calibrate on a short prefix of one head, then size the per-step sample for a run of a few minutes
+    # calibrate on a short prefix with the heads a step runs (in parallel, as in a step), then size the per-step
+    # sample so that the whole run takes about two minutes
+    n = max(1, min(wl.Hkv, cores))
+    heads = list(range(n))
     Lc = max(wl.L // 16, 256)
     wc = wl.with_L(Lc)
-    tc = oracle_time_heads(wc, K[:, :Lc], V[:, :Lc], Q, [0])
-    per_head = tc * wl.L / Lc
+    tc = oracle_time_heads(wc, np.ascontiguousarray(K[:, :Lc]), np.ascontiguousarray(V[:, :Lc]), Q, heads)
+    per_step = tc * wl.L / Lc
     total = args.steps + args.warmup
-    n = max(1, min(wl.Hkv, cores))            # heads run in parallel: a step takes about one head's time
     Ls = wl.L
-    if total * per_head > 150.0:
-        Ls = max(2048, int(wl.L * 150.0 / (total * per_head)) // 128 * 128)
+    if total * per_step > 100.0:
+        Ls = max(2048, int(wl.L * 100.0 / (total * per_step)) // 128 * 128)
     ws = wl.with_L(Ls)
     Ks, Vs = np.ascontiguousarray(K[:, :Ls]), np.ascontiguousarray(V[:, :Ls])
-    heads = list(range(n))
     for _ in range(args.warmup):
         oracle_time_heads(ws, Ks, Vs, Q, heads)
     t = [oracle_time_heads(ws, Ks, Vs, Q, heads) for _ in range(args.steps)]
