@@ -194,7 +194,8 @@ jq_status jq_hit_rate(const int32_t *cur, const int32_t *ref, int Hkv, int ncur,
  * Kc, Vc: device, bf16 [Hkv, n, 128] (what jq_evict_layer wrote), 16-byte aligned.  q: device, bf16 [Hq, 128].
  * out: device, fp32 [Hq, 128], 16-byte aligned.  workspace: device, 16-byte aligned, at least
  * jq_decode_workspace_bytes(Hkv, Hq, n) bytes (0 for arguments the call would reject); no initialisation
- * needed, contents undefined afterwards.  Hq / Hkv <= 8.  Asynchronous on `stream`; two launches.
+ * needed, contents undefined afterwards.  Hq / Hkv <= 8.  Asynchronous on `stream`; one launch (and a memset
+ * of Hkv counters in the workspace).
  */
 size_t jq_decode_workspace_bytes(int Hkv, int Hq, int n);
 jq_status jq_decode_attention(const void *Kc, const void *Vc, const void *q, int Hkv, int Hq, int n, float *out,

@@ -1,10 +1,12 @@
 // One decoding step over the pruned cache (the step after the eviction pass: decoding continues with the
 // retained pairs only).  Single-position GQA attention, out[h] = softmax_j(q[h] . Kc[kv,j] / sqrt(d)) Vc[kv],
 // split over the keys:
-//   decode_partial  one CTA per (chunk of 64 keys, KV head): stages the chunk's K and V rows in shared memory
-//                   with coalesced 16-byte loads, computes the logits of every query head of the group, their
-//                   chunk-local softmax statistics (m, l) and the unnormalised weighted sum of the V rows.
-//   decode_combine  one CTA per query head: merges the chunks' (m, l, o) by the usual rescaling.
+//   one CTA per (chunk of 64 keys, KV head) stages the chunk's K and V rows in shared memory with coalesced
+//   16-byte loads, computes the logits of every query head of the group, their chunk-local softmax statistics
+//   (m, l) and the unnormalised weighted sum of the V rows, and writes them to the workspace; the CTA that
+//   finishes last for a KV head (a ticket counter per head, zeroed by the call) merges the chunks' (m, l, o)
+//   of the head's query heads by the usual rescaling, in chunk order, so the result does not depend on which
+//   CTA that is.
 // The work is a single read of the two compacted arrays (2 * Hkv * n * 256 bytes): bound by HBM/L2 latency at
 // these sizes, no tensor cores (a matrix-vector product per head).
 #include <cuda_bf16.h>
@@ -24,9 +26,10 @@ __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u 
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
 __global__ void __launch_bounds__(kDecThreads)
-decode_partial(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, const __nv_bfloat16 *__restrict__ q, int n,
-               int group, float scale_log2, float *__restrict__ part)
+decode_step(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, const __nv_bfloat16 *__restrict__ q, int n,
+            int group, float scale_log2, float *__restrict__ part, unsigned int *__restrict__ tickets, float *__restrict__ out)
 {
+    __shared__ int is_last;
     __shared__ __align__(16) __nv_bfloat16 Ks[kDecChunk * kKRow];
     __shared__ __align__(16) __nv_bfloat16 Vs[kDecChunk * kD];
     __shared__ float qs[kDecMaxGroup * kD];
@@ -104,24 +107,32 @@ decode_partial(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, const
             *(float2 *)(dst + 2 * cp) = make_float2(o0, o1);
         }
     }
-}
 
-__global__ void __launch_bounds__(kD)
-decode_combine(const float *__restrict__ part, int nsplit, int group, float *__restrict__ out)
-{
-    cudaGridDependencySynchronize();
-    const int h = blockIdx.x, kv = h / group, hg = h - kv * group, c = threadIdx.x;
-    float M = -INFINITY, Lsum = 0.f, O = 0.f;
-    for (int s = 0; s < nsplit; ++s) {
-        const float *src = part + ((size_t)(kv * nsplit + s) * group + hg) * kPartial;
-        const float m = src[0], l = src[1], o = src[2 + c];
-        const float Mn = fmaxf(M, m);
-        const float fa = exp2f(M - Mn), fb = exp2f(m - Mn);         // M = -inf only before the first chunk: fa = 0
-        Lsum = Lsum * fa + l * fb;
-        O = O * fa + o * fb;
-        M = Mn;
+    // the last CTA of the head to get here merges all chunks (release/acquire through the ticket)
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) is_last = (atomicAdd(&tickets[kv], 1u) == (unsigned)nsplit - 1u);
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    for (int item = tid; item < group * kD; item += kDecThreads) {
+        const int h = item / kD, c = item - h * kD;
+        // the head's maximum first, then plain sums in chunk order: no value depends on the previous load
+        const float *base = part + ((size_t)kv * nsplit * group + h) * kPartial;
+        const size_t step = (size_t)group * kPartial;
+        float M = -INFINITY;
+#pragma unroll 8
+        for (int sp = 0; sp < nsplit; ++sp) M = fmaxf(M, __ldcg(base + sp * step));
+        float Lsum = 0.f, O = 0.f;
+#pragma unroll 8
+        for (int sp = 0; sp < nsplit; ++sp) {
+            const float *src = base + sp * step;
+            const float f = exp2f(__ldcg(src) - M);
+            Lsum = fmaf(__ldcg(src + 1), f, Lsum);
+            O = fmaf(__ldcg(src + 2 + c), f, O);
+        }
+        out[((size_t)kv * group + h) * kD + c] = O / Lsum;
     }
-    out[(size_t)h * kD + c] = O / Lsum;
 }
 
 }  // namespace
@@ -131,7 +142,7 @@ extern "C" size_t jq_decode_workspace_bytes(int Hkv, int Hq, int n)
 {
     if (Hkv < 1 || Hq < 1 || Hq % Hkv || Hq / Hkv > jq::kDecMaxGroup || n < 1) return 0;
     const size_t nsplit = ((size_t)n + jq::kDecChunk - 1) / jq::kDecChunk;
-    return jq::align_up((size_t)Hq * nsplit * jq::kPartial * sizeof(float), 256);
+    return jq::align_up((size_t)Hq * nsplit * jq::kPartial * sizeof(float), 256) + jq::align_up((size_t)Hkv * sizeof(unsigned int), 256);
 }
 
 extern "C" jq_status jq_decode_attention(const void *Kc, const void *Vc, const void *q, int Hkv, int Hq, int n, float *out,
@@ -147,23 +158,10 @@ extern "C" jq_status jq_decode_attention(const void *Kc, const void *Vc, const v
     const int nsplit = (n + jq::kDecChunk - 1) / jq::kDecChunk;
     cudaStream_t st = (cudaStream_t)stream;
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)jq::kD);
-    jq::decode_partial<<<dim3((unsigned)nsplit, (unsigned)Hkv), jq::kDecThreads, 0, st>>>(
-        (const uint4 *)Kc, (const uint4 *)Vc, (const __nv_bfloat16 *)q, n, group, scale_log2, (float *)workspace);
-    jq::count_launch(1);
-    if (jq::check_launch() != JQ_OK) return JQ_ERR_CUDA;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)Hq);
-    cfg.blockDim = dim3(jq::kD);
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, jq::decode_combine, (const float *)workspace, nsplit, group, out) != cudaSuccess) {
-        cudaGetLastError();
-        return JQ_ERR_CUDA;
-    }
+    unsigned int *tickets = (unsigned int *)((char *)workspace + jq::align_up((size_t)Hq * nsplit * jq::kPartial * sizeof(float), 256));
+    if (cudaMemsetAsync(tickets, 0, (size_t)Hkv * sizeof(unsigned int), st) != cudaSuccess) return JQ_ERR_CUDA;
+    jq::decode_step<<<dim3((unsigned)nsplit, (unsigned)Hkv), jq::kDecThreads, 0, st>>>(
+        (const uint4 *)Kc, (const uint4 *)Vc, (const __nv_bfloat16 *)q, n, group, scale_log2, (float *)workspace, tickets, out);
     jq::count_launch(1);
     return jq::check_launch();
 }
