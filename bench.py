@@ -45,7 +45,9 @@ def parse():
     ap.add_argument("--seq", type=int, default=1, help="cfg4 only: which sequence of the ragged batch (0..3)")
     ap.add_argument("--budget", type=int, default=None)
     ap.add_argument("--layers", type=int, default=None, help="layer calls per step (default: the workload's)")
-    ap.add_argument("--call", default="stacked", choices=["stacked", "per-layer"])
+    ap.add_argument("--call", default="layers", choices=["layers", "stacked", "per-layer"],
+                    help="layers: one jq_evict_layers call per step on per-layer buffers (default); stacked: one jq_evict_layer call on "
+                         "layers concatenated along the KV-head axis; per-layer: one jq_evict_layer call per layer")
     ap.add_argument("--windowed", action="store_true",
                     help="window-inclusive scoring (jq_evict_layer_windowed): the causal keys of the query positions join the softmax")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -66,6 +68,7 @@ def config_of(wl, layers, distinct, call="per-layer"):
     return {"workload": wl.name, "L": wl.L, "Hkv": wl.Hkv, "Hq": wl.Hq, "d": wl.d, "w": wl.w,
             "budget": wl.budget, "pool": wl.pool, "layers_per_step": layers, "distinct_layers": distinct,
             "call": {"stacked": "one jq_evict_layer call per step, the layers stacked along the KV-head axis",
+                     "layers": "one jq_evict_layers call per step, every layer in buffers of its own",
                      "per-layer": "one jq_evict_layer call per layer",
                      "oracle": "the CPU oracle on a bounded sample of one layer"}[call],
             "l2": "inputs larger than L2 (K of one step: %.0f MiB)" % (distinct * wl.Hkv * wl.L * wl.d * 2 / 2**20)}
@@ -249,7 +252,8 @@ def run_ours(args):
     # the layers of the cache stacked along the KV-head axis (a layer repeated in the workload is copied, so
     # that every layer of the step has memory of its own)
     sS = jq.shape(wl.Hkv * layers, wl.Hq * layers, wl.L, wl.w, wl.budget, wl.pool, wl.d)
-    if args.call == "stacked":
+    one_call = args.call in ("stacked", "layers")
+    if one_call:
         order = [i % distinct for i in range(layers)]
         KS = torch.cat([Ks[j] for j in order], 0)
         VS = torch.cat([Vs[j] for j in order], 0)
@@ -266,7 +270,21 @@ def run_ours(args):
         else:
             jq.evict_layer(KS, VS, QS, sS, KoS, VoS, idxS, wsS, stream=stream)
 
-    step = step_stacked if args.call == "stacked" else step_per_layer
+    if args.call == "layers":
+        # the layers as a cache holds them: a tensor each (a layer the workload repeats gets a copy of its own)
+        seen = set()
+        KL, VL, QL = [], [], []
+        for j in order:
+            KL.append(Ks[j] if j not in seen else Ks[j].clone())
+            VL.append(Vs[j] if j not in seen else Vs[j].clone())
+            QL.append(Qs[j] if j not in seen else Qs[j].clone())
+            seen.add(j)
+        wsL = jq.new_layers_workspace(s, layers)
+
+    def step_layers():
+        jq.evict_layers(KL, VL, QL, s, KoS, VoS, idxS, wsL, stream=stream)
+
+    step = {"stacked": step_stacked, "layers": step_layers, "per-layer": step_per_layer}[args.call]
 
     def barrier():
         if world > 1:
@@ -287,8 +305,8 @@ def run_ours(args):
     ms = e0.elapsed_time(e1)
     launches = jq.launch_count() - n0
     assert jq.last_device_status(ws) == jq.JQ_OK, "device status not ok"
-    if args.call == "stacked":
-        assert jq.last_device_status(wsS) == jq.JQ_OK, "device status not ok"
+    if one_call:
+        assert jq.last_device_status(wsL if args.call == "layers" else wsS) == jq.JQ_OK, "device status not ok"
         # the same work as one call per layer, for comparison (and its results must be the same bits)
         for _ in range(3):
             step_per_layer()
@@ -324,7 +342,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         return ev[0].elapsed_time(ev[1]) / nb
 
-    if args.call == "stacked":
+    if one_call:
         scoresS = torch.empty((sS.Hkv, wl.L), dtype=torch.float32, device="cuda")
         nb = 4
         if args.windowed:
@@ -421,7 +439,7 @@ def run_ours(args):
         peak, peak_src = 6650.0, "fallback"
     # dominant kernel: score_fused (jq_score, both passes); algorithmic bytes = two reads of K.  One launch
     # covers one layer, or all stacked layers of the step.
-    per_launch = layers if args.call == "stacked" else 1
+    per_launch = layers if one_call else 1
     score_bytes = 2 * wl.Hkv * wl.L * wl.d * 2 * per_launch
     ms_launch = float(stage_ms[0]) * per_launch
     achieved = score_bytes / (ms_launch * 1e-3) / 1e9

@@ -165,6 +165,22 @@ jq_status jq_evict_layer(const void *K, const void *V, const void *Qwin, const j
                          jq_stream_t stream);
 
 /*
+ * jq_evict_layer over nlayers layers of one shape whose K, V and Qwin live in buffers of their own (the usual
+ * layout of a cache): one call, two launches, the same results as nlayers calls of jq_evict_layer.  (Heads are
+ * independent units of the pass, so the layers are scored and selected as nlayers x Hkv heads; this is the
+ * fastest way to evict a whole cache after a prefill.)
+ * K, V, Qwin: HOST arrays of nlayers DEVICE pointers, each as jq_evict_layer takes it for `layer`; read before
+ * the call returns.  Kout, Vout: device, bf16 [nlayers * Hkv, nkeep, d]; kept_idx: device [nlayers * Hkv, nkeep]
+ * (layer l at rows l * Hkv ...).  ws: as for jq_evict_layer but of jq_layers_workspace_bytes(layer, nlayers)
+ * bytes (0 for arguments the call would reject), its first 256 bytes initialised by jq_workspace_init.
+ * nlayers <= 128 and nlayers * Hkv <= 65535, else JQ_ERR_UNSUPPORTED.
+ */
+size_t jq_layers_workspace_bytes(const jq_shape *layer, int nlayers);
+jq_status jq_evict_layers(const void *const *K, const void *const *V, const void *const *Qwin, int nlayers,
+                          const jq_shape *layer, void *Kout, void *Vout, int32_t *kept_idx, void *ws, size_t ws_bytes,
+                          jq_stream_t stream);
+
+/*
  * jq_evict_layer for callers whose tensors live in HOST memory (pinned memory gives asynchronous
  * copies).  hK, hV, hQwin are copied to the device, the layer is evicted, and hKout, hVout,
  * hkept_idx are copied back, all on `stream`; the call returns without synchronising.  When hV is

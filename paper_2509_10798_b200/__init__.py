@@ -18,7 +18,7 @@ EXPORTS = (
     "jq_score_fma", "jq_select_topk", "jq_compact_kv", "jq_evict_layer", "jq_host_call_bytes",
     "jq_evict_layer_host", "jq_last_device_status", "jq_launch_count", "jq_status_string",
     "jq_score_static", "jq_score_windowed", "jq_evict_layer_windowed", "jq_hit_rate",
-    "jq_decode_workspace_bytes", "jq_decode_attention",
+    "jq_decode_workspace_bytes", "jq_decode_attention", "jq_layers_workspace_bytes", "jq_evict_layers",
 )
 
 
@@ -60,6 +60,9 @@ def lib():
         L.jq_decode_workspace_bytes.argtypes = [ci, ci, ci]
         L.jq_decode_workspace_bytes.restype = ctypes.c_size_t
         L.jq_decode_attention.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, ctypes.c_size_t, vp]
+        L.jq_layers_workspace_bytes.argtypes = [sp, ci]
+        L.jq_layers_workspace_bytes.restype = ctypes.c_size_t
+        L.jq_evict_layers.argtypes = [vp, vp, vp, ci, sp, vp, vp, vp, vp, sz, vp]
         L.jq_hit_rate.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         L.jq_score_windowed.argtypes = [vp, vp, vp, sp, vp, vp, sz, vp]
         L.jq_evict_layer_windowed.argtypes = [vp, vp, vp, vp, sp, vp, vp, vp, vp, sz, vp]
@@ -187,6 +190,30 @@ def evict_layer_host(hK, hV, hQwin, s, hKout, hVout, hkept_idx, dev_buf, stream=
     _raise("jq_evict_layer_host",
            lib().jq_evict_layer_host(_ptr(hK), _ptr(hV), _ptr(hQwin), ctypes.byref(s), _ptr(hKout), _ptr(hVout),
                                      _ptr(hkept_idx), _ptr(dev_buf), dev_buf.numel(), _stream(stream)))
+
+
+def layers_workspace_bytes(s, nlayers):
+    return int(lib().jq_layers_workspace_bytes(ctypes.byref(s), int(nlayers)))
+
+
+def new_layers_workspace(s, nlayers, device="cuda", stream=None):
+    """Allocates and initialises a workspace tensor (uint8) for evict_layers on nlayers layers of shape `s`."""
+    torch = _torch()
+    n = layers_workspace_bytes(s, nlayers)
+    if n == 0:
+        raise JqError("jq_layers_workspace_bytes", check_shape(s) or JQ_ERR_UNSUPPORTED)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    _raise("jq_workspace_init", lib().jq_workspace_init(_ptr(ws), ws.numel(), _stream(stream)))
+    return ws
+
+
+def evict_layers(Ks, Vs, Qwins, s, Kout, Vout, kept_idx, ws, stream=None):
+    """jq_evict_layers: Ks, Vs, Qwins are lists of per-layer CUDA tensors of shape `s`; the outputs are stacked."""
+    n = len(Ks)
+    arr = lambda ts: (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
+    _raise("jq_evict_layers",
+           lib().jq_evict_layers(arr(Ks), arr(Vs), arr(Qwins), n, ctypes.byref(s), _ptr(Kout), _ptr(Vout), _ptr(kept_idx),
+                                 _ptr(ws), ws.numel(), _stream(stream)))
 
 
 def decode_workspace_bytes(Hkv, Hq, n):

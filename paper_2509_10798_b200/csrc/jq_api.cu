@@ -149,6 +149,58 @@ jq_status jq_evict_layer(const void *K, const void *V, const void *Qwin, const j
     return launch_select(w.scores, *s, kept_idx, nullptr, w, st, K, V, Kout, Vout);   // selects, then copies the kept rows
 }
 
+// The shape of nlayers layers of shape `layer` stacked along the KV-head axis.
+static jq_status stacked_shape(const jq_shape *layer, int nlayers, jq_shape *out)
+{
+    jq_status rc = check_shape(layer);
+    if (rc != JQ_OK) return rc;
+    if (nlayers < 1) return JQ_ERR_INVALID_ARG;
+    if (nlayers > kMaxLayers) return JQ_ERR_UNSUPPORTED;
+    *out = *layer;
+    out->Hkv = layer->Hkv * nlayers;
+    out->Hq = layer->Hq * nlayers;
+    return check_shape(out);
+}
+
+size_t jq_layers_workspace_bytes(const jq_shape *layer, int nlayers)
+{
+    jq_shape S;
+    if (stacked_shape(layer, nlayers, &S) != JQ_OK) return 0;
+    return carve(nullptr, S).bytes + layer_tables_bytes(nlayers);
+}
+
+jq_status jq_evict_layers(const void *const *K, const void *const *V, const void *const *Qwin, int nlayers,
+                          const jq_shape *layer, void *Kout, void *Vout, int32_t *kept_idx, void *ws, size_t ws_bytes,
+                          jq_stream_t stream)
+{
+    jq_shape S;
+    jq_status rc = stacked_shape(layer, nlayers, &S);
+    if (rc != JQ_OK) return rc;
+    if (!K || !V || !Qwin || !aligned16(Kout) || !aligned16(Vout) || !aligned16(kept_idx)) return JQ_ERR_INVALID_ARG;
+    for (int l = 0; l < nlayers; ++l)
+        if (!aligned16(K[l]) || !aligned16(V[l]) || !aligned16(Qwin[l])) return JQ_ERR_INVALID_ARG;
+    if (!aligned16(ws) || ((uintptr_t)ws & 255u)) return JQ_ERR_INVALID_ARG;
+    const Workspace w = carve(ws, S);
+    if (ws_bytes < w.bytes + layer_tables_bytes(nlayers)) return JQ_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    // tables behind the workspace proper: tensor maps, then the K and the V base pointers
+    char *tab = (char *)ws + w.bytes;
+    const size_t maps_bytes = align_up((size_t)nlayers * 2 * kTensorMapBytes, 256), ptr_bytes = align_up((size_t)nlayers * sizeof(void *), 256);
+    alignas(64) unsigned char host_maps[kMaxLayers * 2 * kTensorMapBytes];
+    if (!build_layer_maps(K, Qwin, nlayers, *layer, host_maps)) return JQ_ERR_CUDA;
+    // (copies from pageable host memory are staged before the call returns, so the sources may live on this stack)
+    if (cudaMemcpyAsync(tab, host_maps, (size_t)nlayers * 2 * kTensorMapBytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
+    if (cudaMemcpyAsync(tab + maps_bytes, K, (size_t)nlayers * sizeof(void *), cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
+    if (cudaMemcpyAsync(tab + maps_bytes + ptr_bytes, V, (size_t)nlayers * sizeof(void *), cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
+    LayerTables t;
+    t.maps = tab;
+    t.K = (const void *const *)(tab + maps_bytes);
+    t.V = (const void *const *)(tab + maps_bytes + ptr_bytes);
+    t.hpl = layer->Hkv;
+    if ((rc = launch_score_tc(K[0], Qwin[0], S, w.scores, w, st, nullptr, &t)) != JQ_OK) return rc;
+    return launch_select(w.scores, S, kept_idx, nullptr, w, st, nullptr, nullptr, Kout, Vout, &t);
+}
+
 size_t jq_host_call_bytes(const jq_shape *s)
 {
     if (check_shape(s) != JQ_OK) return 0;

@@ -49,6 +49,23 @@ static inline Workspace carve(void *base, const jq_shape &s)
     return w;
 }
 
+// Layers of equal shape living in buffers of their own (jq_evict_layers): tables in device memory, behind the
+// workspace proper.  KV head kv of the stacked numbering belongs to layer kv / hpl and is head kv % hpl of it.
+constexpr int kMaxLayers = 128;
+constexpr size_t kTensorMapBytes = 128;
+struct LayerTables {
+    const void *maps = nullptr;          // device: [nlayers][2] TMA tensor maps (K, Qwin)
+    const void *const *K = nullptr;      // device: [nlayers] base of K
+    const void *const *V = nullptr;      // device: [nlayers] base of V
+    int hpl = 0;                         // KV heads per layer (0: no tables, one buffer)
+};
+static inline size_t layer_tables_bytes(int nlayers)
+{
+    return align_up((size_t)nlayers * 2 * kTensorMapBytes, 256) + 2 * align_up((size_t)nlayers * sizeof(void *), 256);
+}
+// Fills host_maps ([nlayers][2] tensor maps) for K[l] [hpl][L][128] and Qwin[l] [hpl][R][128].
+bool build_layer_maps(const void *const *K, const void *const *Qwin, int nlayers, const jq_shape &layer, void *host_maps);
+
 // Host-side bookkeeping.
 void count_launch(int n = 1);
 jq_status check_launch();   // cudaGetLastError -> JQ_OK / JQ_ERR_CUDA
@@ -57,12 +74,14 @@ jq_status check_launch();   // cudaGetLastError -> JQ_OK / JQ_ERR_CUDA
 jq_status launch_score_fma(const void *K, const void *Q, const jq_shape &s, float *scores,
                            const Workspace &w, cudaStream_t st);
 // Kwin, when not null: keys [Hkv][w][128] of the query positions themselves (window-inclusive softmax).
+// With tables (s is then the stacked shape, K and Q those of the first layer) the tiles come from the layers' own buffers.
 jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float *scores,
-                          const Workspace &w, cudaStream_t st, const void *Kwin = nullptr);
+                          const Workspace &w, cudaStream_t st, const void *Kwin = nullptr,
+                          const LayerTables *tables = nullptr);
 // With K, V, Kout, Vout given, the kernel also copies the kept rows (the fused layer path).
 jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, float *pooled,
                         const Workspace &w, cudaStream_t st, const void *K = nullptr, const void *V = nullptr,
-                        void *Kout = nullptr, void *Vout = nullptr);
+                        void *Kout = nullptr, void *Vout = nullptr, const LayerTables *tables = nullptr);
 jq_status launch_gather(const void *K, const void *V, const int32_t *idx, const jq_shape &s,
                         void *Kout, void *Vout, cudaStream_t st);
 

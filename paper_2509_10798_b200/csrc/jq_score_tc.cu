@@ -122,6 +122,8 @@ struct Params {
     int *status;             // status block (kStatusWords ints)
     int wtile;               // 1 in window-inclusive mode: every head has one more tile, the last, holding the w window keys
     int w;                   // soft-token queries per query head
+    const CUtensorMap *maps; // not null: [layers][2] tensor maps (K, Qwin) of layers in buffers of their own, hpl KV heads each
+    int hpl;
 #ifdef JQ_TRACE
     long long *trace;
 #endif
@@ -451,6 +453,8 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             TR_DECL;
             uint32_t st = 0, ph = 0, qn = 0;                  // ring stage and its phase; query loads so far
             int prev_kv = -1;
+            const CUtensorMap *head_mapK = &mapK, *head_mapQ = &mapQ;   // maps and head coordinate of the current KV head
+            int head_c2 = 0;
             bool ok = true;
 #pragma unroll 1
             for (int s = 0; s < nseg && ok; ++s) {
@@ -461,11 +465,15 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                 for (int n = 0; n < ntiles; ++n, walk(pass, tph, kv, tt)) {
                     TR_ADD(2);
                     if (kv != prev_kv) {
+                        if (P.maps) {                         // the head's layer has tensor maps of its own
+                            const int lay = kv / P.hpl;
+                            head_mapK = P.maps + 2 * lay; head_mapQ = head_mapK + 1; head_c2 = kv - lay * P.hpl;
+                        } else head_c2 = kv;
                         const uint32_t qb = qn & 1;
                         if (!mbar_wait(&ctl->q_empty[qb], ((qn >> 1) & 1) ^ 1, ctl, status, kSleepLong)) { ok = false; break; }
                         mbar_expect_tx(&ctl->q_full[qb], q_bytes);
-                        tma_load_3d(qbuf + (size_t)qb * q_bytes, &mapQ, &ctl->q_full[qb], 0, 0, kv);
-                        tma_load_3d(qbuf + (size_t)qb * q_bytes + q_bytes / 2, &mapQ, &ctl->q_full[qb], 64, 0, kv);
+                        tma_load_3d(qbuf + (size_t)qb * q_bytes, head_mapQ, &ctl->q_full[qb], 0, 0, head_c2);
+                        tma_load_3d(qbuf + (size_t)qb * q_bytes + q_bytes / 2, head_mapQ, &ctl->q_full[qb], 64, 0, head_c2);
                         prev_kv = kv; ++qn;
                         TR_ADD(0);
                     }
@@ -475,10 +483,10 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     // window-inclusive mode: in pass 1 the last tile of a head is its window keys (rows past w read as
                     // zero); in pass 2 that tile lies past the prefix, reads as zero and its scores are never stored
                     const bool wt = P.wtile && pass == 1 && tt == tph - 1;
-                    const CUtensorMap *map = wt ? &mapW : &mapK;
+                    const CUtensorMap *map = wt ? &mapW : head_mapK;
                     const int j0 = wt ? 0 : tt * kTile;
-                    tma_load_3d(kbuf + (size_t)st * kStageBytes, map, &ctl->full[st], 0, j0, kv);
-                    tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, map, &ctl->full[st], 64, j0, kv);
+                    tma_load_3d(kbuf + (size_t)st * kStageBytes, map, &ctl->full[st], 0, j0, head_c2);
+                    tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, map, &ctl->full[st], 64, j0, head_c2);
                     if (++st == (uint32_t)stages) { st = 0; ph ^= 1; }
                 }
             }
@@ -926,8 +934,19 @@ static long long *g_trace = nullptr;
 extern "C" void jq_debug_set_trace(long long *p) { g_trace = p; }   // [grid][32 warps][16] int64, device memory
 #endif
 
+bool build_layer_maps(const void *const *K, const void *const *Qwin, int nlayers, const jq_shape &layer, void *host_maps)
+{
+    static_assert(sizeof(CUtensorMap) == kTensorMapBytes, "tensor map size");
+    CUtensorMap *m = (CUtensorMap *)host_maps;
+    const int R = layer.group * layer.w;
+    for (int l = 0; l < nlayers; ++l)
+        if (!make_map(&m[2 * l], K[l], layer.L, layer.Hkv, kTile) || !make_map(&m[2 * l + 1], Qwin[l], R, layer.Hkv, R <= 128 ? 128 : 256))
+            return false;
+    return true;
+}
+
 jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float *scores, const Workspace &w,
-                          cudaStream_t st, const void *Kwin)
+                          cudaStream_t st, const void *Kwin, const LayerTables *tables)
 {
     DeviceInfo dev;
     if (!device_info(&dev)) return JQ_ERR_CUDA;
@@ -944,11 +963,14 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
     P.c = 1.4426950408889634f / sqrtf((float)s.d);
     P.part = w.part; P.Mrow = w.Mrow; P.scores = scores; P.status = w.status;
     P.w = s.w;
+    P.maps = tables ? (const CUtensorMap *)tables->maps : nullptr;
+    P.hpl = tables ? tables->hpl : 0;
 #ifdef JQ_TRACE
     P.trace = g_trace;
 #endif
     CUtensorMap mapK, mapQ, mapW;
-    if (!make_map(&mapK, K, s.L, s.Hkv, kTile) || !make_map(&mapQ, Q, R, s.Hkv, P.Rbox)) return JQ_ERR_CUDA;
+    const int map_heads = tables ? tables->hpl : s.Hkv;   // with tables these two describe the first layer and are not used
+    if (!make_map(&mapK, K, s.L, map_heads, kTile) || !make_map(&mapQ, Q, R, map_heads, P.Rbox)) return JQ_ERR_CUDA;
     if (Kwin) { if (!make_map(&mapW, Kwin, s.w, s.Hkv, kTile)) return JQ_ERR_CUDA; } else mapW = mapK;
 
     const int groups = R > 128 ? kGroupsWide : kGroupsNarrow;

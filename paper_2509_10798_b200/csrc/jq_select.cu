@@ -100,16 +100,19 @@ __device__ __forceinline__ void find_digit(const uint32_t *g, int krem, SelCtl &
 // r-th share of them, once every index of the head has been written.
 template <int CL>
 __device__ __forceinline__ void copy_kept_rows(cg::cluster_group &cluster, const int32_t *out, int kv, int L, int nkeep,
-                                               const uint4 *Kin, const uint4 *Vin, uint4 *Kout, uint4 *Vout)
+                                               const uint4 *Kin, const uint4 *Vin, uint4 *Kout, uint4 *Vout,
+                                               const uint4 *const *Ktab, const uint4 *const *Vtab, int hpl)
 {
     __threadfence();
     cluster.sync();
+    int kv_in = kv;                       // head index within the buffer the rows come from
+    if (Ktab) { const int lay = kv / hpl; Kin = Ktab[lay]; Vin = Vtab[lay]; kv_in = kv - lay * hpl; }
     const int rank = (int)cluster.block_rank();
     const int r0 = (int)((long long)rank * nkeep / CL), r1 = (int)((long long)(rank + 1) * nkeep / CL);
     const int lane16 = threadIdx.x & 15;
     for (int t = r0 + (int)(threadIdx.x >> 4); t < r1; t += kSelThreads / 16) {
         const int j = min(max(__ldcg(out + t), 0), L - 1);
-        const size_t src = ((size_t)kv * L + j) * 16 + lane16, dst = ((size_t)kv * nkeep + t) * 16 + lane16;
+        const size_t src = ((size_t)kv_in * L + j) * 16 + lane16, dst = ((size_t)kv * nkeep + t) * 16 + lane16;
         Kout[dst] = Kin[src];
         Vout[dst] = Vin[src];
     }
@@ -121,7 +124,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(kSelThreads, 2)
 select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, int32_t *__restrict__ idx,
                float *__restrict__ pooled, uint32_t *__restrict__ gkeys, int chunk, int keys_in_smem, int raw_tile,
                const uint4 *__restrict__ Kin, const uint4 *__restrict__ Vin, uint4 *__restrict__ Kout,
-               uint4 *__restrict__ Vout)
+               uint4 *__restrict__ Vout, const uint4 *const *__restrict__ Ktab, const uint4 *const *__restrict__ Vtab, int hpl)
 {
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
@@ -222,7 +225,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     }
     if (nkeep >= L) {   // everything is kept (uniform over the cluster; no cluster traffic yet)
         for (int e = tid; e < n; e += kSelThreads) out[j0 + e] = j0 + e;
-        if (Kin) copy_kept_rows<CL>(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout);
+        if (Kin || Ktab) copy_kept_rows<CL>(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout, Ktab, Vtab, hpl);
         return;
     }
     for (int i = tid; i < 3 * kBins; i += kSelThreads) ghist[i] = 0;
@@ -376,7 +379,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         gt_before += __popc(bg);
         eq_before += __popc(be);
     }
-    if (Kin) copy_kept_rows<CL>(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout);
+    if (Kin || Ktab) copy_kept_rows<CL>(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout, Ktab, Vtab, hpl);
 }
 
 // Shared memory of a CTA whose cluster has `cl` CTAs, the share of the head it holds, and whether its keys stay on chip.
@@ -418,7 +421,8 @@ SelPlan choose_plan(int Hkv, int L, int sms)
 
 template <int CL>
 jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape &s, int nkeep, int32_t *idx, float *pooled,
-                           const Workspace &w, cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout, int dev)
+                           const Workspace &w, cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout, int dev,
+                           const LayerTables *tables)
 {
     static bool attr_done[64] = {};
     if (!attr_done[dev]) {
@@ -440,7 +444,9 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (cudaLaunchKernelEx(&cfg, select_cluster<CL>, scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, w.keys, p.chunk,
-                           p.in_smem, p.raw_tile, (const uint4 *)K, (const uint4 *)V, (uint4 *)Kout, (uint4 *)Vout) != cudaSuccess) {
+                           p.in_smem, p.raw_tile, (const uint4 *)K, (const uint4 *)V, (uint4 *)Kout, (uint4 *)Vout,
+                           (const uint4 *const *)(tables ? tables->K : nullptr), (const uint4 *const *)(tables ? tables->V : nullptr),
+                           tables ? tables->hpl : 0) != cudaSuccess) {
         cudaGetLastError();
         return JQ_ERR_CUDA;
     }
@@ -451,7 +457,8 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
 }  // namespace
 
 jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, float *pooled,
-                        const Workspace &w, cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout)
+                        const Workspace &w, cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout,
+                        const LayerTables *tables)
 {
     const int nkeep = s.budget < s.L ? s.budget : s.L;
     static int sms[64] = {};
@@ -460,9 +467,9 @@ jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, fl
     if (!sms[dev] && cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return JQ_ERR_CUDA;
     const SelPlan p = choose_plan(s.Hkv, s.L, sms[dev]);
     switch (p.cl) {
-    case 2: return launch_select_cl<2>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev);
-    case 4: return launch_select_cl<4>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev);
-    default: return launch_select_cl<8>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev);
+    case 2: return launch_select_cl<2>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables);
+    case 4: return launch_select_cl<4>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables);
+    default: return launch_select_cl<8>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables);
     }
 }
 

@@ -81,6 +81,14 @@ def test_pointer_errors_are_caught_on_the_host():
     assert lib.jq_decode_attention(a, a, a, 1, 16, 100, a, a, 1 << 20, None) == jq.JQ_ERR_UNSUPPORTED     # group > 8
     assert lib.jq_decode_attention(a, a, a, 2, 8, 100, a, a, 16, None) == jq.JQ_ERR_WORKSPACE
     assert jq.decode_workspace_bytes(2, 8, 100) >= 8 * 2 * 130 * 4 and jq.decode_workspace_bytes(2, 7, 100) == 0
+    ptrs = (ctypes.c_void_p * 2)(0x1000, 0x2000)
+    assert lib.jq_evict_layers(ptrs, ptrs, ptrs, 2, ref, a, a, a, a, 16, None) == jq.JQ_ERR_WORKSPACE
+    assert lib.jq_evict_layers(ptrs, ptrs, ptrs, 0, ref, a, a, a, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
+    assert lib.jq_evict_layers(ptrs, ptrs, ptrs, 129, ref, a, a, a, a, 1 << 40, None) == jq.JQ_ERR_UNSUPPORTED
+    assert lib.jq_evict_layers(None, ptrs, ptrs, 2, ref, a, a, a, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
+    odd_ptrs = (ctypes.c_void_p * 2)(0x1000, 0x2008)
+    assert lib.jq_evict_layers(odd_ptrs, ptrs, ptrs, 2, ref, a, a, a, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
+    assert jq.layers_workspace_bytes(s, 2) > jq.workspace_bytes(jq.shape(4, 16, 2048, 16, 256)) and jq.layers_workspace_bytes(s, 0) == 0
     assert lib.jq_hit_rate(a, a, 0, 4, 4, a, None) == jq.JQ_ERR_INVALID_ARG
     assert lib.jq_last_device_status(None, None) == jq.JQ_ERR_INVALID_ARG
     assert jq.status_string(jq.JQ_ERR_TIMEOUT) and jq.status_string(99)

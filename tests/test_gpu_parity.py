@@ -481,3 +481,36 @@ def test_evict_then_decode_then_evict_again():
     K2, V2, Q2, _ = W.make_layer(small_wl(2, 4, 16, 200, 400), layer=1)
     Kn, Vn = np.concatenate([Kc, K2], axis=1), np.concatenate([Vc, V2], axis=1)
     run_e2e(small_wl(2, 4, 16, Kn.shape[1], 400), Kn, Vn, Q2)
+
+
+# ------------------------------------------------------------------ several layers in buffers of their own, one call
+
+@pytest.mark.parametrize("Hkv,g,w,L,B,nl", [(2, 4, 16, 3000, 400, 5), (2, 4, 64, 2049, 300, 3), (8, 4, 32, 8192, 1024, 32),
+                                            (1, 1, 1, 5, 3, 2), (3, 2, 8, 130, 1000, 7)])
+def test_evict_layers_matches_calls_per_layer(Hkv, g, w, L, B, nl):
+    wl = small_wl(Hkv, g, w, L, B)
+    s = shape_of(wl)
+    layers = [W.make_layer(wl, layer=i) for i in range(nl)]
+    pad = torch.empty(1000, dtype=torch.uint8, device="cuda")     # keeps the layers' buffers from being neighbours
+    dK, dV, dQ = [], [], []
+    for K, V, Q, _ in layers:
+        dK.append(dev_bf16(K)); dV.append(dev_bf16(V)); dQ.append(dev_bf16(Q))
+        pad = torch.empty(pad.numel() + 4096, dtype=torch.uint8, device="cuda")
+    nkeep = wl.nkeep
+    Ko = torch.zeros((nl * Hkv, nkeep, 128), dtype=torch.bfloat16, device="cuda")
+    Vo = torch.zeros_like(Ko)
+    idx = torch.full((nl * Hkv, nkeep), -1, dtype=torch.int32, device="cuda")
+    ws = jq.new_layers_workspace(s, nl)
+    for _ in range(2):                                            # twice: the workspace is reusable as it is left
+        Ko.zero_(); Vo.zero_(); idx.fill_(-1)
+        jq.evict_layers(dK, dV, dQ, s, Ko, Vo, idx, ws)
+        assert jq.last_device_status(ws) == jq.JQ_OK
+        gK, gV, gi = host_bits(Ko), host_bits(Vo), idx.cpu().numpy()
+        for i, (K, V, Q, _) in enumerate(layers):
+            wK, wV, wi = gpu_evict(K, V, Q, s)
+            sl = slice(i * Hkv, (i + 1) * Hkv)
+            assert np.array_equal(gi[sl], wi) and np.array_equal(gK[sl], wK) and np.array_equal(gV[sl], wV)
+    # and one layer of it against the oracle, under the end-to-end rule
+    K, V, Q, _ = layers[nl - 1]
+    pooled = oracle.pool(oracle.score(K, Q), wl.pool)
+    assert_kept_sets_agree(gi[(nl - 1) * Hkv:], oracle.select(pooled, wl.budget), pooled, nkeep)
