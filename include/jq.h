@@ -173,7 +173,9 @@ jq_status jq_evict_layer(const void *K, const void *V, const void *Qwin, const j
  * the call returns.  Kout, Vout: device, bf16 [nlayers * Hkv, nkeep, d]; kept_idx: device [nlayers * Hkv, nkeep]
  * (layer l at rows l * Hkv ...).  ws: as for jq_evict_layer but of jq_layers_workspace_bytes(layer, nlayers)
  * bytes (0 for arguments the call would reject), its first 256 bytes initialised by jq_workspace_init.
- * nlayers <= 128 and nlayers * Hkv <= 65535, else JQ_ERR_UNSUPPORTED.
+ * nlayers <= 128 and nlayers * Hkv <= 65535, else JQ_ERR_UNSUPPORTED.  The call copies its small tables (tensor
+ * maps, base pointers) from ordinary host memory to the device on `stream`, so it cannot be captured into a
+ * CUDA graph; capture nlayers calls of jq_evict_layer, or one on a stacked tensor, instead.
  */
 size_t jq_layers_workspace_bytes(const jq_shape *layer, int nlayers);
 jq_status jq_evict_layers(const void *const *K, const void *const *V, const void *const *Qwin, int nlayers,
