@@ -252,6 +252,8 @@ def run_ours(args):
     # the layers of the cache stacked along the KV-head axis (a layer repeated in the workload is copied, so
     # that every layer of the step has memory of its own)
     sS = jq.shape(wl.Hkv * layers, wl.Hq * layers, wl.L, wl.w, wl.budget, wl.pool, wl.d)
+    if args.windowed and args.call == "layers":
+        args.call = "stacked"          # the window-inclusive entry point takes one (stacked) tensor per operand
     one_call = args.call in ("stacked", "layers")
     if one_call:
         order = [i % distinct for i in range(layers)]
