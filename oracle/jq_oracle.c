@@ -7,29 +7,28 @@
  *
  * What it computes, with the passage of the paper each step follows:
  *
- *   score   Eq. 3 ("attention of every soft token with respect to the prompt,
- *           combined over the token dimension") and the inference section
- *           ("the attention map of the soft tokens over the input decides what
- *           is kept"):  for KV head kv, for every query head h of its GQA
- *           group and every soft token i,
+ *   score   Eq. 3 (the attention of each soft token over the prompt's keys,
+ *           combined over the soft tokens) as the inference section uses it
+ *           to rank the prompt's key-value pairs:  for KV head kv, for every
+ *           query head h of its GQA group and every soft token i,
  *               s_j = (Q[h,i,:] . K[kv,j,:]) / sqrt(d)        j = 0..L-1
  *               P_j = exp(s_j - max_j s) / sum_j exp(s_j - max_j s)
  *               score[kv,j] += P_j
  *           The softmax runs over the L prefix keys only; the sum (not the
  *           1/n mean of Eq. 3) is taken, a monotone rescale that leaves the
  *           kept set unchanged.
- *   pool    Experimental-setting paragraph (all methods share one "pooling
- *           configuration"): max over a centred window of odd width p, stride
+ *   pool    Experimental-setting paragraph (one pooling set-up shared by all
+ *           compared methods): max over a centred window of odd width p, stride
  *           1, same length, taps outside [0,L) ignored.
- *   select  Inference section ("retain the pairs with the top-k highest
- *           scores, discard the rest"): the nkeep = min(budget, L) largest
+ *   select  Inference section (only the k best-scored pairs stay in the
+ *           cache): the nkeep = min(budget, L) largest
  *           pooled values per KV head; equal values are ordered by lower
  *           index first; the kept indices are returned ascending.
  *   compact Inference section (the pruned cache is what decoding continues
  *           with): rows K[kv,idx,:], V[kv,idx,:] copied bit for bit.
  *
  * (jq_oracle_decode_attention is the step after the pass: one decoding step's attention over the pruned
- * cache, the inference section's "decoding continues with the retained pairs"; pinned against a library
+ * cache (inference section: generation goes on from the pruned cache); pinned against a library
  * softmax and matrix product, the q = 0 mean, a dominant key and n = 1.)
  *
  * (jq_oracle_score_windowed is the window-inclusive variant of the scores; its pins are a library

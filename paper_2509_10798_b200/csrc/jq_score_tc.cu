@@ -1,16 +1,15 @@
 // Tensor-core scoring for sm_100a: Eq. 3 in two streaming passes over K, ONE persistent kernel per call.
 //
 // The grid is one CTA per SM, launched cooperatively (all CTAs are resident, so they may wait on one
-// another).  A CTA is warp-specialised:
+// another).  A CTA is warp-specialised; the first four warps run the machinery:
 //   warp 0        TMA producer: K tiles of 128 keys (two 64-column halves, 128-byte swizzle) into a ring of
 //                 shared-memory stages; the query rows of a KV head into one of two stationary buffers;
 //   warp 1        issues tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory; the warp stays converged, one
 //                 elected lane issues) and owns the TMEM allocation;
-//   warps 2..     kGroups epilogue groups of 128 threads (3 for up to 128 query rows per KV head, 4 above).
-//                 Accumulator block u (128 TMEM lanes x 128 columns) sits in slot u % 4 and is taken by
-//                 group u % kGroups, 32 columns at a time;
-//   then          one warp that merges the per-warp partial row statistics of pass 1 across the grid,
-//                 and one that stages the merged row normalisers of the next KV head of pass 2.
+//   warp 2        merges the per-warp partial row statistics of pass 1 across the grid;
+//   warp 3        stages the merged row normalisers of the next KV head of pass 2;
+//   warps 4..     kGroups epilogue groups of 128 threads.  Accumulator block u (128 TMEM lanes x 128
+//                 columns) sits in slot u % 4 and is taken by group u % kGroups.
 // The operand roles are swapped between the passes so that no reduction crosses threads:
 //   pass 1  S[128 x 128] = Q K^T  (A = a block of 128 query rows): a thread owns a QUERY ROW and keeps
 //           the running max m and l = sum_j exp2(c (s_j - m)); per-warp partial (m, l) go to the workspace;
@@ -18,8 +17,17 @@
 //           and adds exp2(c s - M_r) over the rows, M_r = c m_r + log2(l_r) merged from the partials.
 //           With more than 128 query rows a key gets two blocks, added into the scores with red.add
 //           (two commutative additions onto zero: the result does not depend on their order).
-// A share of the exponentials can be evaluated on the FMA pipe (round, degree-4 polynomial on
+// A share of the exponentials is evaluated on the FMA pipe (round, degree-4 polynomial on
 // [-1/2, 1/2], exponent insertion) because the ex2 unit, at 16 results per clock per SM, is the binding unit.
+//
+// An epilogue warp is the only source of work for the ex2 unit of its scheduler, and it has two or three
+// peers there: whatever it does between two exponentials leaves the unit idle unless a peer happens to be
+// inside its own stream.  So an epilogue warp reads its accumulators 16 columns at a time into two
+// register arrays that alternate: the read of the next 16 columns - of the same block, or of the warp's
+// next block if that one is already complete - is in flight while the current 16 are exponentiated, the
+// accumulator slot goes back to the MMA warp as soon as its last columns are in registers, and the
+// bookkeeping per block (which tile, which head, where the result goes) is a handful of integer
+// operations on a cursor that moves by a fixed stride.
 //
 // KV heads are taken in groups whose keys fit in a share of the L2.  The tiles of a group are split
 // statically and contiguously over the CTAs, the same split in both passes, and pass 2 walks its range
@@ -34,43 +42,27 @@
 // JQ_ERR_TIMEOUT in the status word and raises a CTA-wide abort flag that every other wait polls; all
 // roles then run out of their loops without touching data and leave through the common exit (which
 // frees the tensor memory).
-//
-// The code outside the exponential stream is kept short (rolled loops over 32-column pieces, one copy of
-// each block routine, 32-bit index arithmetic, no division per tile, a warp visits only its own blocks):
-// a warp executes it at a fraction of an instruction per clock, and the ex2 unit idles meanwhile.
 #include "jq_internal.cuh"
 #include "jq_tmem_ld.cuh"
 #include <cuda.h>
 #include <cstddef>
-#include <cstdlib>
 #include <mutex>
 
 namespace jq {
 namespace {
 
-// Optional per-warp cycle accounting (compiled in with -DJQ_TRACE, for tuning only): every role adds the
-// cycles it spends in each kind of wait or work to sixteen counters and writes them out on exit.
-#ifdef JQ_TRACE
-#define TR_DECL long long tr_[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}; const long long tr_start_ = clock64(); long long tr_t_ = tr_start_
-#define TR_ADD(i) do { const long long n_ = clock64(); tr_[i] += n_ - tr_t_; tr_t_ = n_; } while (0)
-#define TR_DUMP do { tr_[15] = clock64() - tr_start_; if (P.trace && lane == 0) for (int k_ = 0; k_ < 16; ++k_) P.trace[((size_t)blockIdx.x * 32 + warp) * 16 + k_] = tr_[k_]; } while (0)
-#else
-#define TR_DECL
-#define TR_ADD(i)
-#define TR_DUMP
-#endif
-
-#ifndef JQ_POLY_OF8
-#define JQ_POLY_OF8 2
-#endif
-
 constexpr int kTile = 128;                       // keys per tile
 constexpr int kMaxStages = 5;                    // K ring depth (5 when R <= 128, 3 above)
-// Epilogue groups of 128 threads: the kernel is built for 3 (R <= 128) and for 4 (R > 128, where the fourth
-// group is worth more than the slot it takes from the MMA's lead: config 5 runs 3 % faster, config 3 4 % slower)
-constexpr int kGroupsNarrow = 3, kGroupsWide = 4;
+#ifndef JQ_GROUPS_NARROW
+#define JQ_GROUPS_NARROW 3
+#endif
+#ifndef JQ_GROUPS_WIDE
+#define JQ_GROUPS_WIDE 4
+#endif
+constexpr int kGroupsNarrow = JQ_GROUPS_NARROW, kGroupsWide = JQ_GROUPS_WIDE;   // epilogue groups for R <= 128 / R > 128
 constexpr int kTSlots = 4;                       // accumulator slots in tensor memory
-constexpr int threads_for(int groups) { return (4 * groups + 4) * 32; }   // producer, MMA, 4 warps per group, merge, stage
+constexpr int kSpecialWarps = 4;                 // producer, MMA, merge, stage: one warpgroup
+__host__ __device__ constexpr int threads_for(int groups) { return (kSpecialWarps + 4 * groups) * 32; }
 constexpr uint32_t kHalfBytes = kTile * 128;     // one 64-column half of a K tile (128-byte rows)
 constexpr uint32_t kStageBytes = 2 * kHalfBytes; // 32 KiB
 constexpr uint32_t kCtlBytes = 3072;             // barriers, flags, M_r
@@ -78,19 +70,11 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSlotCols = kTmemCols / kTSlots;
 constexpr long long kWaitCycles = 4000000000ll;  // about 2 s of SM clock per wait
 constexpr int kRing = 4;                         // grid counters per kind
-#ifndef JQ_SLEEP_LONG
-#define JQ_SLEEP_LONG 256
+constexpr uint32_t kSleepLong = 256;             // ns between polls of a waiter that runs ahead (producer, stager)
+constexpr uint32_t kSleepShort = 32;             // ns between polls of a waiter on the critical path
+#ifndef JQ_POLY_OF8
+#define JQ_POLY_OF8 2
 #endif
-#ifndef JQ_SLEEP_SHORT
-#define JQ_SLEEP_SHORT 32
-#endif
-constexpr uint32_t kSleepLong = JQ_SLEEP_LONG;   // ns between polls of a waiter that runs ahead (producer, stager)
-constexpr uint32_t kSleepShort = JQ_SLEEP_SHORT; // ns between polls of a waiter on the critical path
-#ifndef JQ_CHUNK
-#define JQ_CHUNK 32
-#endif
-constexpr int kChunk = JQ_CHUNK;                 // accumulator columns per tensor-memory read (32 or 64)
-static_assert(kChunk == 32 || kChunk == 64, "kChunk");
 constexpr int kPolyOf8 = JQ_POLY_OF8;            // of every 8 pairs of exponentials, this many go to the FMA pipe
 // words of the workspace status block
 constexpr int kWStatus = 0, kWDone = 1, kWCnt1 = 8, kWCnt2 = 12;
@@ -110,11 +94,11 @@ static_assert(offsetof(Ctl, Ms) % 16 == 0, "Ms must be 16-byte aligned");
 static_assert(sizeof(Ctl) <= kCtlBytes, "control block too large");
 
 struct Params {
-    int L, R, Rbox, Rpad;    // Rbox = 128 or 256: query rows staged per KV head (rows >= R are zero)
+    int L, R, Rbox, Rpad;    // Rbox = 128 or 256: query rows staged per KV head (rows >= R are zero); Rpad = R rounded up to 32
     int Hkv, tph;            // KV heads; tiles per head (the window tile included)
     int hpg, ngroups;        // heads per group, groups
     int stages;              // K ring depth
-    int depth;               // pass 2 of a group starts after pass 1 of `depth` groups: 1 = P1(0) P2(0) P1(1) ..., 2 = P1(0) P1(1) P2(0) P1(2) ..., 3 = P1(0) P1(1) P1(2) P2(0) ...
+    int depth;               // pass 2 of a group starts after pass 1 of `depth` groups: 1 = P1(0) P2(0) P1(1) ..., 2 = P1(0) P1(1) P2(0) P1(2) ...
     float c;                 // log2(e) / sqrt(d)
     float2 *part;            // [Hkv][kSlots][R]
     float *Mrow;             // [Hkv][R]   c*m + log2(l) per query row
@@ -124,9 +108,6 @@ struct Params {
     int w;                   // soft-token queries per query head
     const CUtensorMap *maps; // not null: [layers][2] tensor maps (K, Qwin) of layers in buffers of their own, hpl KV heads each
     int hpl;
-#ifdef JQ_TRACE
-    long long *trace;
-#endif
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -151,6 +132,17 @@ __device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity)
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// One look at the barrier, no waiting.
+__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
@@ -211,6 +203,13 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, u
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
+// A tensor map that the host wrote into global memory (with an ordinary copy) must be acquired by the
+// tensor-map proxy before a TMA instruction of this CTA reads it.
+__device__ __forceinline__ void tensormap_acquire(const CUtensorMap *map)
+{
+    asm volatile("fence.proxy.tensormap::generic.acquire.sys [%0], 128;" ::"l"(map) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -245,7 +244,6 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
     return y;
 }
-
 
 // Shared-memory matrix descriptor: K-major, 128-byte swizzle, rows of 128 bytes, 8-row groups 1024
 // bytes apart (stride byte offset), leading byte offset 16 (unused for swizzled K-major), version 1.
@@ -303,15 +301,17 @@ __device__ __noinline__ bool cta_has_tile(uint32_t b, uint32_t T, uint32_t G) { 
 
 // ------------------------------------------------------------------ exponentials
 
-// exp2 of a pair on the FMA pipe.  x is clamped to [-126, 127] (so that the exponent insertion cannot
-// wrap; 2^-126 stands in for anything smaller), split into n = round(x) and r = x - n in [-1/2, 1/2]
-// by the add-a-large-constant trick, 2^r comes from a degree-4 polynomial (relative error < 3e-6,
-// a least-maximum fit of 2^r on that interval) and n is added into the exponent field.
+// exp2 of a pair on the FMA pipe, for x <= 0 (both passes only ever ask for that: the argument is a
+// logit minus something that is at least the row's largest).  x is clamped to >= -126 (so that the
+// exponent insertion cannot wrap; 2^-126 stands in for anything smaller), split into n = round(x) and
+// r = x - n in [-1/2, 1/2] by the add-a-large-constant trick, 2^r comes from a degree-4 polynomial
+// (relative error < 3e-6, a least-maximum fit of 2^r on that interval) and n is added into the
+// exponent field.
 __device__ __forceinline__ float2 exp2_fma_pair(float2 x)
 {
     const float kMagic = 12582912.f;   // 1.5 * 2^23: x + kMagic holds round(x) in its low mantissa bits
-    x.x = fminf(fmaxf(x.x, -126.f), 127.f);
-    x.y = fminf(fmaxf(x.y, -126.f), 127.f);
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
     const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
     const float2 nn = __ffma2_rn(t, make_float2(-1.f, -1.f), make_float2(kMagic, kMagic));   // -round(x)
     const float2 r = __fadd2_rn(x, nn);
@@ -332,37 +332,66 @@ __device__ __forceinline__ void exp_acc2(float2 &acc, uint32_t v0, uint32_t v1, 
     acc = __fadd2_rn(acc, POLY ? exp2_fma_pair(x) : make_float2(ex2(x.x), ex2(x.y)));
 }
 
-// 32 values, value t against bias[t] (shared memory, or a register array holding one bias 32 times
-// would waste registers: pass 1 passes a pointer to a 4-float broadcast instead, see STRIDE).
-// STRIDE = 1: bias[t]; STRIDE = 0: the same 4 floats for every quad.
-template <int STRIDE>
-__device__ __forceinline__ void exp_acc32(float2 &a0, float2 &a1, const uint32_t *v, float2 cc, const float4 *bias)
+// Pair i of the 8 pairs of a 16-column read goes to the FMA pipe when this says so: kPolyOf8 of them, spread evenly.
+__host__ __device__ constexpr bool poly_pair(int i) { return ((i + 1) * kPolyOf8) / 8 != (i * kPolyOf8) / 8; }
+
+// 16 values against 16 biases (pass 2: the negated row normalisers, from shared memory).
+__device__ __forceinline__ void exp_acc16(float2 &a0, float2 &a1, const uint32_t (&v)[16], float2 cc, const float4 *bias)
 {
-#pragma unroll
-    for (int t = 0; t < 32; t += 16) {
-        const float4 b0 = bias[STRIDE * (t / 4)], b1 = bias[STRIDE * (t / 4 + 1)];
-        const float4 b2 = bias[STRIDE * (t / 4 + 2)], b3 = bias[STRIDE * (t / 4 + 3)];
-        exp_acc2<(kPolyOf8 > 0)>(a0, v[t + 0], v[t + 1], cc, make_float2(b0.x, b0.y));
-        exp_acc2<false>(a1, v[t + 2], v[t + 3], cc, make_float2(b0.z, b0.w));
-        exp_acc2<(kPolyOf8 > 4)>(a0, v[t + 4], v[t + 5], cc, make_float2(b1.x, b1.y));
-        exp_acc2<(kPolyOf8 > 2)>(a1, v[t + 6], v[t + 7], cc, make_float2(b1.z, b1.w));
-        exp_acc2<(kPolyOf8 > 1)>(a0, v[t + 8], v[t + 9], cc, make_float2(b2.x, b2.y));
-        exp_acc2<false>(a1, v[t + 10], v[t + 11], cc, make_float2(b2.z, b2.w));
-        exp_acc2<(kPolyOf8 > 5)>(a0, v[t + 12], v[t + 13], cc, make_float2(b3.x, b3.y));
-        exp_acc2<(kPolyOf8 > 3)>(a1, v[t + 14], v[t + 15], cc, make_float2(b3.z, b3.w));
-    }
+    const float4 b0 = bias[0], b1 = bias[1], b2 = bias[2], b3 = bias[3];
+    exp_acc2<poly_pair(0)>(a0, v[0], v[1], cc, make_float2(b0.x, b0.y));
+    exp_acc2<poly_pair(1)>(a1, v[2], v[3], cc, make_float2(b0.z, b0.w));
+    exp_acc2<poly_pair(2)>(a0, v[4], v[5], cc, make_float2(b1.x, b1.y));
+    exp_acc2<poly_pair(3)>(a1, v[6], v[7], cc, make_float2(b1.z, b1.w));
+    exp_acc2<poly_pair(4)>(a0, v[8], v[9], cc, make_float2(b2.x, b2.y));
+    exp_acc2<poly_pair(5)>(a1, v[10], v[11], cc, make_float2(b2.z, b2.w));
+    exp_acc2<poly_pair(6)>(a0, v[12], v[13], cc, make_float2(b3.x, b3.y));
+    exp_acc2<poly_pair(7)>(a1, v[14], v[15], cc, make_float2(b3.z, b3.w));
 }
 
-template <int N>
-__device__ __forceinline__ float max_of(const uint32_t (&v)[N])
+// 16 values against one bias (pass 1: minus the running maximum of the row).
+__device__ __forceinline__ void exp_acc16(float2 &a0, float2 &a1, const uint32_t (&v)[16], float2 cc, float2 b)
+{
+    exp_acc2<poly_pair(0)>(a0, v[0], v[1], cc, b);
+    exp_acc2<poly_pair(1)>(a1, v[2], v[3], cc, b);
+    exp_acc2<poly_pair(2)>(a0, v[4], v[5], cc, b);
+    exp_acc2<poly_pair(3)>(a1, v[6], v[7], cc, b);
+    exp_acc2<poly_pair(4)>(a0, v[8], v[9], cc, b);
+    exp_acc2<poly_pair(5)>(a1, v[10], v[11], cc, b);
+    exp_acc2<poly_pair(6)>(a0, v[12], v[13], cc, b);
+    exp_acc2<poly_pair(7)>(a1, v[14], v[15], cc, b);
+}
+
+__device__ __forceinline__ float max_of16(const uint32_t (&v)[16])
 {
     float c0 = -INFINITY, c1 = -INFINITY;
 #pragma unroll
-    for (int t = 0; t < N; t += 4) {
+    for (int t = 0; t < 16; t += 4) {
         c0 = max3(c0, __uint_as_float(v[t + 0]), __uint_as_float(v[t + 1]));
         c1 = max3(c1, __uint_as_float(v[t + 2]), __uint_as_float(v[t + 3]));
     }
     return fmaxf(c0, c1);
+}
+
+// Pass 1, 16 keys of a query row: online softmax statistics.  The reference is the running max, raised
+// (and l rescaled) when the keys bring a larger value; the max runs on the ALU pipe and, unlike a check
+// of the sum, does not wait for the exponentials in flight.  Keys at column >= valid are not keys (-inf).
+struct RowState { float m; float2 l01, l23; };
+__device__ __forceinline__ void p1_half(uint32_t (&v)[16], int c0, int valid, float c, float2 cc, RowState &st)
+{
+    if (valid < c0 + 16) {
+#pragma unroll
+        for (int t = 0; t < 16; ++t) if (c0 + t >= valid) v[t] = 0xff800000u;
+    }
+    const float cm = max_of16(v);
+    if (cm > st.m) {
+        const float f = ex2(c * (st.m - cm));   // 0 for the first keys (m = -inf)
+        st.l01 = make_float2(st.l01.x * f, st.l01.y * f);
+        st.l23 = make_float2(st.l23.x * f, st.l23.y * f);
+        st.m = cm;
+    }
+    const float nb = -st.m * c;
+    exp_acc16(st.l01, st.l23, v, cc, make_float2(nb, nb));
 }
 
 // ------------------------------------------------------------------ schedule
@@ -408,7 +437,7 @@ __global__ void __launch_bounds__(threads_for(kGroups), 1)
 score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ,
             const __grid_constant__ CUtensorMap mapW, const __grid_constant__ Params P)
 {
-    constexpr int kEpiWarps = 4 * kGroups, kMergeWarp = 2 + kEpiWarps, kStageWarp = kMergeWarp + 1;
+    constexpr int kEpiWarps = 4 * kGroups;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     if (smem_u32(smem_raw) & 1023u) {   // the swizzled tiles need 1024-byte alignment; nothing has been started yet
         if (threadIdx.x == 0) atomicMax(P.status + kWStatus, (int)JQ_ERR_CUDA);
@@ -431,9 +460,8 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         for (int s = 0; s < 2; ++s) {
             mbar_init(&ctl->q_full[s], 1); mbar_init(&ctl->q_empty[s], 1);
             mbar_init(&ctl->ms_full[s], 1); mbar_init(&ctl->ms_empty[s], kEpiWarps);
-
         }
-        for (int s = 0; s < kTSlots; ++s) { mbar_init(&ctl->t_full[s], 1); mbar_init(&ctl->t_empty[s], 128); mbar_init(&ctl->p1_done[s], kEpiWarps); }
+        for (int s = 0; s < kTSlots; ++s) { mbar_init(&ctl->t_full[s], 1); mbar_init(&ctl->t_empty[s], 4); mbar_init(&ctl->p1_done[s], kEpiWarps); }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -447,58 +475,53 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     const uint32_t tmem = *(volatile uint32_t *)&ctl->tmem_base;
     cudaGridDependencySynchronize();   // no global memory has been touched so far
 
-    if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer
-        if (lane == 0) {
-            TR_DECL;
-            uint32_t st = 0, ph = 0, qn = 0;                  // ring stage and its phase; query loads so far
-            int prev_kv = -1;
-            const CUtensorMap *head_mapK = &mapK, *head_mapQ = &mapQ;   // maps and head coordinate of the current KV head
-            int head_c2 = 0;
-            bool ok = true;
+    if (warp < kSpecialWarps) {
+        if (warp == 0) {
+            // ---------------------------------------------------------------- TMA producer
+            if (lane == 0) {
+                uint32_t st = 0, ph = 0, qn = 0;                  // ring stage and its phase; query loads so far
+                int prev_kv = -1, prev_lay = -1;
+                const CUtensorMap *head_mapK = &mapK, *head_mapQ = &mapQ;   // maps and head coordinate of the current KV head
+                int head_c2 = 0;
+                bool ok = true;
 #pragma unroll 1
-            for (int s = 0; s < nseg && ok; ++s) {
-                const Seg sg = segment(s, P);
-                const int pass = sg.pass, ntiles = sg.ntiles;
-                int kv = sg.kv0, tt = sg.t0;
+                for (int s = 0; s < nseg && ok; ++s) {
+                    const Seg sg = segment(s, P);
+                    const int pass = sg.pass, ntiles = sg.ntiles;
+                    int kv = sg.kv0, tt = sg.t0;
 #pragma unroll 1
-                for (int n = 0; n < ntiles; ++n, walk(pass, tph, kv, tt)) {
-                    TR_ADD(2);
-                    if (kv != prev_kv) {
-                        if (P.maps) {                         // the head's layer has tensor maps of its own
-                            const int lay = kv / P.hpl;
-                            head_mapK = P.maps + 2 * lay; head_mapQ = head_mapK + 1; head_c2 = kv - lay * P.hpl;
-                        } else head_c2 = kv;
-                        const uint32_t qb = qn & 1;
-                        if (!mbar_wait(&ctl->q_empty[qb], ((qn >> 1) & 1) ^ 1, ctl, status, kSleepLong)) { ok = false; break; }
-                        mbar_expect_tx(&ctl->q_full[qb], q_bytes);
-                        tma_load_3d(qbuf + (size_t)qb * q_bytes, head_mapQ, &ctl->q_full[qb], 0, 0, head_c2);
-                        tma_load_3d(qbuf + (size_t)qb * q_bytes + q_bytes / 2, head_mapQ, &ctl->q_full[qb], 64, 0, head_c2);
-                        prev_kv = kv; ++qn;
-                        TR_ADD(0);
+                    for (int n = 0; n < ntiles; ++n, walk(pass, tph, kv, tt)) {
+                        if (kv != prev_kv) {
+                            if (P.maps) {                         // the head's layer has tensor maps of its own
+                                const int lay = kv / P.hpl;
+                                head_mapK = P.maps + 2 * lay; head_mapQ = head_mapK + 1; head_c2 = kv - lay * P.hpl;
+                                if (lay != prev_lay) { tensormap_acquire(head_mapK); tensormap_acquire(head_mapQ); prev_lay = lay; }
+                            } else head_c2 = kv;
+                            const uint32_t qb = qn & 1;
+                            if (!mbar_wait(&ctl->q_empty[qb], ((qn >> 1) & 1) ^ 1, ctl, status, kSleepLong)) { ok = false; break; }
+                            mbar_expect_tx(&ctl->q_full[qb], q_bytes);
+                            tma_load_3d(qbuf + (size_t)qb * q_bytes, head_mapQ, &ctl->q_full[qb], 0, 0, head_c2);
+                            tma_load_3d(qbuf + (size_t)qb * q_bytes + q_bytes / 2, head_mapQ, &ctl->q_full[qb], 64, 0, head_c2);
+                            prev_kv = kv; ++qn;
+                        }
+                        if (!mbar_wait(&ctl->empty[st], ph ^ 1, ctl, status, kSleepLong)) { ok = false; break; }
+                        mbar_expect_tx(&ctl->full[st], kStageBytes);
+                        // window-inclusive mode: in pass 1 the last tile of a head is its window keys (rows past w read as
+                        // zero); in pass 2 that tile lies past the prefix, reads as zero and its scores are never stored
+                        const bool wt = P.wtile && pass == 1 && tt == tph - 1;
+                        const CUtensorMap *map = wt ? &mapW : head_mapK;
+                        const int j0 = wt ? 0 : tt * kTile;
+                        tma_load_3d(kbuf + (size_t)st * kStageBytes, map, &ctl->full[st], 0, j0, head_c2);
+                        tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, map, &ctl->full[st], 64, j0, head_c2);
+                        if (++st == (uint32_t)stages) { st = 0; ph ^= 1; }
                     }
-                    if (!mbar_wait(&ctl->empty[st], ph ^ 1, ctl, status, kSleepLong)) { ok = false; break; }
-                    TR_ADD(1);
-                    mbar_expect_tx(&ctl->full[st], kStageBytes);
-                    // window-inclusive mode: in pass 1 the last tile of a head is its window keys (rows past w read as
-                    // zero); in pass 2 that tile lies past the prefix, reads as zero and its scores are never stored
-                    const bool wt = P.wtile && pass == 1 && tt == tph - 1;
-                    const CUtensorMap *map = wt ? &mapW : head_mapK;
-                    const int j0 = wt ? 0 : tt * kTile;
-                    tma_load_3d(kbuf + (size_t)st * kStageBytes, map, &ctl->full[st], 0, j0, head_c2);
-                    tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, map, &ctl->full[st], 64, j0, head_c2);
-                    if (++st == (uint32_t)stages) { st = 0; ph ^= 1; }
                 }
             }
-            TR_DUMP;
-        }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer (all 32 lanes walk the loop)
-        {
-            TR_DECL;
+        } else if (warp == 1) {
+            // ---------------------------------------------------------------- MMA issuer (all 32 lanes walk the loop)
             const uint32_t idesc1 = instr_desc(128, kTile);
-            // pass 2: a block's columns are the query rows it covers, rounded up to 16
-            const uint32_t idesc2a = instr_desc(kTile, min(128, Rpad)), idesc2b = instr_desc(kTile, max(16, Rpad - 128));
+            // pass 2: a block's columns are the query rows it covers, rounded up to 32 (the rows past R are zero)
+            const uint32_t idesc2a = instr_desc(kTile, min(128, Rpad)), idesc2b = instr_desc(kTile, max(32, Rpad - 128));
             uint32_t st = 0, ph = 0, qn = 0, u = 0;           // ring stage and phase, query loads, accumulator blocks so far
             int prev_kv = -1;
             bool ok = true;
@@ -509,65 +532,196 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                 int kv = sg.kv0, tt = sg.t0;
 #pragma unroll 1
                 for (int n = 0; n < ntiles && ok; ++n, walk(pass, tph, kv, tt)) {
-                    TR_ADD(4);
                     if (kv != prev_kv) {
                         if (qn > 0) tc_commit(&ctl->q_empty[(qn - 1) & 1]);   // the previous head's queries are free once its MMAs retire
                         if (!mbar_wait(&ctl->q_full[qn & 1], (qn >> 1) & 1, ctl, status, kSleepShort)) { ok = false; break; }
                         prev_kv = kv; ++qn;
-                        TR_ADD(0);
                     }
                     if (!mbar_wait(&ctl->full[st], ph, ctl, status, kSleepShort)) { ok = false; break; }
-                    TR_ADD(1);
                     const uint32_t k_lo = desc_lo(smem_u32(kbuf) + st * kStageBytes);
                     const uint32_t q_lo = desc_lo(smem_u32(qbuf) + ((qn - 1) & 1) * q_bytes);
 #pragma unroll 1
                     for (int blk = 0; blk < nblk; ++blk, ++u) {
                         const uint32_t slot = u % kTSlots;
                         if (!mbar_wait(&ctl->t_empty[slot], ((u / kTSlots) & 1) ^ 1, ctl, status, kSleepShort)) { ok = false; break; }
-                        TR_ADD(2);
                         tc_fence_after();
                         const uint32_t d = tmem + slot * kSlotCols;
                         const uint32_t qb_lo = q_lo + (uint32_t)blk * (kHalfBytes >> 4);   // query rows [128 blk, 128 blk + 128)
                         if (pass == 1) tc_mma_block(d, qb_lo, k_lo, q_bytes / 2, kHalfBytes, idesc1);
                         else tc_mma_block(d, k_lo, qb_lo, kHalfBytes, q_bytes / 2, blk == 0 ? idesc2a : idesc2b);
                         tc_commit(&ctl->t_full[slot]);
-                        TR_ADD(3);
                     }
                     if (ok) tc_commit(&ctl->empty[st]);
                     if (++st == (uint32_t)stages) { st = 0; ph ^= 1; }
                 }
             }
-            TR_DUMP;
+        } else if (warp == 2) {
+            // ---------------------------------------------------------------- grid-wide merge of the pass-1 partials
+            // Group g: once every epilogue warp of every CTA has published its partials, this CTA combines its
+            // share of the group's rows into M_r = c*m_r + log2(l_r), and counts itself in.
+            const float c = P.c;
+            const uint32_t Gu = (uint32_t)G;
+#pragma unroll 1
+            for (int g = 0; g < P.ngroups; ++g) {
+                int ok = 1;
+                // this CTA's epilogue warps first (their partial stores happen-before the arrival), then the grid
+                ok = mbar_wait(&ctl->p1_done[g & 3], (g >> 2) & 1, ctl, P.status, kSleepLong) ? 1 : 0;
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (lane == 0) {
+                    __threadfence();
+                    atomicAdd(P.status + kWCnt1 + (g & (kRing - 1)), 1);
+                    ok = wait_counter(P.status + kWCnt1 + (g & (kRing - 1)), (g / kRing + 1) * G, ctl, P.status) ? 1 : 0;
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                const int h0 = g * P.hpg, nh = min(P.hpg, P.Hkv - h0);
+                const uint32_t T = (uint32_t)nh * P.tph;
+                // This CTA's rows of the group are blockIdx.x + k G.  They are taken `rows_par` at a time, each by a
+                // sub-group of 32 / rows_par lanes that splits the row's partial slots, four loads in flight per
+                // lane; an empty partial (or one of a CTA that had no tile of the head) counts as (-inf, 0).
+                const int nitems = nh * P.R;
+                const int nrows = (nitems > (int)blockIdx.x) ? (nitems - 1 - (int)blockIdx.x) / G + 1 : 0;
+                int rows_par = 1;
+                while (rows_par < nrows && rows_par < 32) rows_par <<= 1;
+                const int lpr = 32 / rows_par, sub = lane % lpr;
+#pragma unroll 1
+                for (int base = 0; base < nrows; base += rows_par) {
+                    const int my = base + lane / lpr;
+                    const bool have = my < nrows;
+                    const int item = blockIdx.x + (have ? my : 0) * G;
+                    const int hl = item / P.R, r = item - hl * P.R, kv = h0 + hl;
+                    const uint32_t first = (uint32_t)hl * P.tph;
+                    const int b_lo = owner_of_tile(first, T, Gu), b_hi = owner_of_tile(first + P.tph - 1, T, Gu);
+                    const int nsl = have ? (b_hi - b_lo + 1) * kGroups : 0;   // every epilogue group of a contributing CTA wrote a partial
+                    const float2 *src = P.part + ((size_t)kv * kSlots + kGroups * b_lo) * P.R + r;
+                    float m = -INFINITY, l = 0.f;
+#pragma unroll 1
+                    for (int i0 = sub; i0 < nsl; i0 += lpr * 4) {
+                        float2 p[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const int i = i0 + lpr * k;
+                            p[k] = make_float2(-INFINITY, 0.f);
+                            // (a CTA between b_lo and b_hi always has a tile of this head unless the group has fewer tiles than CTAs)
+                            if (i < nsl && (T >= Gu || cta_has_tile(b_lo + i / kGroups, T, Gu)))
+                                p[k] = __ldcg(src + (size_t)i * P.R);
+                        }
+                        float mn = m;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) if (p[k].y > 0.f) mn = fmaxf(mn, p[k].x);
+                        if (mn > -INFINITY) {
+                            float acc = (l > 0.f) ? l * ex2(c * (m - mn)) : 0.f;
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) if (p[k].y > 0.f) acc += p[k].y * ex2(c * (p[k].x - mn));
+                            m = mn; l = acc;
+                        }
+                    }
+                    // butterfly over the sub-group (a fixed order, hence deterministic): first the common
+                    // reference, then the sum against it
+                    float mw = (l > 0.f) ? m : -INFINITY;
+                    for (int o = lpr >> 1; o >= 1; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, o));
+                    l = (l > 0.f) ? l * ex2(c * (m - mw)) : 0.f;
+                    for (int o = lpr >> 1; o >= 1; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+                    const float M = c * mw + log2f(l);
+                    if (have && sub == 0) P.Mrow[(size_t)kv * P.R + r] = M;
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    atomicAdd(P.status + kWCnt2 + (g & (kRing - 1)), 1);
+                }
+            }
+        } else {
+            // ---------------------------------------------------------------- pass-2 stager
+            // Walks the pass-2 segments in order.  Per segment: with two blocks per key, zeroes the scores of
+            // this CTA's keys (the epilogue adds into them); waits until the group's normalisers are merged;
+            // then feeds -M_r of each KV head of the segment into the double-buffered shared array.
+            uint32_t hs = 0;
+            int ok = 1;
+#pragma unroll 1
+            for (int s = 0; s < nseg && ok; ++s) {
+                const Seg sg = segment(s, P);
+                if (sg.pass != 2 || sg.ntiles == 0) continue;
+                if (nblk == 2) {
+                    int kv = sg.kv0, tt = sg.t0;
+                    for (int n = 0; n < sg.ntiles; ++n, walk(2, tph, kv, tt)) {
+                        float *dst = P.scores + (size_t)kv * P.L + tt * kTile;
+                        for (int t = lane; t < kTile && tt * kTile + t < P.L; t += 32) dst[t] = 0.f;
+                    }
+                    __threadfence();
+                }
+                if (lane == 0)
+                    ok = wait_counter(P.status + kWCnt2 + (sg.g & (kRing - 1)), (sg.g / kRing + 1) * G, ctl, P.status) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                int prev_kv = -1;
+                int kv = sg.kv0, tt = sg.t0;
+#pragma unroll 1
+                for (int n = 0; n < sg.ntiles && ok; ++n, walk(2, tph, kv, tt)) {
+                    if (kv == prev_kv) continue;
+                    prev_kv = kv;
+                    const uint32_t buf = hs & 1;
+                    ok = mbar_wait(&ctl->ms_empty[buf], ((hs >> 1) & 1) ^ 1, ctl, status, kSleepLong) ? 1 : 0;
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    for (int r = lane; r < kMaxR; r += 32)   // stored negated: x = c s + (-M_r); -inf silences a padding column
+                        ctl->Ms[buf][r] = (r < P.R) ? -__ldcg(&P.Mrow[(size_t)kv * P.R + r]) : -INFINITY;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->ms_full[buf], 1);
+                    ++hs;
+                }
+            }
         }
-    } else if (warp < kMergeWarp) {
+    } else {
         // ---------------------------------------------------------------- epilogue groups
-        // A warp only visits the accumulator blocks of its own group (every kGroups-th block of the
-        // CTA's sequence) and moves its tile cursor by the tiles in between: the code outside the
-        // exponential stream is executed at a fraction of an instruction per clock, so there must be
-        // little of it.
-        const int grp = (warp - 2) >> 2, quarter = warp & 3;
+        const int grp = (warp - kSpecialWarps) >> 2, quarter = warp & 3;
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         const int row0 = quarter * 32 + lane;                   // TMEM lane: query row within its block (pass 1), key within its tile (pass 2)
-        const int blk_shift = nblk - 1;                         // blocks per tile is 1 or 2
+        const int bs = nblk - 1;                                // blocks per tile is 1 or 2: shift and mask
         const float c = P.c;
         const float2 cc = make_float2(c, c);
         float *const scores_out = P.scores;
         float2 *const part_out = P.part + (size_t)(kGroups * blockIdx.x + grp) * R;
         const int win_i0 = row0 % P.w, win_i1 = (row0 + 128) % P.w;   // soft-token index of this thread's row in block 0 / block 1
+        const int np0 = min(128, Rpad) >> 5, np1 = (Rpad - 128) >> 5; // pass 2: 32-column pieces of a key's first / second block
         uint32_t u = 0;                                         // accumulator blocks of the CTA before this segment
         int hs = 0;                                             // pass-2 heads of the CTA before this segment
         bool ok = true;
-        TR_DECL;
+        uint32_t va[16], vb[16];                                // the two alternating 16-column reads
+
+        // Slot and parity of the CTA's accumulator block number uu; the block after this group's block uu is uu + kGroups.
+        // Giving a slot back: the warp's reads of it are complete (tcgen05.wait::ld is warp-wide), one lane tells the MMA warp.
+        auto release = [&](uint32_t slot) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->t_empty[slot], 1);
+        };
+        // One look whether block uu is complete; if so its first 16 columns are requested (into va).  Warp-uniform.
+        auto try_begin = [&](uint32_t uu) -> bool {
+            const uint32_t slot = uu % kTSlots;
+            if (!__all_sync(0xffffffffu, mbar_test(&ctl->t_full[slot], (uu / kTSlots) & 1))) return false;
+            tc_fence_after();
+            JQ_TMEM_LD16(lane_addr + slot * kSlotCols, va);
+            return true;
+        };
+        auto begin = [&](uint32_t uu) -> bool {
+            const uint32_t slot = uu % kTSlots;
+            if (!mbar_wait(&ctl->t_full[slot], (uu / kTSlots) & 1, ctl, status, kSleepShort)) return false;
+            tc_fence_after();
+            JQ_TMEM_LD16(lane_addr + slot * kSlotCols, va);
+            return true;
+        };
 
 #pragma unroll 1
-        for (int s = 0; s < nseg; ++s) {
+        for (int s = 0; s < nseg && ok; ++s) {
             const Seg sg = segment(s, P);
-            const int ntiles = sg.ntiles, nunits = ntiles << blk_shift;
+            const int ntiles = sg.ntiles, nunits = ntiles << bs;
             int kv = sg.kv0, tt = sg.t0, at = 0;                // tile cursor: head, tile in head, index in the segment
             int k = (grp + kGroups - (int)(u % kGroups)) % kGroups;   // this group's first block of the segment
+            bool pre = false;                                   // the first read of block k has already been requested
             if (sg.pass == 1) {
                 // Per block of 128 query rows: running max m and l = sum_j exp2(c (s_j - m)).
-                struct RowState { float m; float2 l01, l23; };
                 RowState st0 = {-INFINITY, make_float2(0.f, 0.f), make_float2(0.f, 0.f)}, st1 = st0;
                 int pub = sg.kv0;                               // next head whose partials this warp has to publish
                 // Every group publishes a partial for every head of the CTA's range, an empty one if it saw no block of it.
@@ -583,18 +737,13 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     }
                 };
 #pragma unroll 1
-                for (; k < nunits && ok; k += kGroups) {
-                    const int tl = k >> blk_shift, blk = k & blk_shift;
-                    // at most kGroups tiles ahead: predicated steps, no loop (taken backward branches are dear here)
-#pragma unroll
-                    for (int i_ = 0; i_ < kGroups; ++i_) if (at < tl) { walk(1, tph, kv, tt); ++at; }
-                    publish_upto(kv);
+                for (; k < nunits; k += kGroups) {
+                    const int tl = k >> bs, blk = k & bs;
+                    tt += tl - at; at = tl;
+                    while (tt >= tph) { tt -= tph; ++kv; }
+                    if (kv != pub) publish_upto(kv);
                     const uint32_t uu = u + (uint32_t)k, slot = uu % kTSlots;
-                    TR_ADD(8);
-                    ok = mbar_wait(&ctl->t_full[slot], (uu / kTSlots) & 1, ctl, status, kSleepShort);
-                    if (!ok) break;
-                    TR_ADD(0);
-                    tc_fence_after();
+                    if (!pre && !begin(uu)) { ok = false; break; }
                     const uint32_t taddr = lane_addr + slot * kSlotCols;
                     // keys of this block that count for this thread's row: the prefix keys of the tile, or, in the window
                     // tile, the window keys up to the row's own position (causal)
@@ -602,43 +751,29 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     // one copy of the block code: the second row block borrows the first one's registers
                     if (blk == 1) { const RowState t = st0; st0 = st1; st1 = t; }
 #pragma unroll 1
-                    for (int c0 = 0; c0 < kTile; c0 += kChunk) {
-                        uint32_t v[kChunk];
-                        if (kChunk == 64) JQ_TMEM_LD64(taddr + c0, v); else JQ_TMEM_LD32(taddr + c0, v);
-                        TR_ADD(1);
-                        if (c0 + kChunk == kTile) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], 1); }
-                        if (valid < c0 + kChunk) {
-#pragma unroll
-                            for (int t = 0; t < kChunk; ++t) if (c0 + t >= valid) v[t] = 0xff800000u;   // -inf: not a key
+                    for (int c0 = 0; c0 < kTile; c0 += 32) {
+                        JQ_TMEM_WAIT16(va);
+                        JQ_TMEM_LD16(taddr + c0 + 16, vb);
+                        p1_half(va, c0, valid, c, cc, st0);
+                        JQ_TMEM_WAIT16(vb);
+                        if (c0 + 32 < kTile) JQ_TMEM_LD16(taddr + c0 + 32, va);
+                        else {
+                            release(slot);
+                            pre = (k + kGroups < nunits) && try_begin(uu + kGroups);
                         }
-                        // online softmax statistics: the reference is the running max, raised (and l rescaled) when
-                        // a piece brings a larger value; the max runs on the ALU pipe and, unlike a check of the
-                        // sum, does not wait for the exponentials in flight
-                        const float cm = max_of<kChunk>(v);
-                        if (cm > st0.m) {
-                            const float f = ex2(c * (st0.m - cm));   // 0 for the first piece (m = -inf)
-                            st0.l01 = make_float2(st0.l01.x * f, st0.l01.y * f);
-                            st0.l23 = make_float2(st0.l23.x * f, st0.l23.y * f);
-                            st0.m = cm;
-                        }
-                        const float nb = -st0.m * c;
-                        const float4 b4 = make_float4(nb, nb, nb, nb);
-#pragma unroll
-                        for (int h = 0; h < kChunk; h += 32) exp_acc32<0>(st0.l01, st0.l23, v + h, cc, &b4);
-                        TR_ADD(2);
+                        p1_half(vb, c0 + 16, valid, c, cc, st0);
                     }
                     if (blk == 1) { const RowState t = st0; st0 = st1; st1 = t; }
                 }
-                TR_ADD(8);
                 if (ok && ntiles > 0) {
-                    for (; at < ntiles - 1; ++at) walk(1, tph, kv, tt);
+                    tt += ntiles - 1 - at;
+                    while (tt >= tph) { tt -= tph; ++kv; }
                     publish_upto(kv + 1);
                 }
                 // this warp's share of pass 1 of the group is published: tell the merge warp, which makes the
                 // stores visible to the grid and counts the CTA in (an epilogue warp does not wait for that)
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->p1_done[sg.g & 3], 1);
-                TR_ADD(6);
             } else {
                 // Heads of the segment are numbered hs, hs + 1, ... in walking order (descending KV head); the
                 // stage warp fills buffer (number & 1).  `held` is the number of the head whose normalisers
@@ -653,37 +788,30 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     }
                 };
 #pragma unroll 1
-                for (; k < nunits && ok; k += kGroups) {
-                    const int tl = k >> blk_shift, blk = k & blk_shift;
-#pragma unroll
-                    for (int i_ = 0; i_ < kGroups; ++i_) if (at < tl) { walk(2, tph, kv, tt); ++at; }
-                    TR_ADD(10);
+                for (; k < nunits; k += kGroups) {
+                    const int tl = k >> bs, blk = k & bs;
+                    tt -= tl - at; at = tl;
+                    while (tt < 0) { tt += tph; --kv; }
                     hold(hs + (sg.kv0 - kv));
                     if (!ok) break;
-                    TR_ADD(4);
                     const uint32_t uu = u + (uint32_t)k, slot = uu % kTSlots;
-                    ok = mbar_wait(&ctl->t_full[slot], (uu / kTSlots) & 1, ctl, status, kSleepShort);
-                    if (!ok) break;
-                    TR_ADD(3);
-                    tc_fence_after();
+                    if (!pre && !begin(uu)) { ok = false; break; }
                     const uint32_t taddr = lane_addr + slot * kSlotCols;
-                    const int ncols = min(128, Rpad - blk * 128);      // accumulator columns of this block
-                    const float *bias = ctl->Ms[held & 1] + blk * 128;  // columns that are not query rows carry a bias of -inf
+                    const int np = blk ? np1 : np0;                     // 32-column pieces of this block
+                    const float4 *bias = (const float4 *)(ctl->Ms[held & 1] + blk * 128);  // columns that are not query rows carry a bias of -inf
                     float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
 #pragma unroll 1
-                    for (int c0 = 0; c0 < ncols; c0 += kChunk) {
-                        uint32_t v[kChunk];
-                        if (kChunk == 64) JQ_TMEM_LD64(taddr + c0, v); else JQ_TMEM_LD32(taddr + c0, v);
-                        TR_ADD(1);
-                        if (c0 + kChunk >= ncols) { tc_fence_before(); mbar_arrive(&ctl->t_empty[slot], 1); }
-                        if (ncols < c0 + kChunk) {
-                            // columns the MMA did not write hold whatever tensor memory held: make them finite (their bias is -inf)
-#pragma unroll
-                            for (int t = 0; t < kChunk; ++t) if (c0 + t >= ncols) v[t] = 0u;
+                    for (int p = 0; p < np; ++p) {
+                        JQ_TMEM_WAIT16(va);
+                        JQ_TMEM_LD16(taddr + 32 * p + 16, vb);
+                        exp_acc16(a01, a23, va, cc, bias + 8 * p);
+                        JQ_TMEM_WAIT16(vb);
+                        if (p + 1 < np) JQ_TMEM_LD16(taddr + 32 * p + 32, va);
+                        else {
+                            release(slot);
+                            pre = (k + kGroups < nunits) && try_begin(uu + kGroups);
                         }
-#pragma unroll
-                        for (int h = 0; h < kChunk; h += 32) exp_acc32<1>(a01, a23, v + h, cc, (const float4 *)(bias + c0 + h));
-                        TR_ADD(5);
+                        exp_acc16(a01, a23, vb, cc, bias + 8 * p + 4);
                     }
                     const int key = tt * kTile + row0;
                     if (key < L) {
@@ -693,137 +821,19 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                         else atomicAdd(dst, sum);              // two blocks per key, onto a zero the stage warp wrote
                     }
                 }
-                TR_ADD(10);
                 // take part in the hand-over of every remaining head of the segment, then give the last one back
                 if (ntiles > 0) {
-                    for (; at < ntiles - 1; ++at) walk(2, tph, kv, tt);
+                    tt -= ntiles - 1 - at;
+                    while (tt < 0) { tt += tph; --kv; }
                     const int nheads = sg.kv0 - kv + 1;
                     hold(hs + nheads - 1);
                     if (ok) { __syncwarp(); if (lane == 0) mbar_arrive(&ctl->ms_empty[held & 1], 1); }
                     hs += nheads;
                 }
-                TR_ADD(4);
             }
             u += (uint32_t)nunits;
         }
-        TR_DUMP;
-    } else if (warp == kMergeWarp) {
-        // ---------------------------------------------------------------- grid-wide merge of the pass-1 partials
-        // Group g: once every epilogue warp of every CTA has published its partials, this CTA combines its
-        // share of the group's rows into M_r = c*m_r + log2(l_r), and counts itself in.
-        const float c = P.c;
-        const uint32_t Gu = (uint32_t)G;
-#pragma unroll 1
-        for (int g = 0; g < P.ngroups; ++g) {
-            int ok = 1;
-            // this CTA's epilogue warps first (their partial stores happen-before the arrival), then the grid
-            ok = mbar_wait(&ctl->p1_done[g & 3], (g >> 2) & 1, ctl, P.status, kSleepLong) ? 1 : 0;
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (lane == 0) {
-                __threadfence();
-                atomicAdd(P.status + kWCnt1 + (g & (kRing - 1)), 1);
-                ok = wait_counter(P.status + kWCnt1 + (g & (kRing - 1)), (g / kRing + 1) * G, ctl, P.status) ? 1 : 0;
-            }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) break;
-            const int h0 = g * P.hpg, nh = min(P.hpg, P.Hkv - h0);
-            const uint32_t T = (uint32_t)nh * P.tph;
-            // This CTA's rows of the group are blockIdx.x + k G.  They are taken `rows_par` at a time, each by a
-            // sub-group of 32 / rows_par lanes that splits the row's partial slots, eight loads in flight per
-            // lane; an empty partial (or one of a CTA that had no tile of the head) counts as (-inf, 0).
-            const int nitems = nh * P.R;
-            const int nrows = (nitems > (int)blockIdx.x) ? (nitems - 1 - (int)blockIdx.x) / G + 1 : 0;
-            int rows_par = 1;
-            while (rows_par < nrows && rows_par < 32) rows_par <<= 1;
-            const int lpr = 32 / rows_par, sub = lane % lpr;
-#pragma unroll 1
-            for (int base = 0; base < nrows; base += rows_par) {
-                const int my = base + lane / lpr;
-                const bool have = my < nrows;
-                const int item = blockIdx.x + (have ? my : 0) * G;
-                const int hl = item / P.R, r = item - hl * P.R, kv = h0 + hl;
-                const uint32_t first = (uint32_t)hl * P.tph;
-                const int b_lo = owner_of_tile(first, T, Gu), b_hi = owner_of_tile(first + P.tph - 1, T, Gu);
-                const int nsl = have ? (b_hi - b_lo + 1) * kGroups : 0;   // every epilogue group of a contributing CTA wrote a partial
-                const float2 *src = P.part + ((size_t)kv * kSlots + kGroups * b_lo) * P.R + r;
-                float m = -INFINITY, l = 0.f;
-#pragma unroll 1
-                for (int i0 = sub; i0 < nsl; i0 += lpr * 8) {
-                    float2 p[8];
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const int i = i0 + lpr * k;
-                        p[k] = make_float2(-INFINITY, 0.f);
-                        // (a CTA between b_lo and b_hi always has a tile of this head unless the group has fewer tiles than CTAs)
-                        if (i < nsl && (T >= Gu || cta_has_tile(b_lo + i / kGroups, T, Gu)))
-                            p[k] = __ldcg(src + (size_t)i * P.R);
-                    }
-                    float mn = m;
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) if (p[k].y > 0.f) mn = fmaxf(mn, p[k].x);
-                    if (mn > -INFINITY) {
-                        float acc = (l > 0.f) ? l * ex2(c * (m - mn)) : 0.f;
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) if (p[k].y > 0.f) acc += p[k].y * ex2(c * (p[k].x - mn));
-                        m = mn; l = acc;
-                    }
-                }
-                // butterfly over the sub-group (a fixed order, hence deterministic): first the common
-                // reference, then the sum against it
-                float mw = (l > 0.f) ? m : -INFINITY;
-                for (int o = lpr >> 1; o >= 1; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, o));
-                l = (l > 0.f) ? l * ex2(c * (m - mw)) : 0.f;
-                for (int o = lpr >> 1; o >= 1; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-                const float M = c * mw + log2f(l);
-                if (have && sub == 0) P.Mrow[(size_t)kv * P.R + r] = M;
-            }
-            __syncwarp();
-            if (lane == 0) {
-                __threadfence();
-                atomicAdd(P.status + kWCnt2 + (g & (kRing - 1)), 1);
-            }
-        }
-    } else if (warp == kStageWarp) {
-        // ---------------------------------------------------------------- pass-2 stager
-        // Walks the pass-2 segments in order.  Per segment: with two blocks per key, zeroes the scores of
-        // this CTA's keys (the epilogue adds into them); waits until the group's normalisers are merged;
-        // then feeds -M_r of each KV head of the segment into the double-buffered shared array.
-        uint32_t hs = 0;
-        int ok = 1;
-#pragma unroll 1
-        for (int s = 0; s < nseg && ok; ++s) {
-            const Seg sg = segment(s, P);
-            if (sg.pass != 2 || sg.ntiles == 0) continue;
-            if (nblk == 2) {
-                int kv = sg.kv0, tt = sg.t0;
-                for (int n = 0; n < sg.ntiles; ++n, walk(2, tph, kv, tt)) {
-                    float *dst = P.scores + (size_t)kv * P.L + tt * kTile;
-                    for (int t = lane; t < kTile && tt * kTile + t < P.L; t += 32) dst[t] = 0.f;
-                }
-                __threadfence();
-            }
-            if (lane == 0)
-                ok = wait_counter(P.status + kWCnt2 + (sg.g & (kRing - 1)), (sg.g / kRing + 1) * G, ctl, P.status) ? 1 : 0;
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) break;
-            int prev_kv = -1;
-            int kv = sg.kv0, tt = sg.t0;
-#pragma unroll 1
-            for (int n = 0; n < sg.ntiles && ok; ++n, walk(2, tph, kv, tt)) {
-                if (kv == prev_kv) continue;
-                prev_kv = kv;
-                const uint32_t buf = hs & 1;
-                ok = mbar_wait(&ctl->ms_empty[buf], ((hs >> 1) & 1) ^ 1, ctl, status, kSleepLong) ? 1 : 0;
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                for (int r = lane; r < kMaxR; r += 32)   // stored negated: x = c s + (-M_r); -inf silences a padding column
-                    ctl->Ms[buf][r] = (r < P.R) ? -__ldcg(&P.Mrow[(size_t)kv * P.R + r]) : -INFINITY;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->ms_full[buf], 1);
-                ++hs;
-            }
-        }
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");   // (a read requested ahead on a path that gave up)
     }
 
     // ---------------------------------------------------------------- common exit
@@ -919,20 +929,7 @@ bool device_info(DeviceInfo *out)
     return true;
 }
 
-// Overrides for tuning runs (read once): JQ_SCORE_GROUP_MIB = K bytes per head group, JQ_SCORE_DEPTH = 1..3,
-// the number of groups whose pass 1 precedes the first pass 2.
-long long env_ll(const char *name, long long dflt)
-{
-    const char *v = getenv(name);
-    return (v && *v) ? atoll(v) : dflt;
-}
-
 }  // namespace
-
-#ifdef JQ_TRACE
-static long long *g_trace = nullptr;
-extern "C" void jq_debug_set_trace(long long *p) { g_trace = p; }   // [grid][32 warps][16] int64, device memory
-#endif
 
 bool build_layer_maps(const void *const *K, const void *const *Qwin, int nlayers, const jq_shape &layer, void *host_maps)
 {
@@ -950,24 +947,20 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
 {
     DeviceInfo dev;
     if (!device_info(&dev)) return JQ_ERR_CUDA;
-    static const long long group_mib = env_ll("JQ_SCORE_GROUP_MIB", 32);
-    static const long long order = env_ll("JQ_SCORE_DEPTH", 2);
+    const long long group_mib = 32;   // K bytes of a head group: a share of the L2, so that pass 2 finds its keys there
     const int R = s.group * s.w;
     Params P;
-    P.L = s.L; P.R = R; P.Rbox = R <= 128 ? 128 : 256; P.Rpad = (R + 15) & ~15;
+    P.L = s.L; P.R = R; P.Rbox = R <= 128 ? 128 : 256; P.Rpad = (R + 31) & ~31;
     P.Hkv = s.Hkv;
     P.wtile = Kwin ? 1 : 0;
     P.tph = (s.L + kTile - 1) / kTile + P.wtile;
     P.stages = P.Rbox == 128 ? 5 : 3;
-    P.depth = order < 1 ? 1 : (order > 3 ? 3 : (int)order);
+    P.depth = 2;
     P.c = 1.4426950408889634f / sqrtf((float)s.d);
     P.part = w.part; P.Mrow = w.Mrow; P.scores = scores; P.status = w.status;
     P.w = s.w;
     P.maps = tables ? (const CUtensorMap *)tables->maps : nullptr;
     P.hpl = tables ? tables->hpl : 0;
-#ifdef JQ_TRACE
-    P.trace = g_trace;
-#endif
     CUtensorMap mapK, mapQ, mapW;
     const int map_heads = tables ? tables->hpl : s.Hkv;   // with tables these two describe the first layer and are not used
     if (!make_map(&mapK, K, s.L, map_heads, kTile) || !make_map(&mapQ, Q, R, map_heads, P.Rbox)) return JQ_ERR_CUDA;

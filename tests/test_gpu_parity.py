@@ -234,19 +234,20 @@ def test_cfg3_full_size_layer_budget_sweep():
         run_e2e(W.CFG3.with_budget(budget), K, V, Q, pooled)
 
 
-def test_cfg4_longest_sequence():
-    wl = W.CFG4[3]
-    K, V, Q, _ = W.make_layer(wl, layer=1, seq=3)
+@pytest.mark.parametrize("seq", [2, 3])
+def test_cfg4_long_sequences(seq):
+    wl = W.CFG4[seq]                                           # L = 20480 and 32768 (0 and 1 run in test_evict_layer_end_to_end)
+    K, V, Q, _ = W.make_layer(wl, layer=1, seq=seq)
     run_e2e(wl, K, V, Q)
 
 
-def test_cfg5_full_size_sampled_heads():
-    """L = 131072, R = 256.  The GPU runs the whole layer; the oracle recomputes two of the eight KV
-    heads (heads are independent) and those are compared in full, for every budget of the sweep."""
+def test_cfg5_full_size_all_heads():
+    """L = 131072, R = 256: the whole layer, all eight KV heads, against the oracle, for every budget of
+    the sweep."""
     wl = W.CFG5
     K, V, Q, _ = W.make_layer(wl)
     s = shape_of(wl)
-    heads = [0, 5]
+    heads = list(range(wl.Hkv))
     g = wl.group
     qrows = np.concatenate([np.arange(kv * g, kv * g + g) for kv in heads])
     sc = oracle.score(K[heads], Q[qrows])
@@ -514,3 +515,51 @@ def test_evict_layers_matches_calls_per_layer(Hkv, g, w, L, B, nl):
     K, V, Q, _ = layers[nl - 1]
     pooled = oracle.pool(oracle.score(K, Q), wl.pool)
     assert_kept_sets_agree(gi[(nl - 1) * Hkv:], oracle.select(pooled, wl.budget), pooled, nkeep)
+
+
+def _layers_call(layers, wl, ws=None):
+    """jq_evict_layers on the given (K, V, Q) host layers of workload wl, each in a device buffer of its own."""
+    nl = len(layers)
+    dK, dV, dQ = [dev_bf16(l[0]) for l in layers], [dev_bf16(l[1]) for l in layers], [dev_bf16(l[2]) for l in layers]
+    s = shape_of(wl)
+    Ko = torch.zeros((nl * wl.Hkv, wl.nkeep, 128), dtype=torch.bfloat16, device="cuda")
+    Vo = torch.zeros_like(Ko)
+    idx = torch.full((nl * wl.Hkv, wl.nkeep), -1, dtype=torch.int32, device="cuda")
+    if ws is None:
+        ws = jq.new_layers_workspace(s, nl)
+    jq.evict_layers(dK, dV, dQ, s, Ko, Vo, idx, ws)
+    assert jq.last_device_status(ws) == jq.JQ_OK
+    return host_bits(Ko), host_bits(Vo), idx.cpu().numpy()
+
+
+def test_evict_layers_workspace_reused_with_other_buffers_and_shapes():
+    """One workspace, three calls in a row on different layer buffers, layer counts and shapes: the per-layer
+    tensor maps the call leaves in the workspace are rewritten every time, and the kernel must read the new
+    ones (the first call's buffers are freed before the second runs)."""
+    wa, wb = small_wl(2, 4, 32, 3000, 400), small_wl(4, 4, 64, 1500, 200)
+    ws = jq.new_layers_workspace(shape_of(wa), 6)
+    assert ws.numel() >= jq.layers_workspace_bytes(shape_of(wb), 3)
+    for wl, nl, first in ((wa, 6, 0), (wb, 3, 10), (wa, 4, 20), (wb, 2, 30)):
+        layers = [W.make_layer(wl, layer=first + i) for i in range(nl)]
+        gK, gV, gi = _layers_call(layers, wl, ws)
+        for i, (K, V, Q, _) in enumerate(layers):
+            wK, wV, wi = gpu_evict(K, V, Q, shape_of(wl))
+            sl = slice(i * wl.Hkv, (i + 1) * wl.Hkv)
+            assert np.array_equal(gi[sl], wi) and np.array_equal(gK[sl], wK) and np.array_equal(gV[sl], wV)
+        torch.cuda.empty_cache()
+
+
+def test_evict_layers_cfg5_shape_against_the_oracle():
+    """The benchmark's default call at the 128K-key shape (three distinct layers here), compared with the oracle
+    directly on sampled (layer, head) units."""
+    wl = W.CFG5
+    layers = [W.make_layer(wl, layer=i) for i in range(3)]
+    gK, gV, gi = _layers_call(layers, wl)
+    g = wl.group
+    for layer, kv in ((0, 1), (1, 6), (2, 3), (2, 7)):
+        K, V, Q, _ = layers[layer]
+        po = oracle.pool(oracle.score(K[kv:kv + 1], Q[kv * g:(kv + 1) * g]), wl.pool)
+        u = layer * wl.Hkv + kv
+        assert_kept_sets_agree(gi[u:u + 1], oracle.select(po, wl.budget), po, wl.nkeep)
+        assert np.array_equal(gK[u], K[kv][gi[u]]) and np.array_equal(gV[u], V[kv][gi[u]])
+    assert np.all(np.diff(gi, axis=1) > 0) and gi.min() >= 0 and gi.max() < wl.L
