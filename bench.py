@@ -5,9 +5,12 @@
 
 One step = one pass of the whole hot path (scores -> pool -> top-k -> gather) over every layer of
 one synthetic cache, on one stream.  Every (layer, KV head) is an independent unit of the pass, so the
-layers of a cache are evicted by ONE jq_evict_layer call on tensors that stack the layers along the
-KV-head axis (`--call stacked`, the default: K, V [layers*Hkv, L, d], Qwin [layers*Hq, w, d]); the same
-work as `layers` separate calls (`--call per-layer`) is also timed and reported.  Prints ONE JSON line.
+layers of a cache are evicted by ONE call: jq_evict_layers on the layers' own buffers (`--call layers`,
+the default), or jq_evict_layer on tensors that stack the layers along the KV-head axis (`--call stacked`);
+the same work as one call per layer (`--call per-layer`) is also timed and reported.  The ragged batch
+(`--workload cfg4`: four sequences of different lengths, 32 layers each) is one jq_evict_ragged call per step.
+Every step is bracketed by CUDA events on the launching stream; `value` comes from the time of all K steps
+(first to last event), the median step is reported beside it.  Prints ONE JSON line.
 With N > 1 (torchrun) every rank evicts a cache of its own (independent replicas, no collective on
 the data path); the value is the sum over ranks divided by the slowest rank's time.
 """
@@ -28,9 +31,11 @@ if ROOT not in sys.path:
 import jq_workloads as W  # noqa: E402
 
 METRIC = "prefix tokens evicted/sec per layer"
-# dram__bytes_read.sum + dram__bytes_write.sum of one score_fused launch on one layer (ncu, see profiles/)
-NCU_DRAM_BYTES_PER_LAYER = {"cfg5-llama8b-128k": 355.6e6, "cfg3-llama8b-32k-32layers": 68.8e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of one score_fused launch on one layer (ncu, see profiles/);
+# None once the kernel has changed since the counters were taken
+NCU_DRAM_BYTES_PER_LAYER = {}
 UNIT = "tokens/s"
+SM_MAX_MHZ = 1965.0
 
 
 def parse():
@@ -38,11 +43,12 @@ def parse():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--fma-compare", action="store_true", help="also time the CUDA-core comparator of the scoring step")
     ap.add_argument("--decode", action="store_true", help="also time one decoding step over a layer's pruned cache")
-    ap.add_argument("--steps", type=int, default=60)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg5", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
-    ap.add_argument("--seq", type=int, default=1, help="cfg4 only: which sequence of the ragged batch (0..3)")
+    ap.add_argument("--seq", type=int, default=None,
+                    help="cfg4 only: time one sequence of the ragged batch (0..3) instead of the whole batch in one call")
     ap.add_argument("--budget", type=int, default=None)
     ap.add_argument("--layers", type=int, default=None, help="layer calls per step (default: the workload's)")
     ap.add_argument("--call", default="layers", choices=["layers", "stacked", "per-layer"],
@@ -52,11 +58,12 @@ def parse():
                     help="window-inclusive scoring (jq_evict_layer_windowed): the causal keys of the query positions join the softmax")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the second target cache (the 32K-key workload) of the default line")
     return ap.parse_args()
 
 
 def pick_workload(args):
-    wl = {"cfg2": W.CFG2, "cfg3": W.CFG3, "cfg4": W.CFG4[args.seq % 4], "cfg5": W.CFG5}[args.workload]
+    wl = {"cfg2": W.CFG2, "cfg3": W.CFG3, "cfg4": W.CFG4[(args.seq if args.seq is not None else 3) % 4], "cfg5": W.CFG5}[args.workload]
     if args.workload == "cfg2":
         wl = W.Workload(wl.name, 2, wl.Hkv, wl.Hq, wl.L, wl.w, wl.budget, layers=32, distinct_layers=32)
     if args.budget:
@@ -64,14 +71,18 @@ def pick_workload(args):
     return wl
 
 
+CALLS = {"stacked": "one jq_evict_layer call per step, the layers stacked along the KV-head axis",
+         "layers": "one jq_evict_layers call per step, every layer in buffers of its own",
+         "ragged": "one jq_evict_ragged call per step: every (sequence, layer) a unit with buffers, length and budget of its own",
+         "per-layer": "one jq_evict_layer call per layer",
+         "oracle": "the CPU oracle on a bounded sample of one layer"}
+
+
 def config_of(wl, layers, distinct, call="per-layer"):
     return {"workload": wl.name, "L": wl.L, "Hkv": wl.Hkv, "Hq": wl.Hq, "d": wl.d, "w": wl.w,
             "budget": wl.budget, "pool": wl.pool, "layers_per_step": layers, "distinct_layers": distinct,
-            "call": {"stacked": "one jq_evict_layer call per step, the layers stacked along the KV-head axis",
-                     "layers": "one jq_evict_layers call per step, every layer in buffers of its own",
-                     "per-layer": "one jq_evict_layer call per layer",
-                     "oracle": "the CPU oracle on a bounded sample of one layer"}[call],
-            "l2": "inputs larger than L2 (K of one step: %.0f MiB)" % (distinct * wl.Hkv * wl.L * wl.d * 2 / 2**20)}
+            "call": CALLS[call],
+            "l2": "inputs larger than L2 (K of one step: %.0f MiB)" % (layers * wl.Hkv * wl.L * wl.d * 2 / 2**20)}
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
@@ -167,7 +178,7 @@ class ClockSampler:
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
-                                       "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.f,
+                                       "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.f,
                                       stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
@@ -204,6 +215,45 @@ class ClockSampler:
         return out
 
 
+class Timer:
+    """Steps on one stream with a CUDA event between consecutive steps, the SM clock sampled meanwhile."""
+
+    def __init__(self, torch, stream, barrier, gpu_index, sample_clocks):
+        self.torch, self.stream, self.barrier, self.gpu, self.sample = torch, stream, barrier, gpu_index, sample_clocks
+
+    def run(self, step, steps, warmup=3, min_seconds=0.0):
+        """Returns (total ms of `steps` steps, list of per-step ms, clocks).  With min_seconds the step count is raised so
+        that the region lasts long enough for the clock sampler to see it (the count actually run is len(per-step))."""
+        torch = self.torch
+        for _ in range(warmup):
+            step()
+        self.barrier()
+        if min_seconds > 0:
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            e[0].record(self.stream); step(); e[1].record(self.stream)
+            torch.cuda.synchronize()
+            steps = max(steps, int(min_seconds * 1e3 / max(e[0].elapsed_time(e[1]), 1e-3)) + 1)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        sampler = ClockSampler(self.gpu) if self.sample else None
+        if sampler:
+            time.sleep(0.05)
+        ev[0].record(self.stream)
+        for i in range(steps):
+            step()
+            ev[i + 1].record(self.stream)
+        self.barrier()
+        clocks = sampler.stop() if sampler else None
+        per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+        return ev[0].elapsed_time(ev[steps]), per, clocks
+
+
+def kcycles(ms, clocks):
+    """Thousands of SM cycles a duration corresponds to at the clock sampled while it ran (None without samples)."""
+    if not clocks or not clocks.get("sm_mhz"):
+        return None
+    return ms * clocks["sm_mhz"]
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -217,163 +267,211 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     jq.lib()                                   # fails loudly if the CUDA library is not built
 
-    wl = pick_workload(args)
-    layers = args.layers or wl.layers
-    distinct = min(wl.distinct_layers, layers)
-    s = jq.shape(wl.Hkv, wl.Hq, wl.L, wl.w, wl.budget, wl.pool, wl.d)
-    nkeep = wl.nkeep
-
-    def dev(bits):
-        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
-
-    host0 = None
-    Ks, Vs, Qs, Kws = [], [], [], []
-    for i in range(distinct):
-        K, V, Q, _ = W.make_layer(wl, layer=i, seq=rank)
-        if i == 0:
-            host0 = (K, V, Q)
-        Ks.append(dev(K)); Vs.append(dev(V)); Qs.append(dev(Q))
-        if args.windowed:
-            Kws.append(dev(W.make_window_keys(wl, Q, layer=i, seq=rank)))
-    ws = jq.new_workspace(s)
-    Ko = torch.zeros((wl.Hkv, nkeep, wl.d), dtype=torch.bfloat16, device="cuda")
-    Vo = torch.zeros_like(Ko)
-    idx = torch.zeros((wl.Hkv, nkeep), dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()
-
-    def step_per_layer():
-        for i in range(layers):
-            j = i % distinct
-            if args.windowed:
-                jq.evict_layer_windowed(Ks[j], Vs[j], Qs[j], Kws[j], s, Ko, Vo, idx, ws, stream=stream)
-            else:
-                jq.evict_layer(Ks[j], Vs[j], Qs[j], s, Ko, Vo, idx, ws, stream=stream)
-
-    # the layers of the cache stacked along the KV-head axis (a layer repeated in the workload is copied, so
-    # that every layer of the step has memory of its own)
-    sS = jq.shape(wl.Hkv * layers, wl.Hq * layers, wl.L, wl.w, wl.budget, wl.pool, wl.d)
-    if args.windowed and args.call == "layers":
-        args.call = "stacked"          # the window-inclusive entry point takes one (stacked) tensor per operand
-    one_call = args.call in ("stacked", "layers")
-    if one_call:
-        order = [i % distinct for i in range(layers)]
-        KS = torch.cat([Ks[j] for j in order], 0)
-        VS = torch.cat([Vs[j] for j in order], 0)
-        QS = torch.cat([Qs[j] for j in order], 0)
-        KwS = torch.cat([Kws[j] for j in order], 0) if args.windowed else None
-        wsS = jq.new_workspace(sS)
-        KoS = torch.zeros((sS.Hkv, nkeep, wl.d), dtype=torch.bfloat16, device="cuda")
-        VoS = torch.zeros_like(KoS)
-        idxS = torch.zeros((sS.Hkv, nkeep), dtype=torch.int32, device="cuda")
-
-    def step_stacked():
-        if args.windowed:
-            jq.evict_layer_windowed(KS, VS, QS, KwS, sS, KoS, VoS, idxS, wsS, stream=stream)
-        else:
-            jq.evict_layer(KS, VS, QS, sS, KoS, VoS, idxS, wsS, stream=stream)
-
-    if args.call == "layers":
-        # the layers as a cache holds them: a tensor each (a layer the workload repeats gets a copy of its own)
-        seen = set()
-        KL, VL, QL = [], [], []
-        for j in order:
-            KL.append(Ks[j] if j not in seen else Ks[j].clone())
-            VL.append(Vs[j] if j not in seen else Vs[j].clone())
-            QL.append(Qs[j] if j not in seen else Qs[j].clone())
-            seen.add(j)
-        wsL = jq.new_layers_workspace(s, layers)
-
-    def step_layers():
-        jq.evict_layers(KL, VL, QL, s, KoS, VoS, idxS, wsL, stream=stream)
-
-    step = {"stacked": step_stacked, "layers": step_layers, "per-layer": step_per_layer}[args.call]
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
-    sampler = ClockSampler(local) if rank == 0 else None
+    timer = Timer(torch, stream, barrier, local, rank == 0)
+
+    def dev(bits):
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    def device_layers(wl, layers, distinct, seq):
+        """The layers of a cache as a cache holds them: a tensor each (a layer the workload repeats gets a copy of its own)."""
+        Ks, Vs, Qs, host0 = [], [], [], None
+        for i in range(distinct):
+            K, V, Q, _ = W.make_layer(wl, layer=i, seq=seq)
+            if i == 0:
+                host0 = (K, V, Q)
+            Ks.append(dev(K)); Vs.append(dev(V)); Qs.append(dev(Q))
+        for i in range(distinct, layers):
+            Ks.append(Ks[i % distinct].clone()); Vs.append(Vs[i % distinct].clone()); Qs.append(Qs[i % distinct].clone())
+        return Ks, Vs, Qs, host0
+
+    def one_call_cache(wl, layers, distinct, seq, steps, min_seconds=0.0):
+        """Times jq_evict_layers on a cache of `layers` layers of workload wl: per-layer time, clocks, stage times."""
+        s = jq.shape(wl.Hkv, wl.Hq, wl.L, wl.w, wl.budget, wl.pool, wl.d)
+        Ks, Vs, Qs, _ = device_layers(wl, layers, distinct, seq)
+        Ko = torch.zeros((wl.Hkv * layers, wl.nkeep, wl.d), dtype=torch.bfloat16, device="cuda")
+        Vo = torch.zeros_like(Ko)
+        idx = torch.zeros((wl.Hkv * layers, wl.nkeep), dtype=torch.int32, device="cuda")
+        ws = jq.new_layers_workspace(s, layers)
+        total, per, clocks = timer.run(lambda: jq.evict_layers(Ks, Vs, Qs, s, Ko, Vo, idx, ws, stream=stream), steps, min_seconds=min_seconds)
+        assert jq.last_device_status(ws) == jq.JQ_OK, "device status not ok"
+        t_layer = max_over_ranks(total, world) * 1e-3 / (len(per) * layers)
+        gbs = W.formula_bytes(wl) / t_layer / 1e9
+        return {"workload": wl.name, "L": wl.L, "w": wl.w, "budget": wl.budget, "layers_per_step": layers, "distinct_layers": distinct,
+                "call": CALLS["layers"], "steps": len(per), "ms_per_layer": t_layer * 1e3,
+                "ms_per_layer_median": float(np.median(per)) / layers, "value": job_value(wl, world, t_layer), "unit": UNIT,
+                "layer_formula_gbs": gbs, "layer_frac_of_8tbs": gbs / 8000.0, "clocks": clocks,
+                "kcycles_per_layer": kcycles(t_layer * 1e3, clocks)}
+
+    wl = pick_workload(args)
+    ragged = args.workload == "cfg4" and args.seq is None
+    layers = args.layers or wl.layers
+    distinct = min(wl.distinct_layers, layers)
+    if ragged:
+        distinct = min(distinct, 2)            # two generated layers per sequence, the rest device copies (a step moves the same bytes)
+    s = jq.shape(wl.Hkv, wl.Hq, wl.L, wl.w, wl.budget, wl.pool, wl.d)
+    nkeep = wl.nkeep
+
+    if ragged:
+        # the whole ragged batch in ONE call: unit = (sequence, layer)
+        seqs = [w.with_budget(args.budget) if args.budget else w for w in W.CFG4]
+        RK, RV, RQ, RL, RB = [], [], [], [], []
+        host0 = None
+        for q, wq in enumerate(seqs):
+            Kq, Vq, Qq, h0 = device_layers(wq, layers, distinct, q)
+            if q == 3:
+                host0 = h0
+            RK += Kq; RV += Vq; RQ += Qq; RL += [wq.L] * layers; RB += [wq.budget] * layers
+        rows = jq.ragged_output_rows(s, len(RK), RL, RB)
+        KoR = torch.zeros((rows, wl.d), dtype=torch.bfloat16, device="cuda")
+        VoR = torch.zeros_like(KoR)
+        idxR = torch.zeros((rows,), dtype=torch.int32, device="cuda")
+        wsR = jq.new_ragged_workspace(s, len(RK), RL)
+        tokens_per_layer = sum(w.L for w in seqs)
+        bytes_per_layer = sum(W.formula_bytes(w) for w in seqs)
+
+        def step():
+            jq.evict_ragged(RK, RV, RQ, s, RL, RB, KoR, VoR, idxR, wsR, stream=stream)
+        call = "ragged"
+        Ks, Vs, Qs = RK[3 * layers:], RV[3 * layers:], RQ[3 * layers:]      # the longest sequence, for the per-layer comparison
+    else:
+        Ks, Vs, Qs, host0 = device_layers(wl, layers, distinct, rank)
+        Kws = [dev(W.make_window_keys(wl, host0[2] if i == 0 else W.make_layer(wl, layer=i % distinct, seq=rank)[2], layer=i % distinct, seq=rank))
+               for i in range(layers)] if args.windowed else []
+        tokens_per_layer = wl.L
+        bytes_per_layer = W.formula_bytes(wl)
+        call = args.call
+        if args.windowed and call == "layers":
+            call = "stacked"          # the window-inclusive entry point takes one (stacked) tensor per operand
+    ws = jq.new_workspace(s)
+    Ko = torch.zeros((wl.Hkv, nkeep, wl.d), dtype=torch.bfloat16, device="cuda")
+    Vo = torch.zeros_like(Ko)
+    idx = torch.zeros((wl.Hkv, nkeep), dtype=torch.int32, device="cuda")
+
+    def step_per_layer():
+        for i in range(layers):
+            if args.windowed:
+                jq.evict_layer_windowed(Ks[i], Vs[i], Qs[i], Kws[i], s, Ko, Vo, idx, ws, stream=stream)
+            else:
+                jq.evict_layer(Ks[i], Vs[i], Qs[i], s, Ko, Vo, idx, ws, stream=stream)
+
+    sS = jq.shape(wl.Hkv * layers, wl.Hq * layers, wl.L, wl.w, wl.budget, wl.pool, wl.d)
+    one_call = ragged or call in ("stacked", "layers")
+    if not ragged:
+        KoS = torch.zeros((sS.Hkv, nkeep, wl.d), dtype=torch.bfloat16, device="cuda")
+        VoS = torch.zeros_like(KoS)
+        idxS = torch.zeros((sS.Hkv, nkeep), dtype=torch.int32, device="cuda")
+        if call == "stacked":
+            KS, VS, QS = torch.cat(Ks, 0), torch.cat(Vs, 0), torch.cat(Qs, 0)
+            KwS = torch.cat(Kws, 0) if args.windowed else None
+            wsS = jq.new_workspace(sS)
+
+            def step():
+                if args.windowed:
+                    jq.evict_layer_windowed(KS, VS, QS, KwS, sS, KoS, VoS, idxS, wsS, stream=stream)
+                else:
+                    jq.evict_layer(KS, VS, QS, sS, KoS, VoS, idxS, wsS, stream=stream)
+        elif call == "layers":
+            wsL = jq.new_layers_workspace(s, layers)
+
+            def step():
+                jq.evict_layers(Ks, Vs, Qs, s, KoS, VoS, idxS, wsL, stream=stream)
+        else:
+            step = step_per_layer
+
     n0 = jq.launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(args.steps):
-        step()
-    e1.record(stream)
-    barrier()
-    ms = e0.elapsed_time(e1)
+    total_ms, per_step, clocks = timer.run(step, args.steps, warmup=max(args.warmup, 3))
     launches = jq.launch_count() - n0
     assert jq.last_device_status(ws) == jq.JQ_OK, "device status not ok"
-    if one_call:
-        assert jq.last_device_status(wsL if args.call == "layers" else wsS) == jq.JQ_OK, "device status not ok"
-        # the same work as one call per layer, for comparison (and its results must be the same bits)
-        for _ in range(3):
-            step_per_layer()
-        barrier()
-        e0.record(stream)
-        for _ in range(max(args.steps // 4, 3)):
-            step_per_layer()
-        e1.record(stream)
-        barrier()
-        ms_pl = e0.elapsed_time(e1) / max(args.steps // 4, 3)
-        jlast = (layers - 1) % distinct
-        assert torch.equal(idx, idxS[(layers - 1) * wl.Hkv:]) and torch.equal(Ko, KoS[(layers - 1) * wl.Hkv:]), \
-            "stacked call and per-layer call disagree"
-        per_layer_calls = {"ms_per_layer": ms_pl / layers, "value": world * wl.L / (ms_pl * 1e-3 / layers), "unit": UNIT}
-    else:
-        per_layer_calls = None
-
-    # per-stage times through the stage entry points: batches of back-to-back calls between events on the
-    # launching stream, so that host launch latency is not counted as device time
-    scores = [torch.empty((wl.Hkv, wl.L), dtype=torch.float32, device="cuda") for _ in range(min(distinct, 4))]
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-    nb = max(distinct, 8)
-    stage_ms = np.zeros(3)
-
-    def timed(fn):
-        for j in range(3):
-            fn(j % distinct)
-        torch.cuda.synchronize()
-        ev[0].record(stream)
-        for j in range(nb):
-            fn(j % distinct)
-        ev[1].record(stream)
-        torch.cuda.synchronize()
-        return ev[0].elapsed_time(ev[1]) / nb
-
-    if one_call:
-        scoresS = torch.empty((sS.Hkv, wl.L), dtype=torch.float32, device="cuda")
-        nb = 4
-        if args.windowed:
-            stage_ms[0] = timed(lambda j: jq.score_windowed(KS, QS, KwS, sS, scoresS, wsS, stream=stream)) / layers
-        else:
-            stage_ms[0] = timed(lambda j: jq.score(KS, QS, sS, scoresS, wsS, stream=stream)) / layers
-        stage_ms[1] = timed(lambda j: jq.select_topk(scoresS, sS, idxS, wsS, stream=stream)) / layers
-        stage_ms[2] = timed(lambda j: jq.compact_kv(KS, VS, idxS, sS, KoS, VoS, stream=stream)) / layers
-    else:
-        if args.windowed:
-            stage_ms[0] = timed(lambda j: jq.score_windowed(Ks[j], Qs[j], Kws[j], s, scores[j % len(scores)], ws, stream=stream))
-        else:
-            stage_ms[0] = timed(lambda j: jq.score(Ks[j], Qs[j], s, scores[j % len(scores)], ws, stream=stream))
-        stage_ms[1] = timed(lambda j: jq.select_topk(scores[j % len(scores)], s, idx, ws, stream=stream))
-        stage_ms[2] = timed(lambda j: jq.compact_kv(Ks[j], Vs[j], idx, s, Ko, Vo, stream=stream))
-    clocks = sampler.stop() if sampler else None
-
-    ms = max_over_ranks(ms, world)
+    ms = max_over_ranks(total_ms, world)
     t_layer = ms * 1e-3 / (args.steps * layers)
-    value = job_value(wl, world, t_layer)
+    value = world * tokens_per_layer / t_layer
+
+    per_layer_calls = host_us = None
+    if one_call:
+        one_ws = wsR if ragged else (wsL if call == "layers" else wsS)
+        assert jq.last_device_status(one_ws) == jq.JQ_OK, "device status not ok"
+        # the same work as one call per layer, for comparison (and its results must be the same bits)
+        n_pl = max(args.steps // 4, 3)
+        tot_pl, _, _ = timer.run(step_per_layer, n_pl)
+        if ragged:
+            last = rows - wl.Hkv * nkeep
+            same = torch.equal(idx.reshape(-1), idxR[last:]) and torch.equal(Ko.reshape(-1, wl.d), KoR[last:])
+        else:
+            same = torch.equal(idx, idxS[(layers - 1) * wl.Hkv:]) and torch.equal(Ko, KoS[(layers - 1) * wl.Hkv:])
+        assert same, "the one-call path and the per-layer calls disagree"
+        per_layer_calls = {"ms_per_layer": tot_pl / n_pl / layers, "value": world * wl.L / (tot_pl * 1e-3 / n_pl / layers), "unit": UNIT,
+                           "workload": wl.name}
+        # host time of a call: calls issued back to back into an empty stream, no synchronisation in between
+        host_us = {}
+        for name, fn, n in (("jq_evict_layer", lambda: jq.evict_layer(Ks[0], Vs[0], Qs[0], s, Ko, Vo, idx, ws, stream=stream), 16), (CALLS and ("jq_evict_ragged" if ragged else "jq_evict_layers" if call == "layers" else "jq_evict_layer (stacked)"), step, 3)):
+            fn(); torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(n):
+                fn()
+            host_us[name] = (time.perf_counter() - t0) / n * 1e6
+            torch.cuda.synchronize()
+
+    # per-stage times through the stage entry points, each stage for about half a second so that the clock sampler sees
+    # the clock it runs at (short bursts run at a higher clock than the long timed loop)
+    stage = {}
+    if ragged:
+        sT, KT, VT, QT = s, Ks[0], Vs[0], Qs[0]                                  # one layer of the longest sequence
+        per_launch, wsT, idxT, KoT, VoT = 1, ws, idx, Ko, Vo
+    elif one_call:
+        sT = sS
+        KT, VT, QT = (KS, VS, QS) if call == "stacked" else (torch.cat(Ks, 0), torch.cat(Vs, 0), torch.cat(Qs, 0))
+        per_launch, wsT, idxT, KoT, VoT = layers, (wsS if call == "stacked" else jq.new_workspace(sS)), idxS, KoS, VoS
+        if args.windowed:
+            KwT = KwS
+    else:
+        sT, KT, VT, QT = s, Ks[0], Vs[0], Qs[0]
+        per_launch, wsT, idxT, KoT, VoT = 1, ws, idx, Ko, Vo
+        if args.windowed:
+            KwT = Kws[0]
+    scoresT = torch.empty((sT.Hkv, wl.L), dtype=torch.float32, device="cuda")
+    if args.windowed:
+        f_score = lambda: jq.score_windowed(KT, QT, KwT, sT, scoresT, wsT, stream=stream)
+    else:
+        f_score = lambda: jq.score(KT, QT, sT, scoresT, wsT, stream=stream)
+    for name, fn in (("score", f_score), ("select", lambda: jq.select_topk(scoresT, sT, idxT, wsT, stream=stream)),
+                     ("compact", lambda: jq.compact_kv(KT, VT, idxT, sT, KoT, VoT, stream=stream))):
+        tot, per, ck = timer.run(fn, 4, min_seconds=0.4 if name == "score" else 0.15)
+        m = tot / len(per) / per_launch
+        stage[name] = {"ms_per_layer": m, "sm_mhz": ck and ck["sm_mhz"], "kcycles_per_layer": kcycles(m, ck)}
+    stage_ms = [stage[k]["ms_per_layer"] for k in ("score", "select", "compact")]
+
+    # the second cache the target names (32K keys, 128 query rows per KV head), in the same run: 32 layers, one call
+    secondary = None
+    if args.workload == "cfg5" and not args.no_secondary and not args.windowed:
+        for t in ("KS", "VS", "QS", "KT", "VT", "QT", "scoresT"):
+            locals().pop(t, None)
+        KT = VT = QT = scoresT = None
+        torch.cuda.empty_cache()
+        secondary = one_call_cache(W.CFG3 if not args.budget else W.CFG3.with_budget(args.budget), W.CFG3.layers, 8, rank,
+                                   max(args.steps, 20), min_seconds=0.3)
 
     # the CUDA-core comparator of the scoring step (optional, outside the metric): same two passes with fp32 FMAs
     fma_cmp = None
     if args.fma_compare:
-        nb = 8
-        t_tc = timed(lambda j: jq.score(Ks[j], Qs[j], s, scores[j % len(scores)], ws, stream=stream))
-        t_fma = timed(lambda j: jq.score(Ks[j], Qs[j], s, scores[j % len(scores)], ws, fma=True, stream=stream))
+        sc1 = torch.empty((wl.Hkv, wl.L), dtype=torch.float32, device="cuda")
+        t_tc = timer.run(lambda: jq.score(Ks[0], Qs[0], s, sc1, ws, stream=stream), 8)[0] / 8
+        t_fma = timer.run(lambda: jq.score(Ks[0], Qs[0], s, sc1, ws, fma=True, stream=stream), 8)[0] / 8
         fma_cmp = {"what": "jq_score (tcgen05) against jq_score_fma (CUDA cores), one layer per call",
                    "ms_per_layer_tensor": float(t_tc), "ms_per_layer_fma": float(t_fma), "ratio": float(t_fma / t_tc)}
+
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        with open(peaks_path) as f:
+            peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = 6650.0, "fallback"
 
     # the step after the pass (optional, outside the metric): one decoding position over the pruned cache of a layer
     decode = None
@@ -399,8 +497,11 @@ def run_ours(args):
         g1.record()
         torch.cuda.synchronize()
         t_dec = g0.elapsed_time(g1) / (4 * 32)
+        dec_bytes = 2.0 * wl.Hkv * nkeep * wl.d * 2
         decode = {"what": "jq_decode_attention over one layer's pruned cache (1 launch)", "n": nkeep, "ms_per_layer": float(t_dec),
-                  "cache_gbs": 2.0 * wl.Hkv * nkeep * wl.d * 2 / (t_dec * 1e-3) / 1e9}
+                  "roofline": {"bound": "hbm", "kernel": "decode_step", "achieved": dec_bytes / (t_dec * 1e-3) / 1e9, "peak": peak,
+                               "peak_source": peak_src, "unit": "GB/s", "frac": dec_bytes / (t_dec * 1e-3) / 1e9 / peak,
+                               "bytes_per_launch": dec_bytes, "traffic": None}}
 
     # end to end through the host-buffer entry point: pinned host tensors in, pinned host results out
     e2e = None
@@ -412,45 +513,35 @@ def run_ours(args):
         hidx = torch.zeros((wl.Hkv, nkeep), dtype=torch.int32).pin_memory()
         buf = torch.empty(jq.host_call_bytes(s), dtype=torch.uint8, device="cuda")
         e2e_layers = 2
+
+        def step_e2e():
+            for _ in range(e2e_layers):
+                jq.evict_layer_host(hK, hV, hQ, s, hKo, hVo, hidx, buf, stream=stream)
         n_e2e = max(3, min(args.steps, 10))
-        for _ in range(2):
-            jq.evict_layer_host(hK, hV, hQ, s, hKo, hVo, hidx, buf, stream=stream)
-        barrier()
-        e0.record(stream)
-        for _ in range(n_e2e * e2e_layers):
-            jq.evict_layer_host(hK, hV, hQ, s, hKo, hVo, hidx, buf, stream=stream)
-        e1.record(stream)
-        barrier()
-        t_e2e_layer = max_over_ranks(e0.elapsed_time(e1), world) * 1e-3 / (n_e2e * e2e_layers)
+        tot, _, _ = timer.run(step_e2e, n_e2e, warmup=2)
+        t_e2e_layer = max_over_ranks(tot, world) * 1e-3 / (n_e2e * e2e_layers)
         # K and the queries are copied whole; of V (page-locked) only the kept rows cross, read in place by the kernel
         h2d = e2e_layers * (hK.numel() + hQ.numel() + hVo.numel()) * 2
         d2h = e2e_layers * (2 * hKo.numel() * 2 + hidx.numel() * 4)
         e2e = {"value": world * wl.L / t_e2e_layer, "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "layers_per_step": e2e_layers, "ms_per_layer": t_e2e_layer * 1e3}
+               "d2h_bytes_per_step": d2h, "layers_per_step": e2e_layers, "ms_per_layer": t_e2e_layer * 1e3, "workload": wl.name}
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        with open(peaks_path) as f:
-            peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured"
-    else:
-        peak, peak_src = 6650.0, "fallback"
     # dominant kernel: score_fused (jq_score, both passes); algorithmic bytes = two reads of K.  One launch
     # covers one layer, or all stacked layers of the step.
-    per_launch = layers if one_call else 1
     score_bytes = 2 * wl.Hkv * wl.L * wl.d * 2 * per_launch
     ms_launch = float(stage_ms[0]) * per_launch
     achieved = score_bytes / (ms_launch * 1e-3) / 1e9
-    layer_gbs = W.formula_bytes(wl) / t_layer / 1e9
-    # DRAM bytes of one score_fused launch on ONE layer of this workload from an ncu capture of the kernel
-    # as it stands (profiles/), scaled to the launch by the layers it covers; None where no capture exists
+    layer_gbs = bytes_per_layer / t_layer / 1e9
     traffic_one_layer = NCU_DRAM_BYTES_PER_LAYER.get(wl.name)
     n_exp = 2.0 * wl.R * wl.L * wl.Hkv * per_launch                      # exponentials per launch
-    ex2_peak = 148 * 16 * 1965e6 / 1e9                                   # G/s: 16 results per clock per SM at the maximum SM clock
+    ex2_peak = 148 * 16 * SM_MAX_MHZ * 1e6 / 1e9                         # G/s: 16 results per clock per SM at the maximum SM clock
+    step_kc = kcycles(ms / args.steps / layers, clocks)
+    stage_kc = [stage[k]["kcycles_per_layer"] for k in ("score", "select")]
     roofline = {"bound": "hbm", "kernel": "score_fused (jq_score, pass 1 + pass 2)", "achieved": achieved, "peak": peak,
                 "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None if traffic_one_layer is None else traffic_one_layer * per_launch,
@@ -460,16 +551,26 @@ def run_ours(args):
                 "ex2_unit": {"note": "the unit that binds this kernel (DRAM is below a quarter of its peak under ncu)",
                              "achieved": n_exp / (ms_launch * 1e-3) / 1e9, "peak": ex2_peak, "unit": "Gexp/s",
                              "frac": n_exp / (ms_launch * 1e-3) / 1e9 / ex2_peak},
-                "stage_ms_per_layer": {"score": float(stage_ms[0]), "select": float(stage_ms[1]), "compact": float(stage_ms[2])}}
+                "stage_ms_per_layer": {k: float(stage[k]["ms_per_layer"]) for k in stage},
+                "stages": stage,
+                "clock_normalised": {"what": "thousands of SM cycles per layer = time x SM MHz sampled while that loop ran",
+                                     "step": step_kc, "score": stage_kc[0], "select": stage_kc[1],
+                                     "stages_over_step": None if None in (step_kc, stage_kc[0], stage_kc[1]) or ragged else (stage_kc[0] + stage_kc[1]) / step_kc}}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "ms_per_step_median": float(np.median(per_step)),
+            "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": dict(config_of(wl, layers, distinct, args.call),
+            "config": dict(config_of(wl, layers, distinct, call),
                            softmax=("prefix keys and the causal window keys" if args.windowed else "prefix keys only")),
-            "ms_per_layer": t_layer * 1e3,
-            "per_layer_calls": per_layer_calls,
-            "tokens_discarded_per_s": world * (wl.L - nkeep) / t_layer,
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline}
+            "ms_per_layer": t_layer * 1e3, "ms_per_layer_median": float(np.median(per_step)) / layers,
+            "per_layer_calls": per_layer_calls, "host_us_per_call": host_us,
+            "tokens_discarded_per_s": world * (tokens_per_layer - (sum(w.nkeep for w in seqs) if ragged else nkeep)) / t_layer,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "secondary": secondary}
+    if ragged:
+        line["config"].update(workload="cfg4-mistral7b-ragged-batch", L=[w.L for w in seqs], sequences=len(seqs),
+                              tokens_per_layer=tokens_per_layer, units_per_call=len(RK),
+                              l2="inputs larger than L2 (K of one step: %.0f MiB)" % (layers * tokens_per_layer * wl.Hkv * wl.d * 2 / 2**20),
+                              note="stage times, per-layer calls and e2e are those of the longest sequence (L = %d)" % wl.L)
     if decode is not None:
         line["decode_step"] = decode
     if fma_cmp is not None:

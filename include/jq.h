@@ -165,17 +165,36 @@ jq_status jq_evict_layer(const void *K, const void *V, const void *Qwin, const j
                          jq_stream_t stream);
 
 /*
- * jq_evict_layer over nlayers layers of one shape whose K, V and Qwin live in buffers of their own (the usual
- * layout of a cache): one call, two launches, the same results as nlayers calls of jq_evict_layer.  (Heads are
- * independent units of the pass, so the layers are scored and selected as nlayers x Hkv heads; this is the
- * fastest way to evict a whole cache after a prefill.)
- * K, V, Qwin: HOST arrays of nlayers DEVICE pointers, each as jq_evict_layer takes it for `layer`; read before
- * the call returns.  Kout, Vout: device, bf16 [nlayers * Hkv, nkeep, d]; kept_idx: device [nlayers * Hkv, nkeep]
- * (layer l at rows l * Hkv ...).  ws: as for jq_evict_layer but of jq_layers_workspace_bytes(layer, nlayers)
- * bytes (0 for arguments the call would reject), its first 256 bytes initialised by jq_workspace_init.
- * nlayers <= 128 and nlayers * Hkv <= 65535, else JQ_ERR_UNSUPPORTED.  The call copies its small tables (tensor
- * maps, base pointers) from ordinary host memory to the device on `stream`, so it cannot be captured into a
- * CUDA graph; capture nlayers calls of jq_evict_layer, or one on a stacked tensor, instead.
+ * The pass over several units in ONE call of two launches.  A unit is a layer of a cache, or a layer of one
+ * sequence of a batch: K, V [Hkv, L_u, d] and Qwin [Hq, w, d] in buffers of its own, with a prefix length L_u
+ * and a budget B_u of its own; all units share the head geometry of `common` (Hkv, Hq, group, d, w, pool).
+ * (Every (unit, KV head) is an independent instance of the pass of the inference section; lengths that differ
+ * are the 4K-32K contexts of the paper's length sweeps, budgets that differ per layer are the layer-wise
+ * schedule its experimental-setting paragraph describes for one of the compared methods.)  The results are
+ * those of one jq_evict_layer call per unit, bit for bit.
+ *   K, V, Qwin: HOST arrays of nunits DEVICE pointers, each as jq_evict_layer takes it for unit u;
+ *   L, budget:  HOST arrays of nunits ints, or NULL for "common->L / common->budget for every unit"
+ *               (the corresponding field of `common` is ignored when the array is given);
+ *   all five arrays are only read before the call returns;
+ *   Kout, Vout: device, bf16 [rows, d];  kept_idx: device int32 [rows], where unit u's block of
+ *               Hkv * nkeep_u rows (head-major, as jq_evict_layer writes them), nkeep_u = min(B_u, L_u),
+ *               starts at row sum_{u' < u} Hkv * nkeep_u' and rows = jq_ragged_output_rows(...);
+ *   ws: device, 256-byte aligned, at least jq_ragged_workspace_bytes(common, nunits, L) bytes (0 for arguments
+ *       the call would reject), its first 256 bytes initialised by jq_workspace_init.
+ * nunits <= 4096 and nunits * Hkv <= 65535, else JQ_ERR_UNSUPPORTED.  The call copies its tables (tensor maps,
+ * base pointers, per-head lengths and offsets) from host memory of its own to the device on `stream`, so it
+ * cannot be captured into a CUDA graph; capture calls of jq_evict_layer instead.
+ */
+size_t jq_ragged_workspace_bytes(const jq_shape *common, int nunits, const int *L);
+long long jq_ragged_output_rows(const jq_shape *common, int nunits, const int *L, const int *budget);
+jq_status jq_evict_ragged(const void *const *K, const void *const *V, const void *const *Qwin, int nunits,
+                          const jq_shape *common, const int *L, const int *budget, void *Kout, void *Vout,
+                          int32_t *kept_idx, void *ws, size_t ws_bytes, jq_stream_t stream);
+
+/*
+ * jq_evict_ragged for nlayers layers of ONE shape (the usual cache after a prefill): the same call with
+ * L = budget = NULL.  Kout, Vout: device, bf16 [nlayers * Hkv, nkeep, d]; kept_idx: device [nlayers * Hkv, nkeep]
+ * (layer l at rows l * Hkv ...).  ws: at least jq_layers_workspace_bytes(layer, nlayers) bytes.
  */
 size_t jq_layers_workspace_bytes(const jq_shape *layer, int nlayers);
 jq_status jq_evict_layers(const void *const *K, const void *const *V, const void *const *Qwin, int nlayers,
@@ -218,6 +237,27 @@ jq_status jq_hit_rate(const int32_t *cur, const int32_t *ref, int Hkv, int ncur,
 size_t jq_decode_workspace_bytes(int Hkv, int Hq, int n);
 jq_status jq_decode_attention(const void *Kc, const void *Vc, const void *q, int Hkv, int Hq, int n, float *out,
                               void *workspace, size_t workspace_bytes, jq_stream_t stream);
+
+/*
+ * Re-eviction while decoding (the paper's limitations / future-work paragraph: eviction is done once, after
+ * the prefill, and extending it to the decoding stage is left open; the pass itself is the one of the
+ * inference section, run again on the grown cache with the queries of recent positions as judges).
+ * Kc, Vc: the layer's cache, device, bf16 [Hkv, cap, d]: `cap` rows per head of which the first n_old are
+ * retained pairs.  Knew, Vnew: device, bf16 [Hkv, n_new, d], the pairs decoded since (may be NULL when
+ * n_new == 0).  Qrecent: device, bf16 [Hq, w, d], the queries that score (e.g. those of the last w decoded
+ * positions).  shape->L must equal n_old + n_new and be <= cap; shape->budget is the new size.
+ * The call appends the new rows behind the retained ones, runs the pass of jq_evict_layer over the
+ * L rows of every head, and leaves the min(budget, L) kept rows, in ascending order of their position in
+ * that concatenation, in rows [0, nkeep) of Kc and Vc; kept_idx [Hkv, nkeep] holds those positions (values
+ * below n_old are old rows).  Rows [nkeep, cap) are unspecified afterwards.  Same results as jq_evict_layer on
+ * the concatenated tensors.  ws: at least jq_append_workspace_bytes(shape) bytes (it also holds the compacted
+ * rows before they are moved to the head of the cache), first 256 bytes initialised by jq_workspace_init.
+ * Two launches and up to six strided device copies, all on `stream`.
+ */
+size_t jq_append_workspace_bytes(const jq_shape *shape);
+jq_status jq_evict_append(void *Kc, void *Vc, int cap, int n_old, const void *Knew, const void *Vnew, int n_new,
+                          const void *Qrecent, const jq_shape *shape, int32_t *kept_idx, void *ws, size_t ws_bytes,
+                          jq_stream_t stream);
 
 /*
  * Synchronises `stream` and reads the status word kernels of earlier calls left in the workspace:

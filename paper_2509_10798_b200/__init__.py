@@ -19,6 +19,8 @@ EXPORTS = (
     "jq_evict_layer_host", "jq_last_device_status", "jq_launch_count", "jq_status_string",
     "jq_score_static", "jq_score_windowed", "jq_evict_layer_windowed", "jq_hit_rate",
     "jq_decode_workspace_bytes", "jq_decode_attention", "jq_layers_workspace_bytes", "jq_evict_layers",
+    "jq_ragged_workspace_bytes", "jq_ragged_output_rows", "jq_evict_ragged",
+    "jq_append_workspace_bytes", "jq_evict_append",
 )
 
 
@@ -63,6 +65,14 @@ def lib():
         L.jq_layers_workspace_bytes.argtypes = [sp, ci]
         L.jq_layers_workspace_bytes.restype = ctypes.c_size_t
         L.jq_evict_layers.argtypes = [vp, vp, vp, ci, sp, vp, vp, vp, vp, sz, vp]
+        L.jq_ragged_workspace_bytes.argtypes = [sp, ci, vp]
+        L.jq_ragged_workspace_bytes.restype = ctypes.c_size_t
+        L.jq_ragged_output_rows.argtypes = [sp, ci, vp, vp]
+        L.jq_ragged_output_rows.restype = ctypes.c_longlong
+        L.jq_evict_ragged.argtypes = [vp, vp, vp, ci, sp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.jq_append_workspace_bytes.argtypes = [sp]
+        L.jq_append_workspace_bytes.restype = ctypes.c_size_t
+        L.jq_evict_append.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, sp, vp, vp, sz, vp]
         L.jq_hit_rate.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         L.jq_score_windowed.argtypes = [vp, vp, vp, sp, vp, vp, sz, vp]
         L.jq_evict_layer_windowed.argtypes = [vp, vp, vp, vp, sp, vp, vp, vp, vp, sz, vp]
@@ -214,6 +224,58 @@ def evict_layers(Ks, Vs, Qwins, s, Kout, Vout, kept_idx, ws, stream=None):
     _raise("jq_evict_layers",
            lib().jq_evict_layers(arr(Ks), arr(Vs), arr(Qwins), n, ctypes.byref(s), _ptr(Kout), _ptr(Vout), _ptr(kept_idx),
                                  _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def _ints(xs):
+    return None if xs is None else (ctypes.c_int * len(xs))(*[int(x) for x in xs])
+
+
+def ragged_workspace_bytes(s, nunits, L=None):
+    return int(lib().jq_ragged_workspace_bytes(ctypes.byref(s), int(nunits), _ints(L)))
+
+
+def ragged_output_rows(s, nunits, L=None, budget=None):
+    return int(lib().jq_ragged_output_rows(ctypes.byref(s), int(nunits), _ints(L), _ints(budget)))
+
+
+def new_ragged_workspace(s, nunits, L=None, device="cuda", stream=None):
+    """Allocates and initialises a workspace tensor (uint8) for evict_ragged on nunits units of geometry `s`."""
+    torch = _torch()
+    n = ragged_workspace_bytes(s, nunits, L)
+    if n == 0:
+        raise JqError("jq_ragged_workspace_bytes", check_shape(s) or JQ_ERR_UNSUPPORTED)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    _raise("jq_workspace_init", lib().jq_workspace_init(_ptr(ws), ws.numel(), _stream(stream)))
+    return ws
+
+
+def evict_ragged(Ks, Vs, Qwins, s, L, budget, Kout, Vout, kept_idx, ws, stream=None):
+    """jq_evict_ragged: Ks, Vs, Qwins are lists of per-unit CUDA tensors; L, budget lists of ints (or None for
+    s.L / s.budget everywhere); the outputs hold the units' blocks of Hkv * nkeep_u rows one after the other."""
+    n = len(Ks)
+    arr = lambda ts: (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
+    _raise("jq_evict_ragged",
+           lib().jq_evict_ragged(arr(Ks), arr(Vs), arr(Qwins), n, ctypes.byref(s), _ints(L), _ints(budget), _ptr(Kout),
+                                 _ptr(Vout), _ptr(kept_idx), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def new_append_workspace(s, device="cuda", stream=None):
+    torch = _torch()
+    n = int(lib().jq_append_workspace_bytes(ctypes.byref(s)))
+    if n == 0:
+        raise JqError("jq_append_workspace_bytes", check_shape(s) or JQ_ERR_UNSUPPORTED)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    _raise("jq_workspace_init", lib().jq_workspace_init(_ptr(ws), ws.numel(), _stream(stream)))
+    return ws
+
+
+def evict_append(Kc, Vc, n_old, Knew, Vnew, Qrecent, s, kept_idx, ws, stream=None):
+    """jq_evict_append: Kc, Vc [Hkv, cap, d] hold n_old retained rows per head; Knew, Vnew [Hkv, n_new, d] are appended and
+    the cache is evicted again to s.budget rows (s.L = n_old + n_new), in place."""
+    n_new = 0 if Knew is None else int(Knew.shape[1])
+    _raise("jq_evict_append",
+           lib().jq_evict_append(_ptr(Kc), _ptr(Vc), int(Kc.shape[1]), int(n_old), _ptr(Knew), _ptr(Vnew), n_new, _ptr(Qrecent),
+                                 ctypes.byref(s), _ptr(kept_idx), _ptr(ws), ws.numel(), _stream(stream)))
 
 
 def decode_workspace_bytes(Hkv, Hq, n):

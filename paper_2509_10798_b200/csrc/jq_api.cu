@@ -1,6 +1,7 @@
 // The C ABI: argument validation, workspace carve-up, stage sequencing.  See include/jq.h.
 #include "jq_internal.cuh"
 #include <atomic>
+#include <vector>
 
 namespace jq {
 
@@ -149,56 +150,186 @@ jq_status jq_evict_layer(const void *K, const void *V, const void *Qwin, const j
     return launch_select(w.scores, *s, kept_idx, nullptr, w, st, K, V, Kout, Vout);   // selects, then copies the kept rows
 }
 
-// The shape of nlayers layers of shape `layer` stacked along the KV-head axis.
-static jq_status stacked_shape(const jq_shape *layer, int nlayers, jq_shape *out)
+// ---- units of one head geometry in buffers of their own: lengths, budgets and offsets per unit
+
+namespace {
+
+struct RaggedPlan {
+    jq_shape S;                 // head geometry with the total head count (L = longest prefix, budget = largest nkeep)
+    size_t keys = 0;            // sum over units of Hkv * L
+    long long rows = 0;         // sum over units of Hkv * nkeep
+    int max_L = 0;
+};
+
+// Validates the arguments the two ragged entry points share and sums the sizes.  L and budget may be NULL
+// (then every unit has common->L / common->budget).
+jq_status plan_ragged(const jq_shape *common, int nunits, const int *L, const int *budget, RaggedPlan *out)
 {
-    jq_status rc = check_shape(layer);
+    if (!common) return JQ_ERR_INVALID_ARG;
+    if (nunits < 1) return JQ_ERR_INVALID_ARG;
+    if (nunits > kMaxUnits) return JQ_ERR_UNSUPPORTED;
+    RaggedPlan pl;
+    int max_keep = 0;
+    for (int u = 0; u < nunits; ++u) {
+        jq_shape su = *common;
+        if (L) su.L = L[u];
+        if (budget) su.budget = budget[u];
+        const jq_status rc = check_shape(&su);
+        if (rc != JQ_OK) return rc;
+        const int nkeep = su.budget < su.L ? su.budget : su.L;
+        pl.keys += (size_t)su.Hkv * su.L;
+        pl.rows += (long long)su.Hkv * nkeep;
+        if (su.L > pl.max_L) pl.max_L = su.L;
+        if (nkeep > max_keep) max_keep = nkeep;
+    }
+    if ((long long)common->Hkv * nunits > 65535) return JQ_ERR_UNSUPPORTED;
+    pl.S = *common;
+    pl.S.Hkv = common->Hkv * nunits;
+    pl.S.Hq = common->Hq * nunits;
+    pl.S.L = pl.max_L;
+    pl.S.budget = max_keep;
+    *out = pl;
+    return JQ_OK;
+}
+
+}  // namespace
+
+size_t jq_ragged_workspace_bytes(const jq_shape *common, int nunits, const int *L)
+{
+    RaggedPlan pl;
+    if (plan_ragged(common, nunits, L, nullptr, &pl) != JQ_OK) return 0;
+    return carve(nullptr, (size_t)pl.S.Hkv, (size_t)common->group * common->w, pl.keys).bytes + unit_tables_bytes(nunits, common->Hkv);
+}
+
+long long jq_ragged_output_rows(const jq_shape *common, int nunits, const int *L, const int *budget)
+{
+    RaggedPlan pl;
+    if (plan_ragged(common, nunits, L, budget, &pl) != JQ_OK) return 0;
+    return pl.rows;
+}
+
+jq_status jq_evict_ragged(const void *const *K, const void *const *V, const void *const *Qwin, int nunits,
+                          const jq_shape *common, const int *L, const int *budget, void *Kout, void *Vout,
+                          int32_t *kept_idx, void *ws, size_t ws_bytes, jq_stream_t stream)
+{
+    RaggedPlan pl;
+    jq_status rc = plan_ragged(common, nunits, L, budget, &pl);
     if (rc != JQ_OK) return rc;
-    if (nlayers < 1) return JQ_ERR_INVALID_ARG;
-    if (nlayers > kMaxLayers) return JQ_ERR_UNSUPPORTED;
-    *out = *layer;
-    out->Hkv = layer->Hkv * nlayers;
-    out->Hq = layer->Hq * nlayers;
-    return check_shape(out);
+    if (!K || !V || !Qwin || !aligned16(Kout) || !aligned16(Vout) || !aligned16(kept_idx)) return JQ_ERR_INVALID_ARG;
+    for (int u = 0; u < nunits; ++u)
+        if (!aligned16(K[u]) || !aligned16(V[u]) || !aligned16(Qwin[u])) return JQ_ERR_INVALID_ARG;
+    if (!aligned16(ws) || ((uintptr_t)ws & 255u)) return JQ_ERR_INVALID_ARG;
+    const int hpu = common->Hkv, R = common->group * common->w;
+    const Workspace w = carve(ws, (size_t)pl.S.Hkv, (size_t)R, pl.keys);
+    const size_t tab_bytes = unit_tables_bytes(nunits, hpu);
+    if (ws_bytes < w.bytes + tab_bytes) return JQ_ERR_WORKSPACE;
+    const int sms = score_sms();
+    if (sms < 1) return JQ_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    // All tables are assembled in one host buffer of the library's own (so that the caller's arrays are only read
+    // before the call returns, whatever memory they live in) and go to the device in one copy.
+    static thread_local std::vector<unsigned char> staging;
+    staging.assign(tab_bytes, 0);
+    unsigned char *hb = staging.data();
+    const size_t maps_bytes = align_up((size_t)nunits * 2 * kTensorMapBytes, 256), ptr_bytes = align_up((size_t)nunits * sizeof(void *), 256);
+    const size_t grp_bytes = align_up((size_t)nunits * hpu * sizeof(GroupRec), 256);
+    unsigned char *h_maps = hb;
+    const void **h_K = (const void **)(hb + maps_bytes), **h_V = (const void **)(hb + maps_bytes + ptr_bytes);
+    GroupRec *h_grp = (GroupRec *)(hb + maps_bytes + 2 * ptr_bytes);
+    HeadRec *h_head = (HeadRec *)(hb + maps_bytes + 2 * ptr_bytes + grp_bytes);
+    UnitTables t;
+    long long soff = 0, ooff = 0;
+    int ngroups = 0;
+    for (int u = 0; u < nunits; ++u) {
+        const int Lu = L ? L[u] : common->L, Bu = budget ? budget[u] : common->budget;
+        const int nkeep = Bu < Lu ? Bu : Lu, tph = (Lu + 127) / 128;
+        if (!make_tensor_map(h_maps + (size_t)(2 * u) * kTensorMapBytes, K[u], Lu, hpu, 128) ||
+            !make_tensor_map(h_maps + (size_t)(2 * u + 1) * kTensorMapBytes, Qwin[u], R, hpu, R <= 128 ? 128 : 256))
+            return JQ_ERR_CUDA;
+        h_K[u] = K[u]; h_V[u] = V[u];
+        const int hpg = heads_per_group(Lu, hpu, tph, sms);
+        for (int h0 = 0; h0 < hpu; h0 += hpg) {
+            GroupRec &g = h_grp[ngroups++];
+            g.h0 = u * hpu + h0; g.nh = h0 + hpg <= hpu ? hpg : hpu - h0;
+            g.tph = tph; g.L = Lu; g.unit = u; g.c20 = h0;
+            g.sbase = soff + (long long)h0 * Lu;
+            if (g.nh * tph > t.max_group_tiles) t.max_group_tiles = g.nh * tph;
+        }
+        for (int h = 0; h < hpu; ++h) {
+            HeadRec &r = h_head[u * hpu + h];
+            r.L = Lu; r.nkeep = nkeep; r.unit = u; r.kv_in = h;
+            r.soff = soff + (long long)h * Lu;
+            r.ooff = ooff + (long long)h * nkeep;
+        }
+        soff += (long long)hpu * Lu;
+        ooff += (long long)hpu * nkeep;
+    }
+    char *tab = (char *)ws + w.bytes;
+    if (cudaMemcpyAsync(tab, hb, tab_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
+    t.maps = tab;
+    t.K = (const void *const *)(tab + maps_bytes);
+    t.V = (const void *const *)(tab + maps_bytes + ptr_bytes);
+    t.groups = (const GroupRec *)(tab + maps_bytes + 2 * ptr_bytes);
+    t.heads = (const HeadRec *)(tab + maps_bytes + 2 * ptr_bytes + grp_bytes);
+    t.ngroups = ngroups; t.hpu = hpu; t.max_L = pl.max_L;
+    if ((rc = launch_score_tc(nullptr, nullptr, pl.S, w.scores, w, st, nullptr, &t)) != JQ_OK) return rc;
+    return launch_select(w.scores, pl.S, kept_idx, nullptr, w, st, nullptr, nullptr, Kout, Vout, &t);
 }
 
 size_t jq_layers_workspace_bytes(const jq_shape *layer, int nlayers)
 {
-    jq_shape S;
-    if (stacked_shape(layer, nlayers, &S) != JQ_OK) return 0;
-    return carve(nullptr, S).bytes + layer_tables_bytes(nlayers);
+    return jq_ragged_workspace_bytes(layer, nlayers, nullptr);
 }
 
 jq_status jq_evict_layers(const void *const *K, const void *const *V, const void *const *Qwin, int nlayers,
                           const jq_shape *layer, void *Kout, void *Vout, int32_t *kept_idx, void *ws, size_t ws_bytes,
                           jq_stream_t stream)
 {
-    jq_shape S;
-    jq_status rc = stacked_shape(layer, nlayers, &S);
+    return jq_evict_ragged(K, V, Qwin, nlayers, layer, nullptr, nullptr, Kout, Vout, kept_idx, ws, ws_bytes, stream);
+}
+
+// ---- streaming re-eviction: the pruned cache of a layer has grown during decoding
+
+size_t jq_append_workspace_bytes(const jq_shape *s)
+{
+    if (check_shape(s) != JQ_OK) return 0;
+    const size_t nkeep = (size_t)(s->budget < s->L ? s->budget : s->L);
+    return carve(nullptr, *s).bytes + 2 * align_up((size_t)s->Hkv * nkeep * s->d * 2, 256);
+}
+
+jq_status jq_evict_append(void *Kc, void *Vc, int cap, int n_old, const void *Knew, const void *Vnew, int n_new,
+                          const void *Qrecent, const jq_shape *s, int32_t *kept_idx, void *ws, size_t ws_bytes,
+                          jq_stream_t stream)
+{
+    jq_status rc = check_shape(s);
     if (rc != JQ_OK) return rc;
-    if (!K || !V || !Qwin || !aligned16(Kout) || !aligned16(Vout) || !aligned16(kept_idx)) return JQ_ERR_INVALID_ARG;
-    for (int l = 0; l < nlayers; ++l)
-        if (!aligned16(K[l]) || !aligned16(V[l]) || !aligned16(Qwin[l])) return JQ_ERR_INVALID_ARG;
-    if (!aligned16(ws) || ((uintptr_t)ws & 255u)) return JQ_ERR_INVALID_ARG;
-    const Workspace w = carve(ws, S);
-    if (ws_bytes < w.bytes + layer_tables_bytes(nlayers)) return JQ_ERR_WORKSPACE;
+    if (n_old < 0 || n_new < 0 || cap < 1 || (long long)n_old + n_new != (long long)s->L || s->L > cap) return JQ_ERR_INVALID_ARG;
+    if (!aligned16(Kc) || !aligned16(Vc) || !aligned16(Qrecent) || !aligned16(kept_idx)) return JQ_ERR_INVALID_ARG;
+    if (n_new > 0 && (!aligned16(Knew) || !aligned16(Vnew))) return JQ_ERR_INVALID_ARG;
+    Workspace w;
+    if ((rc = check_ws(s, ws, ws_bytes, &w)) != JQ_OK) return rc;
+    if (ws_bytes < jq_append_workspace_bytes(s)) return JQ_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
-    // tables behind the workspace proper: tensor maps, then the K and the V base pointers
-    char *tab = (char *)ws + w.bytes;
-    const size_t maps_bytes = align_up((size_t)nlayers * 2 * kTensorMapBytes, 256), ptr_bytes = align_up((size_t)nlayers * sizeof(void *), 256);
-    alignas(64) unsigned char host_maps[kMaxLayers * 2 * kTensorMapBytes];
-    if (!build_layer_maps(K, Qwin, nlayers, *layer, host_maps)) return JQ_ERR_CUDA;
-    // (copies from pageable host memory are staged before the call returns, so the sources may live on this stack)
-    if (cudaMemcpyAsync(tab, host_maps, (size_t)nlayers * 2 * kTensorMapBytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
-    if (cudaMemcpyAsync(tab + maps_bytes, K, (size_t)nlayers * sizeof(void *), cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
-    if (cudaMemcpyAsync(tab + maps_bytes + ptr_bytes, V, (size_t)nlayers * sizeof(void *), cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
-    LayerTables t;
-    t.maps = tab;
-    t.K = (const void *const *)(tab + maps_bytes);
-    t.V = (const void *const *)(tab + maps_bytes + ptr_bytes);
-    t.hpl = layer->Hkv;
-    if ((rc = launch_score_tc(K[0], Qwin[0], S, w.scores, w, st, nullptr, &t)) != JQ_OK) return rc;
-    return launch_select(w.scores, S, kept_idx, nullptr, w, st, nullptr, nullptr, Kout, Vout, &t);
+    const size_t row = (size_t)s->d * 2, nkeep = (size_t)(s->budget < s->L ? s->budget : s->L);
+    char *Ktmp = (char *)ws + w.bytes, *Vtmp = Ktmp + align_up((size_t)s->Hkv * nkeep * row, 256);
+    // 1. the new rows go behind the retained ones, head by head (the cache keeps `cap` rows per head)
+    if (n_new > 0) {
+        if (cudaMemcpy2DAsync((char *)Kc + (size_t)n_old * row, (size_t)cap * row, Knew, (size_t)n_new * row, (size_t)n_new * row,
+                              (size_t)s->Hkv, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
+        if (cudaMemcpy2DAsync((char *)Vc + (size_t)n_old * row, (size_t)cap * row, Vnew, (size_t)n_new * row, (size_t)n_new * row,
+                              (size_t)s->Hkv, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
+    }
+    // 2. the pass over the L = n_old + n_new rows of every head, compacted into the workspace (a row may move
+    //    onto a row that another thread still has to read, so the compaction cannot run in place)
+    if ((rc = launch_score_tc(Kc, Qrecent, *s, w.scores, w, st, nullptr, nullptr, cap)) != JQ_OK) return rc;
+    if ((rc = launch_select(w.scores, *s, kept_idx, nullptr, w, st, Kc, Vc, Ktmp, Vtmp, nullptr, cap)) != JQ_OK) return rc;
+    // 3. back to the head of the cache
+    if (cudaMemcpy2DAsync(Kc, (size_t)cap * row, Ktmp, nkeep * row, nkeep * row, (size_t)s->Hkv, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return JQ_ERR_CUDA;
+    if (cudaMemcpy2DAsync(Vc, (size_t)cap * row, Vtmp, nkeep * row, nkeep * row, (size_t)s->Hkv, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return JQ_ERR_CUDA;
+    return JQ_OK;
 }
 
 size_t jq_host_call_bytes(const jq_shape *s)

@@ -27,44 +27,72 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 // Select scratch per KV head, in 32-bit words: histograms and counters (see jq_select.cu).
 constexpr int kSelWordsPerHead = 4096 + 64;
 
-static inline Workspace carve(void *base, const jq_shape &s)
+// Carve-up of a workspace for `heads` KV heads with R query rows each and `keys` prefix positions in total
+// (heads x L for one shape; the sum over the units of a ragged call).
+static inline Workspace carve(void *base, size_t heads, size_t R, size_t keys)
 {
     Workspace w;
-    const size_t R = (size_t)s.group * s.w;
     char *p = (char *)base;
     size_t off = 0;
     w.status = (int *)(p + off);
     off += align_up(kStatusWords * sizeof(int), 256);
     w.Mrow = (float *)(p + off);
-    off += align_up((size_t)s.Hkv * R * sizeof(float), 256);
+    off += align_up(heads * R * sizeof(float), 256);
     w.part = (float2 *)(p + off);
-    off += align_up((size_t)s.Hkv * kSlots * R * sizeof(float2), 256);
+    off += align_up(heads * kSlots * R * sizeof(float2), 256);
     w.scores = (float *)(p + off);
-    off += align_up((size_t)s.Hkv * s.L * sizeof(float), 256);
+    off += align_up(keys * sizeof(float), 256);
     w.keys = (uint32_t *)(p + off);
-    off += align_up((size_t)s.Hkv * s.L * sizeof(uint32_t), 256);
+    off += align_up(keys * sizeof(uint32_t), 256);
     w.sel = (uint32_t *)(p + off);
-    off += align_up((size_t)s.Hkv * kSelWordsPerHead * sizeof(uint32_t), 256);
+    off += align_up(heads * kSelWordsPerHead * sizeof(uint32_t), 256);
     w.bytes = off;
     return w;
 }
-
-// Layers of equal shape living in buffers of their own (jq_evict_layers): tables in device memory, behind the
-// workspace proper.  KV head kv of the stacked numbering belongs to layer kv / hpl and is head kv % hpl of it.
-constexpr int kMaxLayers = 128;
-constexpr size_t kTensorMapBytes = 128;
-struct LayerTables {
-    const void *maps = nullptr;          // device: [nlayers][2] TMA tensor maps (K, Qwin)
-    const void *const *K = nullptr;      // device: [nlayers] base of K
-    const void *const *V = nullptr;      // device: [nlayers] base of V
-    int hpl = 0;                         // KV heads per layer (0: no tables, one buffer)
-};
-static inline size_t layer_tables_bytes(int nlayers)
+static inline Workspace carve(void *base, const jq_shape &s)
 {
-    return align_up((size_t)nlayers * 2 * kTensorMapBytes, 256) + 2 * align_up((size_t)nlayers * sizeof(void *), 256);
+    return carve(base, (size_t)s.Hkv, (size_t)s.group * s.w, (size_t)s.Hkv * s.L);
 }
-// Fills host_maps ([nlayers][2] tensor maps) for K[l] [hpl][L][128] and Qwin[l] [hpl][R][128].
-bool build_layer_maps(const void *const *K, const void *const *Qwin, int nlayers, const jq_shape &layer, void *host_maps);
+
+// Units (layers, sequences) of one head geometry living in buffers of their own, with prefix lengths and
+// budgets of their own (jq_evict_ragged, jq_evict_layers): tables in device memory, behind the workspace proper.
+// KV heads are numbered through all units; unit u owns heads [u * hpu, (u + 1) * hpu).
+constexpr int kMaxUnits = 4096;
+constexpr size_t kTensorMapBytes = 128;
+// A head group of the scoring kernel: consecutive KV heads of ONE unit whose keys fit a share of the L2.
+struct GroupRec {
+    int h0, nh;          // first KV head (global numbering) and number of heads
+    int tph, L;          // tiles per head, prefix length
+    int unit, c20;       // the unit, and the index of head h0 within it
+    long long sbase;     // offset (floats) of head h0's scores in the scores array
+};
+// A KV head as the selection kernel sees it.
+struct HeadRec {
+    int L, nkeep;
+    int unit, kv_in;     // the unit and the head's index within it
+    long long soff;      // offset (floats / keys) of the head's scores and select keys
+    long long ooff;      // offset (rows) of the head's kept indices and compacted rows in the stacked outputs
+};
+struct UnitTables {
+    const void *maps = nullptr;          // device: [nunits][2] TMA tensor maps (K, Qwin)
+    const void *const *K = nullptr;      // device: [nunits] base of K
+    const void *const *V = nullptr;      // device: [nunits] base of V
+    const GroupRec *groups = nullptr;    // device: [ngroups]
+    const HeadRec *heads = nullptr;      // device: [nunits * hpu]
+    int ngroups = 0, hpu = 0;            // hpu: KV heads per unit
+    int max_group_tiles = 0;             // most tiles in any group (sizes the grid)
+    int max_L = 0;                       // longest prefix (sizes the selection kernel's shared memory)
+};
+static inline size_t unit_tables_bytes(int nunits, int hpu)
+{
+    return align_up((size_t)nunits * 2 * kTensorMapBytes, 256) + 2 * align_up((size_t)nunits * sizeof(void *), 256) +
+           align_up((size_t)nunits * hpu * sizeof(GroupRec), 256) + align_up((size_t)nunits * hpu * sizeof(HeadRec), 256);
+}
+// One tensor map for a bf16 tensor [heads][rows][128], boxes of 64 columns x box_rows rows (host).
+bool make_tensor_map(void *map, const void *ptr, int rows, int heads, int box_rows);
+// Most KV heads of L keys that the scoring kernel takes as one group (tiles of a group are split over `sms` CTAs).
+int heads_per_group(int L, int heads, int tiles_per_head, int sms);
+int score_sms();   // CTAs of the scoring kernel on the current device; 0 on error
 
 // Host-side bookkeeping.
 void count_launch(int n = 1);
@@ -74,14 +102,19 @@ jq_status check_launch();   // cudaGetLastError -> JQ_OK / JQ_ERR_CUDA
 jq_status launch_score_fma(const void *K, const void *Q, const jq_shape &s, float *scores,
                            const Workspace &w, cudaStream_t st);
 // Kwin, when not null: keys [Hkv][w][128] of the query positions themselves (window-inclusive softmax).
-// With tables (s is then the stacked shape, K and Q those of the first layer) the tiles come from the layers' own buffers.
+// With tables, s holds the head geometry and the total head count (s.L, s.budget unused): tiles, lengths and
+// score offsets come from the tables, K and Q are ignored.
+// k_head_rows: rows between consecutive heads of K in memory when the heads are not packed (0: s.L).
 jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float *scores,
                           const Workspace &w, cudaStream_t st, const void *Kwin = nullptr,
-                          const LayerTables *tables = nullptr);
-// With K, V, Kout, Vout given, the kernel also copies the kept rows (the fused layer path).
+                          const UnitTables *tables = nullptr, int k_head_rows = 0);
+// With K, V, Kout, Vout given, the kernel also copies the kept rows (the fused layer path).  With tables, every
+// head has a length, a budget and offsets of its own (s.L, s.budget unused).
+// src_head_rows: rows between consecutive heads of K and V in memory when the heads are not packed (0: s.L).
 jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, float *pooled,
                         const Workspace &w, cudaStream_t st, const void *K = nullptr, const void *V = nullptr,
-                        void *Kout = nullptr, void *Vout = nullptr, const LayerTables *tables = nullptr);
+                        void *Kout = nullptr, void *Vout = nullptr, const UnitTables *tables = nullptr,
+                        int src_head_rows = 0);
 jq_status launch_gather(const void *K, const void *V, const int32_t *idx, const jq_shape &s,
                         void *Kout, void *Vout, cudaStream_t st);
 

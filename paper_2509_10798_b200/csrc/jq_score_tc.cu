@@ -46,6 +46,7 @@
 #include "jq_tmem_ld.cuh"
 #include <cuda.h>
 #include <cstddef>
+#include <cstring>
 #include <mutex>
 
 namespace jq {
@@ -106,8 +107,10 @@ struct Params {
     int *status;             // status block (kStatusWords ints)
     int wtile;               // 1 in window-inclusive mode: every head has one more tile, the last, holding the w window keys
     int w;                   // soft-token queries per query head
-    const CUtensorMap *maps; // not null: [layers][2] tensor maps (K, Qwin) of layers in buffers of their own, hpl KV heads each
-    int hpl;
+    // Units in buffers of their own (ragged calls): the head groups, their lengths and score offsets come from
+    // gtab [ngroups] (L, tph, hpg above are then unused) and the tiles through maps [units][2] (K, Qwin).
+    const GroupRec *gtab;
+    const CUtensorMap *maps;
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -301,9 +304,9 @@ __device__ __noinline__ bool cta_has_tile(uint32_t b, uint32_t T, uint32_t G) { 
 
 // ------------------------------------------------------------------ exponentials
 
-// exp2 of a pair on the FMA pipe, for x <= 0 (both passes only ever ask for that: the argument is a
-// logit minus something that is at least the row's largest).  x is clamped to >= -126 (so that the
-// exponent insertion cannot wrap; 2^-126 stands in for anything smaller), split into n = round(x) and
+// exp2 of a pair on the FMA pipe, for x < 100 (pass 1 asks for at most +64, see p1_half; pass 2 for
+// x <= 0: a logit minus the row's log-sum-exp).  x is clamped to >= -126 (so that the exponent
+// insertion cannot wrap; 2^-126 stands in for anything smaller), split into n = round(x) and
 // r = x - n in [-1/2, 1/2] by the add-a-large-constant trick, 2^r comes from a degree-4 polynomial
 // (relative error < 3e-6, a least-maximum fit of 2^r on that interval) and n is added into the
 // exponent field.
@@ -373,18 +376,23 @@ __device__ __forceinline__ float max_of16(const uint32_t (&v)[16])
     return fmaxf(c0, c1);
 }
 
-// Pass 1, 16 keys of a query row: online softmax statistics.  The reference is the running max, raised
-// (and l rescaled) when the keys bring a larger value; the max runs on the ALU pipe and, unlike a check
-// of the sum, does not wait for the exponentials in flight.  Keys at column >= valid are not keys (-inf).
+// Pass 1, 16 keys of a query row: online softmax statistics (m, l = sum_j exp2(c (s_j - m))).  Any
+// reference m gives the same row normaliser c m + log2 l as long as nothing overflows, so m is not kept
+// equal to the running max: it is raised (and l rescaled) only when the keys bring a value more than
+// `lazy` above it, lazy = 64 / c, i.e. when an exponential would pass 2^64.  A warp of 32 rows restarts
+// its statistics at every segment and would otherwise take the rescaling branch on most reads; now it
+// takes it once per segment.  (exp2 arguments reach +64 at most, l stays below 2^64 times the keys of
+// a segment: far inside fp32.)  The max runs on the ALU pipe and, unlike a check of the sum, does not
+// wait for the exponentials in flight.  Keys at column >= valid are not keys (-inf).
 struct RowState { float m; float2 l01, l23; };
-__device__ __forceinline__ void p1_half(uint32_t (&v)[16], int c0, int valid, float c, float2 cc, RowState &st)
+__device__ __forceinline__ void p1_half(uint32_t (&v)[16], int c0, int valid, float c, float lazy, float2 cc, RowState &st)
 {
     if (valid < c0 + 16) {
 #pragma unroll
         for (int t = 0; t < 16; ++t) if (c0 + t >= valid) v[t] = 0xff800000u;
     }
     const float cm = max_of16(v);
-    if (cm > st.m) {
+    if (cm > st.m + lazy) {
         const float f = ex2(c * (st.m - cm));   // 0 for the first keys (m = -inf)
         st.l01 = make_float2(st.l01.x * f, st.l01.y * f);
         st.l23 = make_float2(st.l23.x * f, st.l23.y * f);
@@ -400,7 +408,21 @@ __device__ __forceinline__ void p1_half(uint32_t (&v)[16], int c0, int valid, fl
 struct Seg {
     int pass, g, h0, ntiles;
     int kv0, t0;   // KV head and tile within the head of the first tile in walking order
+    int tph, L;    // tiles per head and prefix length of the group's heads
+    int unit, c20; // the buffer the group's heads live in and the index of head h0 within it
+    long long sbase;   // offset (floats) of head h0's scores
 };
+
+// Head group g: from the table of a ragged call, else g-th run of hpg heads of the one stacked tensor.
+__device__ __forceinline__ GroupRec group_of(int g, const Params &P)
+{
+    if (P.gtab) return P.gtab[g];
+    GroupRec r;
+    r.h0 = g * P.hpg; r.nh = min(P.hpg, P.Hkv - r.h0);
+    r.tph = P.tph; r.L = P.L; r.unit = 0; r.c20 = r.h0;
+    r.sbase = (long long)r.h0 * P.L;
+    return r;
+}
 
 // (Not inlined: five roles call it once per segment.)
 __device__ __noinline__ Seg segment(int s, const Params &P)
@@ -411,14 +433,14 @@ __device__ __noinline__ Seg segment(int s, const Params &P)
     if (s < D) { sg.pass = 1; sg.g = s; }                                  // lead-in: pass 1 of the first D groups
     else if (t < 2 * (NG - D)) { sg.pass = (t & 1) ? 1 : 2; sg.g = (t & 1) ? D + (t >> 1) : (t >> 1); }
     else { sg.pass = 2; sg.g = s - NG; }                                   // tail: the last D groups' pass 2
-    sg.h0 = sg.g * P.hpg;
-    const int nh = min(P.hpg, P.Hkv - sg.h0);
-    const uint32_t T = (uint32_t)nh * P.tph, G = gridDim.x;
+    const GroupRec r = group_of(sg.g, P);
+    sg.h0 = r.h0; sg.tph = r.tph; sg.L = r.L; sg.unit = r.unit; sg.c20 = r.c20; sg.sbase = r.sbase;
+    const uint32_t T = (uint32_t)r.nh * r.tph, G = gridDim.x;
     const uint32_t t_begin = blockIdx.x * T / G, t_end = (blockIdx.x + 1) * T / G;
     sg.ntiles = (int)(t_end - t_begin);
     const uint32_t first = (sg.pass == 1) ? t_begin : (t_end > 0 ? t_end - 1 : 0);
-    sg.kv0 = sg.h0 + (int)(first / P.tph);
-    sg.t0 = (int)(first % P.tph);
+    sg.kv0 = sg.h0 + (int)(first / r.tph);
+    sg.t0 = (int)(first % r.tph);
     return sg;
 }
 
@@ -450,7 +472,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, stages = P.stages;
-    const int tph = P.tph, L = P.L, R = P.R, Rpad = P.Rpad;   // register copies: the loops below must not touch memory for them
+    const int R = P.R, Rpad = P.Rpad;                         // register copies: the loops below must not touch memory for them
     int *const status = P.status;
     const int nblk = P.Rbox / 128;                            // accumulator blocks per tile, both passes
     const int nseg = 2 * P.ngroups;
@@ -480,23 +502,24 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             // ---------------------------------------------------------------- TMA producer
             if (lane == 0) {
                 uint32_t st = 0, ph = 0, qn = 0;                  // ring stage and its phase; query loads so far
-                int prev_kv = -1, prev_lay = -1;
+                int prev_kv = -1, prev_unit = -1;
                 const CUtensorMap *head_mapK = &mapK, *head_mapQ = &mapQ;   // maps and head coordinate of the current KV head
                 int head_c2 = 0;
                 bool ok = true;
 #pragma unroll 1
                 for (int s = 0; s < nseg && ok; ++s) {
                     const Seg sg = segment(s, P);
-                    const int pass = sg.pass, ntiles = sg.ntiles;
+                    const int pass = sg.pass, ntiles = sg.ntiles, tph = sg.tph;
                     int kv = sg.kv0, tt = sg.t0;
+                    if (P.maps && sg.unit != prev_unit && ntiles > 0) {   // the group's unit has tensor maps of its own
+                        head_mapK = P.maps + 2 * sg.unit; head_mapQ = head_mapK + 1;
+                        tensormap_acquire(head_mapK); tensormap_acquire(head_mapQ);
+                        prev_unit = sg.unit;
+                    }
 #pragma unroll 1
                     for (int n = 0; n < ntiles; ++n, walk(pass, tph, kv, tt)) {
                         if (kv != prev_kv) {
-                            if (P.maps) {                         // the head's layer has tensor maps of its own
-                                const int lay = kv / P.hpl;
-                                head_mapK = P.maps + 2 * lay; head_mapQ = head_mapK + 1; head_c2 = kv - lay * P.hpl;
-                                if (lay != prev_lay) { tensormap_acquire(head_mapK); tensormap_acquire(head_mapQ); prev_lay = lay; }
-                            } else head_c2 = kv;
+                            head_c2 = sg.c20 + (kv - sg.h0);
                             const uint32_t qb = qn & 1;
                             if (!mbar_wait(&ctl->q_empty[qb], ((qn >> 1) & 1) ^ 1, ctl, status, kSleepLong)) { ok = false; break; }
                             mbar_expect_tx(&ctl->q_full[qb], q_bytes);
@@ -528,7 +551,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll 1
             for (int s = 0; s < nseg && ok; ++s) {
                 const Seg sg = segment(s, P);
-                const int pass = sg.pass, ntiles = sg.ntiles;
+                const int pass = sg.pass, ntiles = sg.ntiles, tph = sg.tph;
                 int kv = sg.kv0, tt = sg.t0;
 #pragma unroll 1
                 for (int n = 0; n < ntiles && ok; ++n, walk(pass, tph, kv, tt)) {
@@ -575,8 +598,9 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
-                const int h0 = g * P.hpg, nh = min(P.hpg, P.Hkv - h0);
-                const uint32_t T = (uint32_t)nh * P.tph;
+                const GroupRec gr = group_of(g, P);
+                const int h0 = gr.h0, nh = gr.nh, tph = gr.tph;
+                const uint32_t T = (uint32_t)nh * tph;
                 // This CTA's rows of the group are blockIdx.x + k G.  They are taken `rows_par` at a time, each by a
                 // sub-group of 32 / rows_par lanes that splits the row's partial slots, four loads in flight per
                 // lane; an empty partial (or one of a CTA that had no tile of the head) counts as (-inf, 0).
@@ -591,8 +615,8 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     const bool have = my < nrows;
                     const int item = blockIdx.x + (have ? my : 0) * G;
                     const int hl = item / P.R, r = item - hl * P.R, kv = h0 + hl;
-                    const uint32_t first = (uint32_t)hl * P.tph;
-                    const int b_lo = owner_of_tile(first, T, Gu), b_hi = owner_of_tile(first + P.tph - 1, T, Gu);
+                    const uint32_t first = (uint32_t)hl * tph;
+                    const int b_lo = owner_of_tile(first, T, Gu), b_hi = owner_of_tile(first + tph - 1, T, Gu);
                     const int nsl = have ? (b_hi - b_lo + 1) * kGroups : 0;   // every epilogue group of a contributing CTA wrote a partial
                     const float2 *src = P.part + ((size_t)kv * kSlots + kGroups * b_lo) * P.R + r;
                     float m = -INFINITY, l = 0.f;
@@ -643,11 +667,12 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             for (int s = 0; s < nseg && ok; ++s) {
                 const Seg sg = segment(s, P);
                 if (sg.pass != 2 || sg.ntiles == 0) continue;
+                const int tph = sg.tph;
                 if (nblk == 2) {
                     int kv = sg.kv0, tt = sg.t0;
                     for (int n = 0; n < sg.ntiles; ++n, walk(2, tph, kv, tt)) {
-                        float *dst = P.scores + (size_t)kv * P.L + tt * kTile;
-                        for (int t = lane; t < kTile && tt * kTile + t < P.L; t += 32) dst[t] = 0.f;
+                        float *dst = P.scores + sg.sbase + (size_t)(kv - sg.h0) * sg.L + tt * kTile;
+                        for (int t = lane; t < kTile && tt * kTile + t < sg.L; t += 32) dst[t] = 0.f;
                     }
                     __threadfence();
                 }
@@ -679,7 +704,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
         const int row0 = quarter * 32 + lane;                   // TMEM lane: query row within its block (pass 1), key within its tile (pass 2)
         const int bs = nblk - 1;                                // blocks per tile is 1 or 2: shift and mask
-        const float c = P.c;
+        const float c = P.c, lazy = 64.f / c;
         const float2 cc = make_float2(c, c);
         float *const scores_out = P.scores;
         float2 *const part_out = P.part + (size_t)(kGroups * blockIdx.x + grp) * R;
@@ -716,7 +741,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll 1
         for (int s = 0; s < nseg && ok; ++s) {
             const Seg sg = segment(s, P);
-            const int ntiles = sg.ntiles, nunits = ntiles << bs;
+            const int ntiles = sg.ntiles, nunits = ntiles << bs, tph = sg.tph, L = sg.L;
             int kv = sg.kv0, tt = sg.t0, at = 0;                // tile cursor: head, tile in head, index in the segment
             int k = (grp + kGroups - (int)(u % kGroups)) % kGroups;   // this group's first block of the segment
             bool pre = false;                                   // the first read of block k has already been requested
@@ -754,14 +779,14 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     for (int c0 = 0; c0 < kTile; c0 += 32) {
                         JQ_TMEM_WAIT16(va);
                         JQ_TMEM_LD16(taddr + c0 + 16, vb);
-                        p1_half(va, c0, valid, c, cc, st0);
+                        p1_half(va, c0, valid, c, lazy, cc, st0);
                         JQ_TMEM_WAIT16(vb);
                         if (c0 + 32 < kTile) JQ_TMEM_LD16(taddr + c0 + 32, va);
                         else {
                             release(slot);
                             pre = (k + kGroups < nunits) && try_begin(uu + kGroups);
                         }
-                        p1_half(vb, c0 + 16, valid, c, cc, st0);
+                        p1_half(vb, c0 + 16, valid, c, lazy, cc, st0);
                     }
                     if (blk == 1) { const RowState t = st0; st0 = st1; st1 = t; }
                 }
@@ -815,7 +840,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     }
                     const int key = tt * kTile + row0;
                     if (key < L) {
-                        float *dst = scores_out + (size_t)kv * L + key;
+                        float *dst = scores_out + sg.sbase + (size_t)(kv - sg.h0) * L + key;
                         const float sum = (a01.x + a01.y) + (a23.x + a23.y);
                         if (nblk == 1) *dst = sum;
                         else atomicAdd(dst, sum);              // two blocks per key, onto a zero the stage warp wrote
@@ -875,19 +900,32 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-// bf16 tensor [heads][rows][128] viewed as 3-D (128, rows, heads); box = 64 columns x box_rows rows of
-// one head, 128-byte swizzle; rows past `rows` read as zero.
-bool make_map(CUtensorMap *map, const void *ptr, int rows, int heads, int box_rows)
+// bf16 tensor [heads][head_rows][128] of which the first `rows` rows of every head are data, viewed as 3-D
+// (128, rows, heads); box = 64 columns x box_rows rows of one head, 128-byte swizzle; rows past `rows` read
+// as zero.  A tensor map is a pure function of these
+// arguments, so the last few are kept per host thread: a caller that evicts layer after layer (or the same
+// cache again) pays for the driver's encoding once per buffer, not on every call.
+bool make_map(CUtensorMap *map, const void *ptr, int rows, int heads, int box_rows, int head_rows = 0)
 {
+    if (head_rows < rows) head_rows = rows;
+    struct Entry { const void *ptr; int rows, heads, box_rows, head_rows; bool valid; CUtensorMap map; };
+    constexpr int kEntries = 1024;                      // direct-mapped
+    static thread_local Entry cache[kEntries] = {};
+    const uint64_t h = ((uint64_t)(uintptr_t)ptr >> 8) * 0x9E3779B97F4A7C15ull + (uint64_t)rows * 0xC2B2AE3D27D4EB4Full + (uint64_t)head_rows * 0x165667B19E3779F9ull + (uint64_t)(heads * 4 + box_rows / 128);
+    Entry &e = cache[(h >> 40) % kEntries];
+    if (e.valid && e.ptr == ptr && e.rows == rows && e.heads == heads && e.box_rows == box_rows && e.head_rows == head_rows) { *map = e.map; return true; }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)rows, (cuuint64_t)heads};
-    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)rows * kD * 2};
+    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)head_rows * kD * 2};
     cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    e.ptr = ptr; e.rows = rows; e.heads = heads; e.box_rows = box_rows; e.head_rows = head_rows; e.map = *map; e.valid = true;
+    return true;
 }
 
 constexpr size_t smem_bytes(int Rbox, int stages)
@@ -931,56 +969,32 @@ bool device_info(DeviceInfo *out)
 
 }  // namespace
 
-bool build_layer_maps(const void *const *K, const void *const *Qwin, int nlayers, const jq_shape &layer, void *host_maps)
+bool make_tensor_map(void *map, const void *ptr, int rows, int heads, int box_rows)
 {
     static_assert(sizeof(CUtensorMap) == kTensorMapBytes, "tensor map size");
-    CUtensorMap *m = (CUtensorMap *)host_maps;
-    const int R = layer.group * layer.w;
-    for (int l = 0; l < nlayers; ++l)
-        if (!make_map(&m[2 * l], K[l], layer.L, layer.Hkv, kTile) || !make_map(&m[2 * l + 1], Qwin[l], R, layer.Hkv, R <= 128 ? 128 : 256))
-            return false;
-    return true;
+    return make_map((CUtensorMap *)map, ptr, rows, heads, box_rows);
 }
 
-jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float *scores, const Workspace &w,
-                          cudaStream_t st, const void *Kwin, const LayerTables *tables)
+int score_sms()
 {
     DeviceInfo dev;
-    if (!device_info(&dev)) return JQ_ERR_CUDA;
-    const long long group_mib = 32;   // K bytes of a head group: a share of the L2, so that pass 2 finds its keys there
-    const int R = s.group * s.w;
-    Params P;
-    P.L = s.L; P.R = R; P.Rbox = R <= 128 ? 128 : 256; P.Rpad = (R + 31) & ~31;
-    P.Hkv = s.Hkv;
-    P.wtile = Kwin ? 1 : 0;
-    P.tph = (s.L + kTile - 1) / kTile + P.wtile;
-    P.stages = P.Rbox == 128 ? 5 : 3;
-    P.depth = 2;
-    P.c = 1.4426950408889634f / sqrtf((float)s.d);
-    P.part = w.part; P.Mrow = w.Mrow; P.scores = scores; P.status = w.status;
-    P.w = s.w;
-    P.maps = tables ? (const CUtensorMap *)tables->maps : nullptr;
-    P.hpl = tables ? tables->hpl : 0;
-    CUtensorMap mapK, mapQ, mapW;
-    const int map_heads = tables ? tables->hpl : s.Hkv;   // with tables these two describe the first layer and are not used
-    if (!make_map(&mapK, K, s.L, map_heads, kTile) || !make_map(&mapQ, Q, R, map_heads, P.Rbox)) return JQ_ERR_CUDA;
-    if (Kwin) { if (!make_map(&mapW, Kwin, s.w, s.Hkv, kTile)) return JQ_ERR_CUDA; } else mapW = mapK;
+    return device_info(&dev) ? dev.sms : 0;
+}
 
-    const int groups = R > 128 ? kGroupsWide : kGroupsNarrow;
-    int sms = dev.sms;
-    if (groups * sms > kSlots) sms = kSlots / groups;
-    // KV heads are scored in groups whose keys fit in a share of the L2, so that pass 2 finds them there.
-    // Among the admissible group sizes, take the one that wastes the fewest CTA-tile slots.
-    const long long head_bytes = (long long)s.L * kD * 2;
-    long long hmax = (group_mib << 20) / head_bytes;
+// KV heads are scored in groups whose keys fit in a share of the L2 (32 MiB), so that pass 2 finds them there.
+// Among the admissible group sizes, the one that wastes the fewest CTA-tile slots.
+int heads_per_group(int L, int heads, int tiles_per_head, int sms)
+{
+    const long long head_bytes = (long long)L * kD * 2;
+    long long hmax = (32ll << 20) / head_bytes;
     if (hmax < 1) hmax = 1;
-    if (hmax > s.Hkv) hmax = s.Hkv;
+    if (hmax > heads) hmax = heads;
     int best_hpg = 1;
     double best_eff = -1.0;
     for (int hpg = 1; hpg <= (int)hmax; ++hpg) {
         long long work = 0, slots = 0;
-        for (int h0 = 0; h0 < s.Hkv; h0 += hpg) {
-            const long long T = (long long)(h0 + hpg <= s.Hkv ? hpg : s.Hkv - h0) * P.tph;
+        for (int h0 = 0; h0 < heads; h0 += hpg) {
+            const long long T = (long long)(h0 + hpg <= heads ? hpg : heads - h0) * tiles_per_head;
             work += T;
             slots += (T + sms - 1) / sms;
         }
@@ -988,9 +1002,46 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
         if (eff >= best_eff - 1e-9) { best_eff = eff > best_eff ? eff : best_eff; best_hpg = hpg; }
         if (hmax > 64 && hpg >= 64) break;   // the scan is only worth it over a small range
     }
-    P.hpg = best_hpg;
-    P.ngroups = (s.Hkv + P.hpg - 1) / P.hpg;
-    long long tmax = (long long)(P.hpg < s.Hkv ? P.hpg : s.Hkv) * P.tph;
+    return best_hpg;
+}
+
+jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float *scores, const Workspace &w,
+                          cudaStream_t st, const void *Kwin, const UnitTables *tables, int k_head_rows)
+{
+    DeviceInfo dev;
+    if (!device_info(&dev)) return JQ_ERR_CUDA;
+    const int R = s.group * s.w;
+    Params P;
+    P.R = R; P.Rbox = R <= 128 ? 128 : 256; P.Rpad = (R + 31) & ~31;
+    P.Hkv = s.Hkv;
+    P.wtile = Kwin ? 1 : 0;
+    P.stages = P.Rbox == 128 ? 5 : 3;
+    P.depth = 2;
+    P.c = 1.4426950408889634f / sqrtf((float)s.d);
+    P.part = w.part; P.Mrow = w.Mrow; P.scores = scores; P.status = w.status;
+    P.w = s.w;
+    const int groups = R > 128 ? kGroupsWide : kGroupsNarrow;
+    int sms = dev.sms;
+    if (groups * sms > kSlots) sms = kSlots / groups;
+    CUtensorMap mapK, mapQ, mapW;
+    long long tmax;
+    if (tables) {
+        // every unit has tensor maps of its own in device memory; the three parameter maps are not used
+        memset(&mapK, 0, sizeof mapK); mapQ = mapK; mapW = mapK;
+        P.L = 0; P.tph = 0; P.hpg = 0;
+        P.gtab = tables->groups; P.maps = (const CUtensorMap *)tables->maps;
+        P.ngroups = tables->ngroups;
+        tmax = tables->max_group_tiles;
+    } else {
+        P.L = s.L;
+        P.tph = (s.L + kTile - 1) / kTile + P.wtile;
+        P.gtab = nullptr; P.maps = nullptr;
+        if (!make_map(&mapK, K, s.L, s.Hkv, kTile, k_head_rows) || !make_map(&mapQ, Q, R, s.Hkv, P.Rbox)) return JQ_ERR_CUDA;
+        if (Kwin) { if (!make_map(&mapW, Kwin, s.w, s.Hkv, kTile)) return JQ_ERR_CUDA; } else mapW = mapK;
+        P.hpg = heads_per_group(s.L, s.Hkv, P.tph, sms);
+        P.ngroups = (s.Hkv + P.hpg - 1) / P.hpg;
+        tmax = (long long)(P.hpg < s.Hkv ? P.hpg : s.Hkv) * P.tph;
+    }
     const int grid = (int)(tmax < sms ? tmax : sms);
 
     cudaLaunchConfig_t cfg = {};

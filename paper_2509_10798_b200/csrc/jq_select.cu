@@ -98,37 +98,40 @@ __device__ __forceinline__ void find_digit(const uint32_t *g, int krem, SelCtl &
 
 // The cluster copies the kept K and V rows of its head (256 bytes each: 16 lanes x 16 bytes), CTA r the
 // r-th share of them, once every index of the head has been written.
+// kv_in: the head's index within the buffer the rows come from; orow: the head's first row in the outputs.
 template <int CL>
-__device__ __forceinline__ void copy_kept_rows(cg::cluster_group &cluster, const int32_t *out, int kv, int L, int nkeep,
-                                               const uint4 *Kin, const uint4 *Vin, uint4 *Kout, uint4 *Vout,
-                                               const uint4 *const *Ktab, const uint4 *const *Vtab, int hpl)
+__device__ __forceinline__ void copy_kept_rows(cg::cluster_group &cluster, const int32_t *out, int kv_in, long long orow, int L, int nkeep,
+                                               const uint4 *Kin, const uint4 *Vin, uint4 *Kout, uint4 *Vout, int src_rows)
 {
     __threadfence();
     cluster.sync();
-    int kv_in = kv;                       // head index within the buffer the rows come from
-    if (Ktab) { const int lay = kv / hpl; Kin = Ktab[lay]; Vin = Vtab[lay]; kv_in = kv - lay * hpl; }
     const int rank = (int)cluster.block_rank();
     const int r0 = (int)((long long)rank * nkeep / CL), r1 = (int)((long long)(rank + 1) * nkeep / CL);
     const int lane16 = threadIdx.x & 15;
     for (int t = r0 + (int)(threadIdx.x >> 4); t < r1; t += kSelThreads / 16) {
         const int j = min(max(__ldcg(out + t), 0), L - 1);
-        const size_t src = ((size_t)kv_in * L + j) * 16 + lane16, dst = ((size_t)kv * nkeep + t) * 16 + lane16;
+        const size_t src = ((size_t)kv_in * src_rows + j) * 16 + lane16, dst = (size_t)(orow + t) * 16 + lane16;
         Kout[dst] = Kin[src];
         Vout[dst] = Vin[src];
     }
 }
 
-// grid (Hkv * CL), cluster CL, block 1024.
+// grid (Hkv * CL), cluster CL, block 1024.  With htab (ragged calls) every head has a length, a budget, offsets
+// into the scores, the keys and the outputs, and a source buffer of its own; L, nkeep, chunk, keys_in_smem are
+// then those of the longest head and only size the shared memory.
 template <int CL>
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(kSelThreads, 2)
 select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, int32_t *__restrict__ idx,
                float *__restrict__ pooled, uint32_t *__restrict__ gkeys, int chunk, int keys_in_smem, int raw_tile,
                const uint4 *__restrict__ Kin, const uint4 *__restrict__ Vin, uint4 *__restrict__ Kout,
-               uint4 *__restrict__ Vout, const uint4 *const *__restrict__ Ktab, const uint4 *const *__restrict__ Vtab, int hpl)
+               uint4 *__restrict__ Vout, const HeadRec *__restrict__ htab, const uint4 *const *__restrict__ Ktab,
+               const uint4 *const *__restrict__ Vtab, int src_rows)
 {
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
     const int kv = blockIdx.x / CL;
+    int kv_in = kv;                                  // the head's index within the buffer its rows come from
+    long long soff = (long long)kv * L, orow = (long long)kv * nkeep;
     extern __shared__ __align__(16) uint8_t sm[];
     uint32_t *ghist = (uint32_t *)sm;                       // [3][kBins]; the leading CTA's copy accumulates the cluster
     uint32_t *hist = ghist + 3 * kBins;                     // [kBins]
@@ -138,10 +141,17 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
 
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     cudaGridDependencySynchronize();   // everything above ran while the previous kernel of the stream was finishing
+    if (htab) {
+        const HeadRec r = htab[kv];
+        L = r.L; nkeep = r.nkeep; kv_in = r.kv_in; soff = r.soff; orow = r.ooff; src_rows = L;
+        chunk = ((L + CL - 1) / CL + 31) / 32 * 32;   // (keys_in_smem stays the launch's: the longest head decides whether the region exists)
+        if (Ktab) { Kin = Ktab[r.unit]; Vin = Vtab[r.unit]; }
+    }
     const int j0 = min(rank * chunk, L), j1 = min(j0 + chunk, L), n = j1 - j0;
-    const float *s = scores + (size_t)kv * L;
-    uint32_t *mykeys = keys_in_smem ? keys_s : gkeys + (size_t)kv * L + j0;
-    int32_t *out = idx + (size_t)kv * nkeep;
+    const float *s = scores + soff;
+    uint32_t *mykeys = keys_in_smem ? keys_s : gkeys + soff + j0;
+    int32_t *out = idx + orow;
+    if (pooled) pooled += soff;
 
     // ---- 1. max-pool -> keys
     // With the keys in shared memory and a window of at most 9, a thread pools four neighbouring
@@ -192,7 +202,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
                 if (act) {
                     if (nval == 4) *(uint4 *)(mykeys + t0 + 4 * g4) = make_uint4(key[0], key[1], key[2], key[3]);
                     else for (int i = 0; i < nval; ++i) mykeys[t0 + 4 * g4 + i] = key[i];
-                    if (pooled) for (int i = 0; i < nval; ++i) pooled[(size_t)kv * L + j0 + t0 + 4 * g4 + i] = best[i];
+                    if (pooled) for (int i = 0; i < nval; ++i) pooled[j0 + t0 + 4 * g4 + i] = best[i];
                 }
                 // first-round histogram: one addition per warp when all its positions share the digit (the usual
                 // case: 128 neighbouring positions of similar size), else runs of equal digits per thread
@@ -220,12 +230,12 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
             float best = raw[e];
             for (int u = 1; u <= 2 * radius; ++u) best = fmaxf(best, raw[e + u]);
             mykeys[t0 + e] = order_key(best);
-            if (pooled) pooled[(size_t)kv * L + j0 + t0 + e] = best;
+            if (pooled) pooled[j0 + t0 + e] = best;
         }
     }
     if (nkeep >= L) {   // everything is kept (uniform over the cluster; no cluster traffic yet)
         for (int e = tid; e < n; e += kSelThreads) out[j0 + e] = j0 + e;
-        if (Kin || Ktab) copy_kept_rows<CL>(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout, Ktab, Vtab, hpl);
+        if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, orow, L, nkeep, Kin, Vin, Kout, Vout, src_rows);
         return;
     }
     for (int i = tid; i < 3 * kBins; i += kSelThreads) ghist[i] = 0;
@@ -379,7 +389,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         gt_before += __popc(bg);
         eq_before += __popc(be);
     }
-    if (Kin || Ktab) copy_kept_rows<CL>(cluster, out, kv, L, nkeep, Kin, Vin, Kout, Vout, Ktab, Vtab, hpl);
+    if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, orow, L, nkeep, Kin, Vin, Kout, Vout, src_rows);
 }
 
 // Shared memory of a CTA whose cluster has `cl` CTAs, the share of the head it holds, and whether its keys stay on chip.
@@ -422,7 +432,7 @@ SelPlan choose_plan(int Hkv, int L, int sms)
 template <int CL>
 jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape &s, int nkeep, int32_t *idx, float *pooled,
                            const Workspace &w, cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout, int dev,
-                           const LayerTables *tables)
+                           const UnitTables *tables, int src_rows)
 {
     static bool attr_done[64] = {};
     if (!attr_done[dev]) {
@@ -445,8 +455,8 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
     cfg.numAttrs = 1;
     if (cudaLaunchKernelEx(&cfg, select_cluster<CL>, scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, w.keys, p.chunk,
                            p.in_smem, p.raw_tile, (const uint4 *)K, (const uint4 *)V, (uint4 *)Kout, (uint4 *)Vout,
-                           (const uint4 *const *)(tables ? tables->K : nullptr), (const uint4 *const *)(tables ? tables->V : nullptr),
-                           tables ? tables->hpl : 0) != cudaSuccess) {
+                           tables ? tables->heads : nullptr, (const uint4 *const *)(tables && Kout ? tables->K : nullptr),
+                           (const uint4 *const *)(tables && Kout ? tables->V : nullptr), src_rows) != cudaSuccess) {
         cudaGetLastError();
         return JQ_ERR_CUDA;
     }
@@ -458,18 +468,21 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
 
 jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, float *pooled,
                         const Workspace &w, cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout,
-                        const LayerTables *tables)
+                        const UnitTables *tables, int src_head_rows)
 {
-    const int nkeep = s.budget < s.L ? s.budget : s.L;
+    const int src_rows = src_head_rows > s.L ? src_head_rows : s.L;
+    // with tables: the plan and the shared memory follow the longest head; every head reads its own record
+    const int Lmax = tables ? tables->max_L : s.L;
+    const int nkeep = s.budget < Lmax ? s.budget : Lmax;
     static int sms[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return JQ_ERR_CUDA;
     if (!sms[dev] && cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return JQ_ERR_CUDA;
-    const SelPlan p = choose_plan(s.Hkv, s.L, sms[dev]);
+    const SelPlan p = choose_plan(s.Hkv, Lmax, sms[dev]);
     switch (p.cl) {
-    case 2: return launch_select_cl<2>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables);
-    case 4: return launch_select_cl<4>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables);
-    default: return launch_select_cl<8>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables);
+    case 2: return launch_select_cl<2>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables, src_rows);
+    case 4: return launch_select_cl<4>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables, src_rows);
+    default: return launch_select_cl<8>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables, src_rows);
     }
 }
 

@@ -84,12 +84,25 @@ def test_pointer_errors_are_caught_on_the_host():
     ptrs = (ctypes.c_void_p * 2)(0x1000, 0x2000)
     assert lib.jq_evict_layers(ptrs, ptrs, ptrs, 2, ref, a, a, a, a, 16, None) == jq.JQ_ERR_WORKSPACE
     assert lib.jq_evict_layers(ptrs, ptrs, ptrs, 0, ref, a, a, a, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
-    assert lib.jq_evict_layers(ptrs, ptrs, ptrs, 129, ref, a, a, a, a, 1 << 40, None) == jq.JQ_ERR_UNSUPPORTED
+    assert lib.jq_evict_layers(ptrs, ptrs, ptrs, 4097, ref, a, a, a, a, 1 << 40, None) == jq.JQ_ERR_UNSUPPORTED
+    two = (ctypes.c_int * 2)
+    assert lib.jq_evict_ragged(ptrs, ptrs, ptrs, 2, ref, two(100, 200), two(10, 10), a, a, a, a, 16, None) == jq.JQ_ERR_WORKSPACE
+    assert lib.jq_evict_ragged(ptrs, ptrs, ptrs, 2, ref, two(100, 0), two(10, 10), a, a, a, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
+    assert lib.jq_evict_ragged(ptrs, ptrs, ptrs, 2, ref, two(100, 200), two(10, 0), a, a, a, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
+    assert lib.jq_evict_ragged(ptrs, ptrs, ptrs, 2, ref, None, None, a, a, odd, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
+    assert jq.ragged_workspace_bytes(s, 2, [100, 200]) < jq.ragged_workspace_bytes(s, 2, [100, 300])
+    assert jq.ragged_output_rows(s, 3, [100, 200, 5], [10, 300, 7]) == 2 * (10 + 200 + 5)
     assert lib.jq_evict_layers(None, ptrs, ptrs, 2, ref, a, a, a, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
     odd_ptrs = (ctypes.c_void_p * 2)(0x1000, 0x2008)
     assert lib.jq_evict_layers(odd_ptrs, ptrs, ptrs, 2, ref, a, a, a, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
     assert jq.layers_workspace_bytes(s, 2) > jq.workspace_bytes(jq.shape(4, 16, 2048, 16, 256)) and jq.layers_workspace_bytes(s, 0) == 0
     assert lib.jq_hit_rate(a, a, 0, 4, 4, a, None) == jq.JQ_ERR_INVALID_ARG
+    # jq_evict_append: s.L = 2048 must equal n_old + n_new and fit the cache's rows per head
+    assert lib.jq_evict_append(a, a, 4096, 2000, a, a, 47, a, ref, a, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
+    assert lib.jq_evict_append(a, a, 2047, 2000, a, a, 48, a, ref, a, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
+    assert lib.jq_evict_append(a, a, 4096, 2000, None, a, 48, a, ref, a, a, 1 << 40, None) == jq.JQ_ERR_INVALID_ARG
+    assert lib.jq_evict_append(a, a, 4096, 2000, a, a, 48, a, ref, a, a, n, None) == jq.JQ_ERR_WORKSPACE
+    assert lib.jq_append_workspace_bytes(ref) > n
     assert lib.jq_last_device_status(None, None) == jq.JQ_ERR_INVALID_ARG
     assert jq.status_string(jq.JQ_ERR_TIMEOUT) and jq.status_string(99)
     assert jq.launch_count() == 0      # nothing above reached a launch

@@ -537,8 +537,9 @@ def test_evict_layers_workspace_reused_with_other_buffers_and_shapes():
     tensor maps the call leaves in the workspace are rewritten every time, and the kernel must read the new
     ones (the first call's buffers are freed before the second runs)."""
     wa, wb = small_wl(2, 4, 32, 3000, 400), small_wl(4, 4, 64, 1500, 200)
-    ws = jq.new_layers_workspace(shape_of(wa), 6)
-    assert ws.numel() >= jq.layers_workspace_bytes(shape_of(wb), 3)
+    need = max(jq.layers_workspace_bytes(shape_of(wa), 6), jq.layers_workspace_bytes(shape_of(wb), 3))
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    jq._raise("jq_workspace_init", jq.lib().jq_workspace_init(jq._ptr(ws), ws.numel(), jq._stream(None)))
     for wl, nl, first in ((wa, 6, 0), (wb, 3, 10), (wa, 4, 20), (wb, 2, 30)):
         layers = [W.make_layer(wl, layer=first + i) for i in range(nl)]
         gK, gV, gi = _layers_call(layers, wl, ws)
@@ -563,3 +564,146 @@ def test_evict_layers_cfg5_shape_against_the_oracle():
         assert_kept_sets_agree(gi[u:u + 1], oracle.select(po, wl.budget), po, wl.nkeep)
         assert np.array_equal(gK[u], K[kv][gi[u]]) and np.array_equal(gV[u], V[kv][gi[u]])
     assert np.all(np.diff(gi, axis=1) > 0) and gi.min() >= 0 and gi.max() < wl.L
+
+
+# ------------------------------------------------------------------ ragged units: lengths and budgets of their own, one call
+
+def _ragged_call(units, s_common, Ls, Bs, ws=None):
+    """jq_evict_ragged on host units (K, V, Q); returns per-unit (Kout bits, Vout bits, idx) slices of the stacked outputs."""
+    n = len(units)
+    dK, dV, dQ = [dev_bf16(u[0]) for u in units], [dev_bf16(u[1]) for u in units], [dev_bf16(u[2]) for u in units]
+    rows = jq.ragged_output_rows(s_common, n, Ls, Bs)
+    Hkv = s_common.Hkv
+    keeps = [min(b, l) for b, l in zip(Bs, Ls)]
+    assert rows == Hkv * sum(keeps)
+    Ko = torch.zeros((rows, 128), dtype=torch.bfloat16, device="cuda")
+    Vo = torch.zeros_like(Ko)
+    idx = torch.full((rows,), -1, dtype=torch.int32, device="cuda")
+    if ws is None:
+        ws = jq.new_ragged_workspace(s_common, n, Ls)
+    jq.evict_ragged(dK, dV, dQ, s_common, Ls, Bs, Ko, Vo, idx, ws)
+    assert jq.last_device_status(ws) == jq.JQ_OK
+    gK, gV, gi = host_bits(Ko), host_bits(Vo), idx.cpu().numpy()
+    out, r0 = [], 0
+    for k in keeps:
+        r1 = r0 + Hkv * k
+        out.append((gK[r0:r1].reshape(Hkv, k, 128), gV[r0:r1].reshape(Hkv, k, 128), gi[r0:r1].reshape(Hkv, k)))
+        r0 = r1
+    return out
+
+
+@pytest.mark.parametrize("Hkv,g,w,Ls,Bs", [
+    (2, 4, 32, [3000, 130, 5000, 1, 2049], [400, 1000, 64, 3, 2049]),        # tails, L = 1, budget >= L, budget == L
+    (2, 4, 64, [2049, 700, 4096], [300, 300, 10]),                           # 256 query rows per KV head
+    (8, 4, 32, [4096, 12000, 20480, 8192], [1024, 900, 800, 700]),           # the ragged batch's lengths (shortened), decreasing budgets
+    (1, 1, 1, [5, 7], [3, 2]),
+])
+def test_evict_ragged_matches_calls_per_unit(Hkv, g, w, Ls, Bs):
+    """Units of different lengths and budgets in one call: bit for bit what one jq_evict_layer call per unit gives,
+    and one unit against the oracle under the end-to-end rule."""
+    base = small_wl(Hkv, g, w, max(Ls), max(Bs))
+    units = [W.make_layer(base.with_L(l).with_budget(b), layer=i) for i, (l, b) in enumerate(zip(Ls, Bs))]
+    got = _ragged_call(units, shape_of(base), Ls, Bs)
+    for (K, V, Q, _), (gK, gV, gi), l, b in zip(units, got, Ls, Bs):
+        wK, wV, wi = gpu_evict(K, V, Q, shape_of(base.with_L(l).with_budget(b)))
+        assert np.array_equal(gi, wi) and np.array_equal(gK, wK) and np.array_equal(gV, wV)
+    K, V, Q, _ = units[0]
+    pooled = oracle.pool(oracle.score(K, Q), base.pool)
+    assert_kept_sets_agree(got[0][2], oracle.select(pooled, Bs[0]), pooled, min(Bs[0], Ls[0]))
+
+
+def test_evict_ragged_per_layer_budget_schedule_against_the_oracle():
+    """A layer-wise decreasing budget (the pyramid-shaped schedule of the experimental-setting paragraph) over the
+    layers of one cache, one call; every layer against the oracle."""
+    wl = small_wl(4, 4, 32, 6000, 1024)
+    nl = 6
+    Bs = [1024, 768, 512, 384, 256, 128]
+    units = [W.make_layer(wl, layer=i) for i in range(nl)]
+    got = _ragged_call(units, shape_of(wl), [wl.L] * nl, Bs)
+    for (K, V, Q, _), (gK, gV, gi), b in zip(units, got, Bs):
+        pooled = oracle.pool(oracle.score(K, Q), wl.pool)
+        assert_kept_sets_agree(gi, oracle.select(pooled, b), pooled, b)
+        for kv in range(wl.Hkv):
+            assert np.array_equal(gK[kv], K[kv][gi[kv]]) and np.array_equal(gV[kv], V[kv][gi[kv]])
+
+
+def test_evict_ragged_whole_batch_of_config_4_in_one_call():
+    """The ragged batch at full size: four sequences (4096, 12000, 20480, 32768 keys) x 4 layers each, 16 units, one
+    call; one sampled layer per sequence against the oracle, every unit against its own jq_evict_layer call."""
+    nl = 4
+    units, Ls, Bs, meta = [], [], [], []
+    for seq, wl in enumerate(W.CFG4):
+        for layer in range(nl):
+            units.append(W.make_layer(wl, layer=layer, seq=seq)); Ls.append(wl.L); Bs.append(wl.budget); meta.append((seq, layer, wl))
+    got = _ragged_call(units, shape_of(W.CFG4[3]), Ls, Bs)
+    for (K, V, Q, _), (gK, gV, gi), (seq, layer, wl) in zip(units, got, meta):
+        wK, wV, wi = gpu_evict(K, V, Q, shape_of(wl))
+        assert np.array_equal(gi, wi) and np.array_equal(gK, wK) and np.array_equal(gV, wV)
+        if layer == seq:                                       # one layer per sequence
+            pooled = oracle.pool(oracle.score(K, Q), wl.pool)
+            assert_kept_sets_agree(gi, oracle.select(pooled, wl.budget), pooled, wl.nkeep)
+
+
+def test_evict_ragged_rejects_bad_arguments():
+    wl = small_wl(2, 4, 16, 500, 10)
+    s = shape_of(wl)
+    assert jq.ragged_workspace_bytes(s, 2, [500, 0]) == 0           # a unit without keys
+    assert jq.ragged_workspace_bytes(s, 0) == 0
+    assert jq.ragged_output_rows(s, 2, [500, 300], [10, -1]) == 0
+    assert jq.ragged_output_rows(s, 2, [500, 300], [10, 1000]) == 2 * (10 + 300)
+
+
+# ------------------------------------------------------------------ streaming re-eviction
+
+@pytest.mark.parametrize("Hkv,g,w,n_old,n_new,budget,cap", [(2, 4, 16, 512, 100, 512, 640), (2, 4, 64, 300, 1, 200, 301),
+                                                             (3, 2, 32, 1000, 0, 400, 1500), (1, 1, 8, 10, 30, 64, 40)])
+def test_evict_append_matches_the_pass_on_the_concatenation(Hkv, g, w, n_old, n_new, budget, cap):
+    """The cache of a layer holds n_old retained rows per head in a buffer of `cap` rows; n_new rows are appended and the
+    cache is evicted again, in place.  Expected: the oracle's pass over the concatenated rows (end-to-end rule), and the
+    rows the indices name, bit for bit, at the head of the cache."""
+    wl = small_wl(Hkv, g, w, n_old + n_new, budget)
+    K, V, Q, _ = W.make_layer(wl, layer=3)
+    s = shape_of(wl)
+    Kc = torch.zeros((Hkv, cap, 128), dtype=torch.bfloat16, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    Kc[:, :n_old] = dev_bf16(K[:, :n_old]); Vc[:, :n_old] = dev_bf16(V[:, :n_old])
+    Kn = dev_bf16(K[:, n_old:]) if n_new else None
+    Vn = dev_bf16(V[:, n_old:]) if n_new else None
+    idx = torch.full((Hkv, wl.nkeep), -1, dtype=torch.int32, device="cuda")
+    ws = jq.new_append_workspace(s)
+    jq.evict_append(Kc, Vc, n_old, Kn, Vn, dev_bf16(Q), s, idx, ws)
+    assert jq.last_device_status(ws) == jq.JQ_OK
+    gi = idx.cpu().numpy()
+    pooled = oracle.pool(oracle.score(K, Q), wl.pool)
+    assert_kept_sets_agree(gi, oracle.select(pooled, budget), pooled, wl.nkeep)
+    gK, gV = host_bits(Kc), host_bits(Vc)
+    for kv in range(Hkv):
+        assert np.array_equal(gK[kv, :wl.nkeep], K[kv][gi[kv]]) and np.array_equal(gV[kv, :wl.nkeep], V[kv][gi[kv]])
+    # and bit for bit what jq_evict_layer gives on the packed concatenation
+    wK, wV, wi = gpu_evict(K, V, Q, s)
+    assert np.array_equal(gi, wi) and np.array_equal(gK[:, :wl.nkeep], wK) and np.array_equal(gV[:, :wl.nkeep], wV)
+
+
+def test_evict_append_twice_in_a_row_then_decode():
+    """Evict after the prefill, then two rounds of: decode over the pruned cache, append rows, evict again."""
+    wl = small_wl(2, 4, 16, 2000, 256)
+    K, V, Q, _ = W.make_layer(wl)
+    cap = 256 + 64
+    Ko, Vo, gidx = gpu_evict(K, V, Q, shape_of(wl))
+    Kc = torch.zeros((wl.Hkv, cap, 128), dtype=torch.bfloat16, device="cuda"); Vc = torch.zeros_like(Kc)
+    Kc[:, :256] = dev_bf16(Ko); Vc[:, :256] = dev_bf16(Vo)
+    hostK, hostV = Ko.copy(), Vo.copy()
+    for rnd in range(2):
+        extra = small_wl(2, 4, 16, 64, 256)
+        Kn, Vn, Qn, _ = W.make_layer(extra, layer=50 + rnd)
+        allK, allV = np.concatenate([hostK, Kn], 1), np.concatenate([hostV, Vn], 1)
+        s2 = shape_of(small_wl(2, 4, 16, 320, 256))
+        idx = torch.full((wl.Hkv, 256), -1, dtype=torch.int32, device="cuda")
+        ws = jq.new_append_workspace(s2)
+        jq.evict_append(Kc, Vc, 256, dev_bf16(Kn), dev_bf16(Vn), dev_bf16(Qn), s2, idx, ws)
+        assert jq.last_device_status(ws) == jq.JQ_OK
+        gi = idx.cpu().numpy()
+        pooled = oracle.pool(oracle.score(allK, Qn), wl.pool)
+        assert_kept_sets_agree(gi, oracle.select(pooled, 256), pooled, 256)
+        hostK = np.stack([allK[kv][gi[kv]] for kv in range(wl.Hkv)]); hostV = np.stack([allV[kv][gi[kv]] for kv in range(wl.Hkv)])
+        assert np.array_equal(host_bits(Kc)[:, :256], hostK) and np.array_equal(host_bits(Vc)[:, :256], hostV)
