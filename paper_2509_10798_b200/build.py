@@ -1,4 +1,7 @@
-"""Compile the CUDA sources under csrc/ into paper_2509_10798_b200/libjq.so for sm_100a (in-tree)."""
+"""Compile the CUDA sources under csrc/ into paper_2509_10798_b200/libjq.so for sm_100a (in-tree).
+
+build(debug=True) compiles the same sources with -DJQ_DEBUG into libjq_debug.so: the bounds-checked build
+(csrc/jq_debug.cuh), in which every index the kernels compute is compared with the extent of what it indexes."""
 import glob
 import os
 import subprocess
@@ -8,6 +11,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libjq.so")
+LIB_DEBUG = os.path.join(HERE, "libjq_debug.so")
 OBJDIR = os.path.join(HERE, "_build")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -25,17 +29,20 @@ def _deps():
     return glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
     srcs = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
-    os.makedirs(OBJDIR, exist_ok=True)
+    objdir = OBJDIR + ("_debug" if debug else "")
+    lib = LIB_DEBUG if debug else LIB
+    flags = NVCC_FLAGS + (["-DJQ_DEBUG"] if debug else [])
+    os.makedirs(objdir, exist_ok=True)
     dep_mtime = max(os.path.getmtime(p) for p in _deps())
     objs, rebuilt = [], False
     procs = []
     for src in srcs:
-        obj = os.path.join(OBJDIR, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), dep_mtime):
-            cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
+            cmd = [_nvcc()] + flags + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
             procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
             rebuilt = True
     for src, p in procs:
@@ -44,13 +51,13 @@ def build(force: bool = False, verbose: bool = False) -> str:
             sys.stderr.write(out)
         if p.returncode:
             raise RuntimeError("nvcc failed on %s" % src)
-    if rebuilt or not os.path.exists(LIB):
-        tmp = LIB + ".tmp%d" % os.getpid()
+    if rebuilt or not os.path.exists(lib):
+        tmp = lib + ".tmp%d" % os.getpid()
         cmd = [_nvcc(), "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"]
         subprocess.run(cmd, check=True)
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -243,19 +243,11 @@ jq_status jq_evict_ragged(const void *const *K, const void *const *V, const void
     int ngroups = 0;
     for (int u = 0; u < nunits; ++u) {
         const int Lu = L ? L[u] : common->L, Bu = budget ? budget[u] : common->budget;
-        const int nkeep = Bu < Lu ? Bu : Lu, tph = (Lu + 127) / 128;
+        const int nkeep = Bu < Lu ? Bu : Lu;
         if (!make_tensor_map(h_maps + (size_t)(2 * u) * kTensorMapBytes, K[u], Lu, hpu, 128) ||
             !make_tensor_map(h_maps + (size_t)(2 * u + 1) * kTensorMapBytes, Qwin[u], R, hpu, R <= 128 ? 128 : 256))
             return JQ_ERR_CUDA;
         h_K[u] = K[u]; h_V[u] = V[u];
-        const int hpg = heads_per_group(Lu, hpu, tph, sms);
-        for (int h0 = 0; h0 < hpu; h0 += hpg) {
-            GroupRec &g = h_grp[ngroups++];
-            g.h0 = u * hpu + h0; g.nh = h0 + hpg <= hpu ? hpg : hpu - h0;
-            g.tph = tph; g.L = Lu; g.unit = u; g.c20 = h0;
-            g.sbase = soff + (long long)h0 * Lu;
-            if (g.nh * tph > t.max_group_tiles) t.max_group_tiles = g.nh * tph;
-        }
         for (int h = 0; h < hpu; ++h) {
             HeadRec &r = h_head[u * hpu + h];
             r.L = Lu; r.nkeep = nkeep; r.unit = u; r.kv_in = h;
@@ -265,6 +257,22 @@ jq_status jq_evict_ragged(const void *const *K, const void *const *V, const void
         soff += (long long)hpu * Lu;
         ooff += (long long)hpu * nkeep;
     }
+    // head groups of the scoring kernel: every run of consecutive units of one length is cut into groups of
+    // about 32 MiB of keys (short prefixes share a group across units, so that a group still has tiles for every CTA)
+    for (int u0 = 0; u0 < nunits;) {
+        const int Lu = L ? L[u0] : common->L, tph = (Lu + 127) / 128;
+        int u1 = u0 + 1;
+        while (u1 < nunits && (L ? L[u1] : common->L) == Lu) ++u1;
+        const int heads = (u1 - u0) * hpu, hpg = heads_per_group(Lu, heads, tph, sms);
+        for (int h0 = 0; h0 < heads; h0 += hpg) {
+            GroupRec &g = h_grp[ngroups++];
+            g.h0 = u0 * hpu + h0; g.nh = h0 + hpg <= heads ? hpg : heads - h0;
+            g.tph = tph; g.L = Lu; g.unit = u0 + h0 / hpu; g.c20 = h0 % hpu;
+            g.sbase = h_head[g.h0].soff;
+            if (g.nh * tph > t.max_group_tiles) t.max_group_tiles = g.nh * tph;
+        }
+        u0 = u1;
+    }
     char *tab = (char *)ws + w.bytes;
     if (cudaMemcpyAsync(tab, hb, tab_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return JQ_ERR_CUDA;
     t.maps = tab;
@@ -272,7 +280,7 @@ jq_status jq_evict_ragged(const void *const *K, const void *const *V, const void
     t.V = (const void *const *)(tab + maps_bytes + ptr_bytes);
     t.groups = (const GroupRec *)(tab + maps_bytes + 2 * ptr_bytes);
     t.heads = (const HeadRec *)(tab + maps_bytes + 2 * ptr_bytes + grp_bytes);
-    t.ngroups = ngroups; t.hpu = hpu; t.max_L = pl.max_L;
+    t.ngroups = ngroups; t.hpu = hpu; t.max_L = pl.max_L; t.total_keys = (long long)pl.keys; t.total_rows = pl.rows;
     if ((rc = launch_score_tc(nullptr, nullptr, pl.S, w.scores, w, st, nullptr, &t)) != JQ_OK) return rc;
     return launch_select(w.scores, pl.S, kept_idx, nullptr, w, st, nullptr, nullptr, Kout, Vout, &t);
 }

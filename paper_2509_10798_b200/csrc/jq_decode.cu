@@ -12,6 +12,7 @@
 #include <cuda_bf16.h>
 
 #include "jq_internal.cuh"
+#include "jq_debug.cuh"
 
 namespace jq {
 namespace {
@@ -27,7 +28,7 @@ __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u 
 
 __global__ void __launch_bounds__(kDecThreads)
 decode_step(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, const __nv_bfloat16 *__restrict__ q, int n,
-            int group, float scale_log2, float *__restrict__ part, unsigned int *__restrict__ tickets, float *__restrict__ out)
+            int group, float scale_log2, float *__restrict__ part, unsigned int *__restrict__ tickets, float *__restrict__ out JQ_DBG_PARAM)
 {
     __shared__ int is_last;
     __shared__ __align__(16) __nv_bfloat16 Ks[kDecChunk * kKRow];
@@ -37,16 +38,19 @@ decode_step(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, const __
     const int tid = threadIdx.x, split = blockIdx.x, kv = blockIdx.y, nsplit = gridDim.x;
     const int j0 = split * kDecChunk, valid = min(kDecChunk, n - j0);
 
-    for (int i = tid; i < group * kD; i += kDecThreads) qs[i] = __bfloat162float(q[(size_t)kv * group * kD + i]);
+    const long long n_rows = (long long)gridDim.y * n, n_part = (long long)gridDim.y * nsplit * group * kPartial;   // extents, for the bounds-checked build
+    (void)n_rows; (void)n_part;
+    for (int i = tid; i < group * kD; i += kDecThreads)
+        if (JQ_IN(i, kDecMaxGroup * kD, kDbgDecode, 1)) qs[i] = __bfloat162float(q[(size_t)kv * group * kD + i]);
     for (int i = tid; i < kDecChunk * 16; i += kDecThreads) {       // 16 x 16 bytes per row
         const int r = i >> 4, c = i & 15;
         uint4 k4 = make_uint4(0u, 0u, 0u, 0u), v4 = k4;
-        if (r < valid) {
+        if (r < valid && JQ_IN((long long)kv * n + j0 + r, n_rows, kDbgDecode, 2)) {
             k4 = Kc[((size_t)kv * n + j0 + r) * 16 + c];
             v4 = Vc[((size_t)kv * n + j0 + r) * 16 + c];
         }
-        *(uint4 *)(Ks + r * kKRow + c * 8) = k4;
-        *(uint4 *)(Vs + r * kD + c * 8) = v4;
+        if (JQ_IN(r * kKRow + c * 8 + 7, kDecChunk * kKRow, kDbgDecode, 3)) *(uint4 *)(Ks + r * kKRow + c * 8) = k4;
+        if (JQ_IN(r * kD + c * 8 + 7, kDecChunk * kD, kDbgDecode, 4)) *(uint4 *)(Vs + r * kD + c * 8) = v4;
     }
     __syncthreads();
 
@@ -64,7 +68,7 @@ decode_step(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, const __
                 acc = fmaf(bf16_lo(k4.z), qh[c * 8 + 4], acc); acc = fmaf(bf16_hi(k4.z), qh[c * 8 + 5], acc);
                 acc = fmaf(bf16_lo(k4.w), qh[c * 8 + 6], acc); acc = fmaf(bf16_hi(k4.w), qh[c * 8 + 7], acc);
             }
-            ps[h * kDecChunk + j] = (j < valid) ? acc * scale_log2 : -INFINITY;
+            if (JQ_IN(h * kDecChunk + j, kDecMaxGroup * kDecChunk, kDbgDecode, 5)) ps[h * kDecChunk + j] = (j < valid) ? acc * scale_log2 : -INFINITY;
         }
     }
     __syncthreads();
@@ -85,7 +89,7 @@ decode_step(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, const __
             ps[h * kDecChunk + lane + 32] = pb;
             if (lane == 0) {
                 float *dst = part + ((size_t)(kv * nsplit + split) * group + h) * kPartial;
-                dst[0] = m; dst[1] = l;
+                if (JQ_IN(((long long)(kv * nsplit + split) * group + h) * kPartial + 1, n_part, kDbgDecode, 6)) { dst[0] = m; dst[1] = l; }
             }
         }
     }
@@ -104,7 +108,8 @@ decode_step(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, const __
                 o1 = fmaf(ph[j], bf16_hi(v2), o1);
             }
             float *dst = part + ((size_t)(kv * nsplit + split) * group + h) * kPartial + 2;
-            *(float2 *)(dst + 2 * cp) = make_float2(o0, o1);
+            if (JQ_IN(((long long)(kv * nsplit + split) * group + h) * kPartial + 2 + 2 * cp + 1, n_part, kDbgDecode, 7))
+                *(float2 *)(dst + 2 * cp) = make_float2(o0, o1);
         }
     }
 
@@ -131,7 +136,9 @@ decode_step(const uint4 *__restrict__ Kc, const uint4 *__restrict__ Vc, const __
             Lsum = fmaf(__ldcg(src + 1), f, Lsum);
             O = fmaf(__ldcg(src + 2 + c), f, O);
         }
-        out[((size_t)kv * group + h) * kD + c] = O / Lsum;
+        if (JQ_IN(((long long)kv * group + h) * kD + c, (long long)gridDim.y * group * kD, kDbgDecode, 8) &&
+            JQ_IN(((long long)kv * nsplit * group + h) * kPartial + (long long)(nsplit - 1) * step + 2 + c, n_part, kDbgDecode, 9))
+            out[((size_t)kv * group + h) * kD + c] = O / Lsum;
     }
 }
 
@@ -161,7 +168,7 @@ extern "C" jq_status jq_decode_attention(const void *Kc, const void *Vc, const v
     unsigned int *tickets = (unsigned int *)((char *)workspace + jq::align_up((size_t)Hq * nsplit * jq::kPartial * sizeof(float), 256));
     if (cudaMemsetAsync(tickets, 0, (size_t)Hkv * sizeof(unsigned int), st) != cudaSuccess) return JQ_ERR_CUDA;
     jq::decode_step<<<dim3((unsigned)nsplit, (unsigned)Hkv), jq::kDecThreads, 0, st>>>(
-        (const uint4 *)Kc, (const uint4 *)Vc, (const __nv_bfloat16 *)q, n, group, scale_log2, (float *)workspace, tickets, out);
+        (const uint4 *)Kc, (const uint4 *)Vc, (const __nv_bfloat16 *)q, n, group, scale_log2, (float *)workspace, tickets, out JQ_DBG_ARG);
     jq::count_launch(1);
     return jq::check_launch();
 }

@@ -59,11 +59,12 @@ static inline Workspace carve(void *base, const jq_shape &s)
 // KV heads are numbered through all units; unit u owns heads [u * hpu, (u + 1) * hpu).
 constexpr int kMaxUnits = 4096;
 constexpr size_t kTensorMapBytes = 128;
-// A head group of the scoring kernel: consecutive KV heads of ONE unit whose keys fit a share of the L2.
+// A head group of the scoring kernel: consecutive KV heads of one prefix length whose keys fit a share of the
+// L2.  A group may run over consecutive units of equal length (their scores are consecutive too).
 struct GroupRec {
     int h0, nh;          // first KV head (global numbering) and number of heads
     int tph, L;          // tiles per head, prefix length
-    int unit, c20;       // the unit, and the index of head h0 within it
+    int unit, c20;       // the unit of head h0, and the index of head h0 within it
     long long sbase;     // offset (floats) of head h0's scores in the scores array
 };
 // A KV head as the selection kernel sees it.
@@ -82,6 +83,8 @@ struct UnitTables {
     int ngroups = 0, hpu = 0;            // hpu: KV heads per unit
     int max_group_tiles = 0;             // most tiles in any group (sizes the grid)
     int max_L = 0;                       // longest prefix (sizes the selection kernel's shared memory)
+    long long total_keys = 0;            // keys of all units (floats in the scores array)
+    long long total_rows = 0;            // rows of the stacked outputs
 };
 static inline size_t unit_tables_bytes(int nunits, int hpu)
 {

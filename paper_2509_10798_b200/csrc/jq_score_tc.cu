@@ -44,6 +44,7 @@
 // frees the tensor memory).
 #include "jq_internal.cuh"
 #include "jq_tmem_ld.cuh"
+#include "jq_debug.cuh"
 #include <cuda.h>
 #include <cstddef>
 #include <cstring>
@@ -111,6 +112,11 @@ struct Params {
     // gtab [ngroups] (L, tph, hpg above are then unused) and the tiles through maps [units][2] (K, Qwin).
     const GroupRec *gtab;
     const CUtensorMap *maps;
+    int hpu;                 // KV heads per unit (a group may run over consecutive units of one length)
+#ifdef JQ_DEBUG
+    DebugRecord *dbg_rec;    // bounds-checked build: the violation record, and the floats in the scores array
+    long long n_scores;
+#endif
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -416,7 +422,10 @@ struct Seg {
 // Head group g: from the table of a ragged call, else g-th run of hpg heads of the one stacked tensor.
 __device__ __forceinline__ GroupRec group_of(int g, const Params &P)
 {
-    if (P.gtab) return P.gtab[g];
+#ifdef JQ_DEBUG
+    DebugRecord *dbg = P.dbg_rec;
+#endif
+    if (P.gtab) return P.gtab[JQ_IN(g, P.ngroups, kDbgScore, 1) ? g : 0];
     GroupRec r;
     r.h0 = g * P.hpg; r.nh = min(P.hpg, P.Hkv - r.h0);
     r.tph = P.tph; r.L = P.L; r.unit = 0; r.c20 = r.h0;
@@ -476,6 +485,10 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
     int *const status = P.status;
     const int nblk = P.Rbox / 128;                            // accumulator blocks per tile, both passes
     const int nseg = 2 * P.ngroups;
+#ifdef JQ_DEBUG
+    DebugRecord *const dbg = P.dbg_rec;
+    const long long n_part = (long long)P.Hkv * kSlots * R, n_scores = P.n_scores;
+#endif
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
@@ -511,15 +524,19 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     const Seg sg = segment(s, P);
                     const int pass = sg.pass, ntiles = sg.ntiles, tph = sg.tph;
                     int kv = sg.kv0, tt = sg.t0;
-                    if (P.maps && sg.unit != prev_unit && ntiles > 0) {   // the group's unit has tensor maps of its own
-                        head_mapK = P.maps + 2 * sg.unit; head_mapQ = head_mapK + 1;
-                        tensormap_acquire(head_mapK); tensormap_acquire(head_mapQ);
-                        prev_unit = sg.unit;
-                    }
 #pragma unroll 1
                     for (int n = 0; n < ntiles; ++n, walk(pass, tph, kv, tt)) {
                         if (kv != prev_kv) {
                             head_c2 = sg.c20 + (kv - sg.h0);
+                            if (P.maps) {                         // every unit has tensor maps of its own; the group may run over several units
+                                const int du = head_c2 / P.hpu, unit = sg.unit + du;
+                                head_c2 -= du * P.hpu;
+                                if (unit != prev_unit) {
+                                    head_mapK = P.maps + 2 * unit; head_mapQ = head_mapK + 1;
+                                    tensormap_acquire(head_mapK); tensormap_acquire(head_mapQ);
+                                    prev_unit = unit;
+                                }
+                            }
                             const uint32_t qb = qn & 1;
                             if (!mbar_wait(&ctl->q_empty[qb], ((qn >> 1) & 1) ^ 1, ctl, status, kSleepLong)) { ok = false; break; }
                             mbar_expect_tx(&ctl->q_full[qb], q_bytes);
@@ -534,8 +551,10 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                         const bool wt = P.wtile && pass == 1 && tt == tph - 1;
                         const CUtensorMap *map = wt ? &mapW : head_mapK;
                         const int j0 = wt ? 0 : tt * kTile;
-                        tma_load_3d(kbuf + (size_t)st * kStageBytes, map, &ctl->full[st], 0, j0, head_c2);
-                        tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, map, &ctl->full[st], 64, j0, head_c2);
+                        if (JQ_IN(st, stages, kDbgScore, 2)) {
+                            tma_load_3d(kbuf + (size_t)st * kStageBytes, map, &ctl->full[st], 0, j0, head_c2);
+                            tma_load_3d(kbuf + (size_t)st * kStageBytes + kHalfBytes, map, &ctl->full[st], 64, j0, head_c2);
+                        }
                         if (++st == (uint32_t)stages) { st = 0; ph ^= 1; }
                     }
                 }
@@ -569,6 +588,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                         if (!mbar_wait(&ctl->t_empty[slot], ((u / kTSlots) & 1) ^ 1, ctl, status, kSleepShort)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t d = tmem + slot * kSlotCols;
+                        if (!JQ_IN(slot * kSlotCols + kSlotCols - 1, kTmemCols, kDbgScore, 3) || !JQ_IN(st, stages, kDbgScore, 4)) { ok = false; break; }
                         const uint32_t qb_lo = q_lo + (uint32_t)blk * (kHalfBytes >> 4);   // query rows [128 blk, 128 blk + 128)
                         if (pass == 1) tc_mma_block(d, qb_lo, k_lo, q_bytes / 2, kHalfBytes, idesc1);
                         else tc_mma_block(d, k_lo, qb_lo, kHalfBytes, q_bytes / 2, blk == 0 ? idesc2a : idesc2b);
@@ -629,7 +649,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                             p[k] = make_float2(-INFINITY, 0.f);
                             // (a CTA between b_lo and b_hi always has a tile of this head unless the group has fewer tiles than CTAs)
                             if (i < nsl && (T >= Gu || cta_has_tile(b_lo + i / kGroups, T, Gu)))
-                                p[k] = __ldcg(src + (size_t)i * P.R);
+                                if (JQ_IN(((long long)kv * kSlots + kGroups * b_lo + i) * P.R + r, n_part, kDbgScore, 5)) p[k] = __ldcg(src + (size_t)i * P.R);
                         }
                         float mn = m;
 #pragma unroll
@@ -648,7 +668,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     l = (l > 0.f) ? l * ex2(c * (m - mw)) : 0.f;
                     for (int o = lpr >> 1; o >= 1; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
                     const float M = c * mw + log2f(l);
-                    if (have && sub == 0) P.Mrow[(size_t)kv * P.R + r] = M;
+                    if (have && sub == 0 && JQ_IN((long long)kv * P.R + r, (long long)P.Hkv * P.R, kDbgScore, 6)) P.Mrow[(size_t)kv * P.R + r] = M;
                 }
                 __syncwarp();
                 if (lane == 0) {
@@ -672,7 +692,8 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     int kv = sg.kv0, tt = sg.t0;
                     for (int n = 0; n < sg.ntiles; ++n, walk(2, tph, kv, tt)) {
                         float *dst = P.scores + sg.sbase + (size_t)(kv - sg.h0) * sg.L + tt * kTile;
-                        for (int t = lane; t < kTile && tt * kTile + t < sg.L; t += 32) dst[t] = 0.f;
+                        for (int t = lane; t < kTile && tt * kTile + t < sg.L; t += 32)
+                            if (JQ_IN(sg.sbase + (long long)(kv - sg.h0) * sg.L + tt * kTile + t, n_scores, kDbgScore, 7)) dst[t] = 0.f;
                     }
                     __threadfence();
                 }
@@ -691,7 +712,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     for (int r = lane; r < kMaxR; r += 32)   // stored negated: x = c s + (-M_r); -inf silences a padding column
-                        ctl->Ms[buf][r] = (r < P.R) ? -__ldcg(&P.Mrow[(size_t)kv * P.R + r]) : -INFINITY;
+                        ctl->Ms[buf][r] = (r < P.R && JQ_IN((long long)kv * P.R + r, (long long)P.Hkv * P.R, kDbgScore, 8)) ? -__ldcg(&P.Mrow[(size_t)kv * P.R + r]) : -INFINITY;
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->ms_full[buf], 1);
                     ++hs;
@@ -754,8 +775,9 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 #pragma unroll 1
                     for (; pub < head_end; ++pub) {
                         float2 *dst = part_out + (size_t)pub * kSlots * R;
-                        if (row0 < R) dst[row0] = make_float2(st0.m, (st0.l01.x + st0.l01.y) + (st0.l23.x + st0.l23.y));
-                        if (nblk == 2 && row0 + 128 < R)
+                        const bool in_part = JQ_IN(((long long)pub * kSlots + kGroups * blockIdx.x + grp) * R + (R - 1), n_part, kDbgScore, 9);
+                        if (row0 < R && in_part) dst[row0] = make_float2(st0.m, (st0.l01.x + st0.l01.y) + (st0.l23.x + st0.l23.y));
+                        if (nblk == 2 && row0 + 128 < R && in_part)
                             dst[row0 + 128] = make_float2(st1.m, (st1.l01.x + st1.l01.y) + (st1.l23.x + st1.l23.y));
                         st0.m = st1.m = -INFINITY;
                         st0.l01 = st0.l23 = st1.l01 = st1.l23 = make_float2(0.f, 0.f);
@@ -770,6 +792,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     const uint32_t uu = u + (uint32_t)k, slot = uu % kTSlots;
                     if (!pre && !begin(uu)) { ok = false; break; }
                     const uint32_t taddr = lane_addr + slot * kSlotCols;
+                    if (!JQ_IN(slot * kSlotCols + kTile - 1, kTmemCols, kDbgScore, 10)) { ok = false; break; }
                     // keys of this block that count for this thread's row: the prefix keys of the tile, or, in the window
                     // tile, the window keys up to the row's own position (causal)
                     const int valid = (P.wtile && tt == tph - 1) ? min(P.w, (blk ? win_i1 : win_i0) + 1) : min(kTile, L - tt * kTile);
@@ -824,6 +847,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     const uint32_t taddr = lane_addr + slot * kSlotCols;
                     const int np = blk ? np1 : np0;                     // 32-column pieces of this block
                     const float4 *bias = (const float4 *)(ctl->Ms[held & 1] + blk * 128);  // columns that are not query rows carry a bias of -inf
+                    if (!JQ_IN(slot * kSlotCols + 32 * np - 1, kTmemCols, kDbgScore, 11) || !JQ_IN(blk * 128 + 32 * np - 1, kMaxR, kDbgScore, 12)) { ok = false; break; }
                     float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
 #pragma unroll 1
                     for (int p = 0; p < np; ++p) {
@@ -839,7 +863,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                         exp_acc16(a01, a23, vb, cc, bias + 8 * p + 4);
                     }
                     const int key = tt * kTile + row0;
-                    if (key < L) {
+                    if (key < L && JQ_IN(sg.sbase + (long long)(kv - sg.h0) * L + key, n_scores, kDbgScore, 13)) {
                         float *dst = scores_out + sg.sbase + (size_t)(kv - sg.h0) * L + key;
                         const float sum = (a01.x + a01.y) + (a23.x + a23.y);
                         if (nblk == 1) *dst = sum;
@@ -1029,13 +1053,13 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
         // every unit has tensor maps of its own in device memory; the three parameter maps are not used
         memset(&mapK, 0, sizeof mapK); mapQ = mapK; mapW = mapK;
         P.L = 0; P.tph = 0; P.hpg = 0;
-        P.gtab = tables->groups; P.maps = (const CUtensorMap *)tables->maps;
+        P.gtab = tables->groups; P.maps = (const CUtensorMap *)tables->maps; P.hpu = tables->hpu;
         P.ngroups = tables->ngroups;
         tmax = tables->max_group_tiles;
     } else {
         P.L = s.L;
         P.tph = (s.L + kTile - 1) / kTile + P.wtile;
-        P.gtab = nullptr; P.maps = nullptr;
+        P.gtab = nullptr; P.maps = nullptr; P.hpu = s.Hkv;
         if (!make_map(&mapK, K, s.L, s.Hkv, kTile, k_head_rows) || !make_map(&mapQ, Q, R, s.Hkv, P.Rbox)) return JQ_ERR_CUDA;
         if (Kwin) { if (!make_map(&mapW, Kwin, s.w, s.Hkv, kTile)) return JQ_ERR_CUDA; } else mapW = mapK;
         P.hpg = heads_per_group(s.L, s.Hkv, P.tph, sms);
@@ -1043,6 +1067,11 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
         tmax = (long long)(P.hpg < s.Hkv ? P.hpg : s.Hkv) * P.tph;
     }
     const int grid = (int)(tmax < sms ? tmax : sms);
+#ifdef JQ_DEBUG
+    P.dbg_rec = debug_record();
+    P.n_scores = tables ? tables->total_keys : (long long)s.Hkv * s.L;
+    if (!P.dbg_rec) return JQ_ERR_CUDA;
+#endif
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);

@@ -18,6 +18,7 @@
 //   4. (fused layer path only) the cluster copies the kept K and V rows of its head.
 // Everything is integer arithmetic on bit patterns, hence deterministic and exact.
 #include "jq_internal.cuh"
+#include "jq_debug.cuh"
 #include <cooperative_groups.h>
 
 namespace cg = cooperative_groups;
@@ -33,6 +34,13 @@ constexpr int kHalo = 32;          // >= pool radius
 constexpr int kKeysSmemMax = 24576; // keys a CTA can keep in shared memory
 constexpr int kCandMax = 8192;     // candidates the leading CTA finishes alone (they live in its staging buffer)
 static_assert(kCandMax <= kRawTile, "candidates are kept in the staging buffer");
+
+// Extents of what the kernel indexes (read by the bounds-checked build only).
+struct SelExtents {
+    long long scores;     // floats in the scores array (and keys in the global key array)
+    long long out_rows;   // rows of the stacked outputs (kept indices, compacted K and V)
+    long long src_heads;  // heads in one source buffer of K / V
+};
 
 struct SelCtl {
     uint32_t prefix;
@@ -101,7 +109,8 @@ __device__ __forceinline__ void find_digit(const uint32_t *g, int krem, SelCtl &
 // kv_in: the head's index within the buffer the rows come from; orow: the head's first row in the outputs.
 template <int CL>
 __device__ __forceinline__ void copy_kept_rows(cg::cluster_group &cluster, const int32_t *out, int kv_in, long long orow, int L, int nkeep,
-                                               const uint4 *Kin, const uint4 *Vin, uint4 *Kout, uint4 *Vout, int src_rows)
+                                               const uint4 *Kin, const uint4 *Vin, uint4 *Kout, uint4 *Vout, int src_rows,
+                                               const SelExtents &ext JQ_DBG_PARAM)
 {
     __threadfence();
     cluster.sync();
@@ -111,8 +120,10 @@ __device__ __forceinline__ void copy_kept_rows(cg::cluster_group &cluster, const
     for (int t = r0 + (int)(threadIdx.x >> 4); t < r1; t += kSelThreads / 16) {
         const int j = min(max(__ldcg(out + t), 0), L - 1);
         const size_t src = ((size_t)kv_in * src_rows + j) * 16 + lane16, dst = (size_t)(orow + t) * 16 + lane16;
-        Kout[dst] = Kin[src];
-        Vout[dst] = Vin[src];
+        if (JQ_IN((long long)kv_in * src_rows + j, ext.src_heads * src_rows, kDbgSelect, 1) && JQ_IN(orow + t, ext.out_rows, kDbgSelect, 2)) {
+            Kout[dst] = Kin[src];
+            Vout[dst] = Vin[src];
+        }
     }
 }
 
@@ -125,7 +136,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
                float *__restrict__ pooled, uint32_t *__restrict__ gkeys, int chunk, int keys_in_smem, int raw_tile,
                const uint4 *__restrict__ Kin, const uint4 *__restrict__ Vin, uint4 *__restrict__ Kout,
                uint4 *__restrict__ Vout, const HeadRec *__restrict__ htab, const uint4 *const *__restrict__ Ktab,
-               const uint4 *const *__restrict__ Vtab, int src_rows)
+               const uint4 *const *__restrict__ Vtab, int src_rows, const SelExtents ext JQ_DBG_PARAM)
 {
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
@@ -140,6 +151,8 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     __shared__ SelCtl ctl;
 
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int raw_cap = raw_tile + 2 * kHalo, keys_cap = keys_in_smem ? chunk : 0;   // shared-memory extents (those of the launch)
+    (void)raw_cap; (void)keys_cap;
     cudaGridDependencySynchronize();   // everything above ran while the previous kernel of the stream was finishing
     if (htab) {
         const HeadRec r = htab[kv];
@@ -167,13 +180,13 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
                 const int j = j0 + t0 - radius + i0 + q * kSelThreads;
-                vals[q] = (i0 + q * kSelThreads < tile + 2 * radius && j >= 0 && j < L) ? __ldcg(s + j) : -INFINITY;
+                vals[q] = (i0 + q * kSelThreads < tile + 2 * radius && j >= 0 && j < L && JQ_IN(soff + j, ext.scores, kDbgSelect, 3)) ? __ldcg(s + j) : -INFINITY;
             }
 #pragma unroll
             for (int q = 0; q < 8; ++q)
-                if (i0 + q * kSelThreads < tile + 2 * radius) raw[i0 + q * kSelThreads] = vals[q];
+                if (i0 + q * kSelThreads < tile + 2 * radius && JQ_IN(i0 + q * kSelThreads, raw_cap, kDbgSelect, 4)) raw[i0 + q * kSelThreads] = vals[q];
         }
-        if (fast_pool) for (int i = tid; i < 8; i += kSelThreads) raw[tile + 2 * radius + i] = -INFINITY;   // its 16-byte reads run a little past the window
+        if (fast_pool) for (int i = tid; i < 8; i += kSelThreads) if (JQ_IN(tile + 2 * radius + i, raw_cap, kDbgSelect, 5)) raw[tile + 2 * radius + i] = -INFINITY;   // its 16-byte reads run a little past the window
         __syncthreads();
         if (fast_pool) {
             const int nquads = (tile + 3) / 4;
@@ -183,8 +196,9 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
                 const bool act = g4 < nquads;
                 float x[12];
                 {
-                    const float4 a = act ? raw4[g4] : make_float4(0.f, 0.f, 0.f, 0.f);
-                    const float4 b = act ? raw4[g4 + 1] : a, c = act ? raw4[g4 + 2] : a;
+                    const bool rd = act && JQ_IN(4 * (g4 + 2) + 3, raw_cap, kDbgSelect, 6);
+                    const float4 a = rd ? raw4[g4] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    const float4 b = rd ? raw4[g4 + 1] : a, c = rd ? raw4[g4 + 2] : a;
                     x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
                     x[8] = c.x; x[9] = c.y; x[10] = c.z; x[11] = c.w;
                 }
@@ -199,7 +213,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
                     key[i] = order_key(m);
                 }
                 const int nval = act ? min(4, tile - 4 * g4) : 0;          // positions of this quad inside the tile
-                if (act) {
+                if (act && JQ_IN(t0 + 4 * g4 + nval - 1, keys_cap, kDbgSelect, 7) && (!pooled || JQ_IN(soff + j0 + t0 + 4 * g4 + nval - 1, ext.scores, kDbgSelect, 8))) {
                     if (nval == 4) *(uint4 *)(mykeys + t0 + 4 * g4) = make_uint4(key[0], key[1], key[2], key[3]);
                     else for (int i = 0; i < nval; ++i) mykeys[t0 + 4 * g4 + i] = key[i];
                     if (pooled) for (int i = 0; i < nval; ++i) pooled[j0 + t0 + 4 * g4 + i] = best[i];
@@ -212,7 +226,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
                 const uint32_t lead = __shfl_sync(0xffffffffu, d0, 0);
                 if (__all_sync(0xffffffffu, nval == 0 || (same && d0 == lead))) {
                     const int tot = __reduce_add_sync(0xffffffffu, nval);
-                    if (lane == 0 && tot) atomicAdd(&hist[lead], (uint32_t)tot);
+                    if (lane == 0 && tot && JQ_IN(lead, kBins, kDbgSelect, 9)) atomicAdd(&hist[lead], (uint32_t)tot);
                 } else {
                     uint32_t cur = 0, cnt = 0;
                     for (int i = 0; i < nval; ++i) {
@@ -227,15 +241,16 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         }
 #pragma unroll 4
         for (int e = tid; e < tile; e += kSelThreads) {
+            if (!JQ_IN(e + 2 * radius, raw_cap, kDbgSelect, 10)) continue;
             float best = raw[e];
             for (int u = 1; u <= 2 * radius; ++u) best = fmaxf(best, raw[e + u]);
-            mykeys[t0 + e] = order_key(best);
-            if (pooled) pooled[j0 + t0 + e] = best;
+            if (JQ_IN(keys_in_smem ? t0 + e : soff + j0 + t0 + e, keys_in_smem ? keys_cap : ext.scores, kDbgSelect, 11)) mykeys[t0 + e] = order_key(best);
+            if (pooled && JQ_IN(soff + j0 + t0 + e, ext.scores, kDbgSelect, 12)) pooled[j0 + t0 + e] = best;
         }
     }
     if (nkeep >= L) {   // everything is kept (uniform over the cluster; no cluster traffic yet)
-        for (int e = tid; e < n; e += kSelThreads) out[j0 + e] = j0 + e;
-        if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, orow, L, nkeep, Kin, Vin, Kout, Vout, src_rows);
+        for (int e = tid; e < n; e += kSelThreads) if (JQ_IN(orow + j0 + e, ext.out_rows, kDbgSelect, 13)) out[j0 + e] = j0 + e;
+        if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, orow, L, nkeep, Kin, Vin, Kout, Vout, src_rows, ext JQ_DBG_ARG_DEV);
         return;
     }
     for (int i = tid; i < 3 * kBins; i += kSelThreads) ghist[i] = 0;
@@ -263,6 +278,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
                 const int e = e0 + pos;
                 if (++pos == per) pos = 0;
                 if (e >= e1) continue;
+                if (!JQ_IN(keys_in_smem ? e : soff + j0 + e, keys_in_smem ? keys_cap : ext.scores, kDbgSelect, 14)) continue;
                 const uint32_t k = mykeys[e];
                 const bool live = (round == 0) || ((k >> (shift + width)) == prefix);
                 const uint32_t digit = live ? ((k >> shift) & mask) : 0xffffffffu;
@@ -299,14 +315,14 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
             int *cand_count = &cluster.map_shared_rank(&ctl, 0)->cand_count;
             for (int base = 0; base < n_up; base += kSelThreads) {
                 const int e = base + tid;
-                const uint32_t k = (e < n) ? mykeys[e] : 0u;
+                const uint32_t k = (e < n && JQ_IN(keys_in_smem ? e : soff + j0 + e, keys_in_smem ? keys_cap : ext.scores, kDbgSelect, 19)) ? mykeys[e] : 0u;
                 const bool hit = e < n && (k >> 21) == d0;
                 const uint32_t votes = __ballot_sync(0xffffffffu, hit);
                 if (votes) {
                     int at = 0;
                     if (lane == 0) at = atomicAdd(cand_count, __popc(votes));
                     at = __shfl_sync(0xffffffffu, at, 0);
-                    if (hit) cand[at + __popc(votes & ((1u << lane) - 1u))] = k;
+                    if (hit && JQ_IN(at + __popc(votes & ((1u << lane) - 1u)), raw_cap, kDbgSelect, 15)) cand[at + __popc(votes & ((1u << lane) - 1u))] = k;
                 }
             }
             cluster.sync();
@@ -320,7 +336,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
                     __syncthreads();
                     for (int e = tid; e < nc; e += kSelThreads) {
                         const uint32_t k = mine[e];
-                        if ((k >> (sh + wd)) == pre) atomicAdd(&hist[(k >> sh) & ((1u << wd) - 1u)], 1u);
+                        if ((k >> (sh + wd)) == pre && JQ_IN((k >> sh) & ((1u << wd) - 1u), kBins, kDbgSelect, 16)) atomicAdd(&hist[(k >> sh) & ((1u << wd) - 1u)], 1u);
                     }
                     __syncthreads();
                     find_digit(hist, ctl.krem, ctl);
@@ -347,7 +363,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     int cgt = 0, ceq = 0;
     for (int base = w0; base < w1; base += 32) {
         const int e = base + lane;
-        const uint32_t k = (e < w1) ? mykeys[e] : 0u;
+        const uint32_t k = (e < w1 && JQ_IN(keys_in_smem ? e : soff + j0 + e, keys_in_smem ? keys_cap : ext.scores, kDbgSelect, 20)) ? mykeys[e] : 0u;
         const bool in = e < w1;
         cgt += __popc(__ballot_sync(0xffffffffu, in && k > tau));
         ceq += __popc(__ballot_sync(0xffffffffu, in && k == tau));
@@ -378,18 +394,18 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     for (int base = w0; base < w1; base += 32) {
         const int e = base + lane;
         const bool in = e < w1;
-        const uint32_t k = in ? mykeys[e] : 0u;
+        const uint32_t k = (in && JQ_IN(keys_in_smem ? e : soff + j0 + e, keys_in_smem ? keys_cap : ext.scores, kDbgSelect, 21)) ? mykeys[e] : 0u;
         const uint32_t bg = __ballot_sync(0xffffffffu, in && k > tau);
         const uint32_t be = __ballot_sync(0xffffffffu, in && k == tau);
         const int g_here = gt_before + __popc(bg & lt_mask), e_here = eq_before + __popc(be & lt_mask);
         if (in) {
-            if (k > tau) out[g_here + min(e_here, need_eq)] = j0 + e;
-            else if (k == tau && e_here < need_eq) out[g_here + e_here] = j0 + e;
+            if (k > tau) { if (JQ_IN(g_here + min(e_here, need_eq), nkeep, kDbgSelect, 17)) out[g_here + min(e_here, need_eq)] = j0 + e; }
+            else if (k == tau && e_here < need_eq) { if (JQ_IN(g_here + e_here, nkeep, kDbgSelect, 18)) out[g_here + e_here] = j0 + e; }
         }
         gt_before += __popc(bg);
         eq_before += __popc(be);
     }
-    if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, orow, L, nkeep, Kin, Vin, Kout, Vout, src_rows);
+    if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, orow, L, nkeep, Kin, Vin, Kout, Vout, src_rows, ext JQ_DBG_ARG_DEV);
 }
 
 // Shared memory of a CTA whose cluster has `cl` CTAs, the share of the head it holds, and whether its keys stay on chip.
@@ -441,6 +457,10 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
             return JQ_ERR_CUDA;
         attr_done[dev] = true;
     }
+    SelExtents ext;
+    ext.scores = tables ? tables->total_keys : (long long)s.Hkv * s.L;
+    ext.out_rows = tables ? tables->total_rows : (long long)s.Hkv * nkeep;
+    ext.src_heads = tables ? tables->hpu : s.Hkv;
     // Launched with programmatic stream serialisation: the CTAs may be set up while the kernel before it in
     // the stream (the scoring kernel) drains; the kernel waits for that kernel's memory before reading anything.
     cudaLaunchConfig_t cfg = {};
@@ -456,7 +476,7 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
     if (cudaLaunchKernelEx(&cfg, select_cluster<CL>, scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, w.keys, p.chunk,
                            p.in_smem, p.raw_tile, (const uint4 *)K, (const uint4 *)V, (uint4 *)Kout, (uint4 *)Vout,
                            tables ? tables->heads : nullptr, (const uint4 *const *)(tables && Kout ? tables->K : nullptr),
-                           (const uint4 *const *)(tables && Kout ? tables->V : nullptr), src_rows) != cudaSuccess) {
+                           (const uint4 *const *)(tables && Kout ? tables->V : nullptr), src_rows, ext JQ_DBG_ARG) != cudaSuccess) {
         cudaGetLastError();
         return JQ_ERR_CUDA;
     }
