@@ -108,6 +108,18 @@ jq_status jq_evict_layer_windowed(const void *K, const void *V, const void *Qwin
                                   void *ws, size_t ws_bytes, jq_stream_t stream);
 
 /*
+ * The window-inclusive pass with the window itself retained, the way the last-window methods of the paper's
+ * experimental section use their budget: of `budget` rows per KV head, w are the query positions' own pairs
+ * (always kept) and budget - w are chosen among the L prefix positions by jq_evict_layer_windowed's scores.
+ * Vwin [Hkv, w, d] bf16: the values of the query positions.  Kout, Vout: bf16 [Hkv, np + w, d] with
+ * np = min(budget - w, L): the kept prefix rows in ascending position, then the w window rows in order.
+ * kept_idx [Hkv, np] int32: the kept prefix positions.  Needs w <= 128 and budget > w (JQ_ERR_INVALID_ARG).
+ */
+jq_status jq_evict_layer_window_kept(const void *K, const void *V, const void *Qwin, const void *Kwin, const void *Vwin,
+                                     const jq_shape *shape, void *Kout, void *Vout, int32_t *kept_idx, void *ws,
+                                     size_t ws_bytes, jq_stream_t stream);
+
+/*
  * jq_score for callers that cannot allocate device memory: an inference server that has handed every
  * free byte of the GPU to its KV-cache pool, a plug-in running inside somebody else's memory budget, a
  * call site that must not touch the allocator.  (The paper has no counterpart; this is a property of

@@ -20,7 +20,7 @@ EXPORTS = (
     "jq_score_static", "jq_score_windowed", "jq_evict_layer_windowed", "jq_hit_rate",
     "jq_decode_workspace_bytes", "jq_decode_attention", "jq_layers_workspace_bytes", "jq_evict_layers",
     "jq_ragged_workspace_bytes", "jq_ragged_output_rows", "jq_evict_ragged",
-    "jq_append_workspace_bytes", "jq_evict_append",
+    "jq_append_workspace_bytes", "jq_evict_append", "jq_evict_layer_window_kept",
 )
 
 
@@ -70,6 +70,7 @@ def lib():
         L.jq_ragged_output_rows.argtypes = [sp, ci, vp, vp]
         L.jq_ragged_output_rows.restype = ctypes.c_longlong
         L.jq_evict_ragged.argtypes = [vp, vp, vp, ci, sp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.jq_evict_layer_window_kept.argtypes = [vp, vp, vp, vp, vp, sp, vp, vp, vp, vp, sz, vp]
         L.jq_append_workspace_bytes.argtypes = [sp]
         L.jq_append_workspace_bytes.restype = ctypes.c_size_t
         L.jq_evict_append.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, sp, vp, vp, sz, vp]
@@ -177,6 +178,13 @@ def evict_layer_windowed(K, V, Qwin, Kwin, s, Kout, Vout, kept_idx, ws, stream=N
     _raise("jq_evict_layer_windowed",
            lib().jq_evict_layer_windowed(_ptr(K), _ptr(V), _ptr(Qwin), _ptr(Kwin), ctypes.byref(s), _ptr(Kout), _ptr(Vout),
                                          _ptr(kept_idx), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def evict_layer_window_kept(K, V, Qwin, Kwin, Vwin, s, Kout, Vout, kept_idx, ws, stream=None):
+    """jq_evict_layer_window_kept: budget - w prefix rows chosen by the window-inclusive scores, then the w window rows."""
+    _raise("jq_evict_layer_window_kept",
+           lib().jq_evict_layer_window_kept(_ptr(K), _ptr(V), _ptr(Qwin), _ptr(Kwin), _ptr(Vwin), ctypes.byref(s), _ptr(Kout),
+                                            _ptr(Vout), _ptr(kept_idx), _ptr(ws), ws.numel(), _stream(stream)))
 
 
 def select_topk(scores, s, kept_idx, ws, pooled=None, stream=None):

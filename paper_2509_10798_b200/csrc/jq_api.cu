@@ -102,6 +102,33 @@ jq_status jq_evict_layer_windowed(const void *K, const void *V, const void *Qwin
     return launch_select(w.scores, *s, kept_idx, nullptr, w, st, K, V, Kout, Vout);
 }
 
+jq_status jq_evict_layer_window_kept(const void *K, const void *V, const void *Qwin, const void *Kwin, const void *Vwin,
+                                     const jq_shape *s, void *Kout, void *Vout, int32_t *kept_idx, void *ws, size_t ws_bytes,
+                                     jq_stream_t stream)
+{
+    jq_status rc = check_shape(s);
+    if (rc != JQ_OK) return rc;
+    if (s->w > 128) return JQ_ERR_UNSUPPORTED;                 // the window keys of a head must fit one tile
+    if (s->budget <= s->w) return JQ_ERR_INVALID_ARG;          // the window alone would fill the budget
+    if (!aligned16(K) || !aligned16(V) || !aligned16(Qwin) || !aligned16(Kwin) || !aligned16(Vwin) || !aligned16(Kout) ||
+        !aligned16(Vout) || !aligned16(kept_idx))
+        return JQ_ERR_INVALID_ARG;
+    Workspace w;
+    if ((rc = check_ws(s, ws, ws_bytes, &w)) != JQ_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    // prefix rows: the window-inclusive pass with budget - w; then the w window rows behind them, head by head
+    jq_shape sp = *s;
+    sp.budget = s->budget - s->w;
+    const size_t row = (size_t)s->d * 2, np = (size_t)(sp.budget < s->L ? sp.budget : s->L), nt = np + (size_t)s->w;
+    // the kept prefix rows of head kv go to rows [kv * nt, kv * nt + np) of the outputs, its window rows behind them
+    if ((rc = launch_score_tc(K, Qwin, sp, w.scores, w, st, Kwin)) != JQ_OK) return rc;
+    if ((rc = launch_select(w.scores, sp, kept_idx, nullptr, w, st, K, V, Kout, Vout, nullptr, 0, (int)nt)) != JQ_OK) return rc;
+    if (cudaMemcpy2DAsync((char *)Kout + np * row, nt * row, Kwin, (size_t)s->w * row, (size_t)s->w * row, (size_t)s->Hkv, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+        cudaMemcpy2DAsync((char *)Vout + np * row, nt * row, Vwin, (size_t)s->w * row, (size_t)s->w * row, (size_t)s->Hkv, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return JQ_ERR_CUDA;
+    return JQ_OK;
+}
+
 jq_status jq_score_fma(const void *K, const void *Qwin, const jq_shape *s, float *scores, void *ws,
                        size_t ws_bytes, jq_stream_t stream)
 {

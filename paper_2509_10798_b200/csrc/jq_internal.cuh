@@ -113,11 +113,12 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
                           const UnitTables *tables = nullptr, int k_head_rows = 0);
 // With K, V, Kout, Vout given, the kernel also copies the kept rows (the fused layer path).  With tables, every
 // head has a length, a budget and offsets of its own (s.L, s.budget unused).
-// src_head_rows: rows between consecutive heads of K and V in memory when the heads are not packed (0: s.L).
+// src_head_rows: rows between consecutive heads of K and V in memory when the heads are not packed (0: s.L);
+// out_head_rows: rows between consecutive heads of Kout and Vout when more than nkeep (0: nkeep).
 jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, float *pooled,
                         const Workspace &w, cudaStream_t st, const void *K = nullptr, const void *V = nullptr,
                         void *Kout = nullptr, void *Vout = nullptr, const UnitTables *tables = nullptr,
-                        int src_head_rows = 0);
+                        int src_head_rows = 0, int out_head_rows = 0);
 jq_status launch_gather(const void *K, const void *V, const int32_t *idx, const jq_shape &s,
                         void *Kout, void *Vout, cudaStream_t st);
 

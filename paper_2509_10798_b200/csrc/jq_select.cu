@@ -136,13 +136,14 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
                float *__restrict__ pooled, uint32_t *__restrict__ gkeys, int chunk, int keys_in_smem, int raw_tile,
                const uint4 *__restrict__ Kin, const uint4 *__restrict__ Vin, uint4 *__restrict__ Kout,
                uint4 *__restrict__ Vout, const HeadRec *__restrict__ htab, const uint4 *const *__restrict__ Ktab,
-               const uint4 *const *__restrict__ Vtab, int src_rows, const SelExtents ext JQ_DBG_PARAM)
+               const uint4 *const *__restrict__ Vtab, int src_rows, int out_rows, const SelExtents ext JQ_DBG_PARAM)
 {
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
     const int kv = blockIdx.x / CL;
     int kv_in = kv;                                  // the head's index within the buffer its rows come from
-    long long soff = (long long)kv * L, orow = (long long)kv * nkeep;
+    long long soff = (long long)kv * L, orow = (long long)kv * nkeep;   // offsets of the head's scores and of its kept indices
+    long long krow = (long long)kv * out_rows;                          // first row of the head in the compacted outputs
     extern __shared__ __align__(16) uint8_t sm[];
     uint32_t *ghist = (uint32_t *)sm;                       // [3][kBins]; the leading CTA's copy accumulates the cluster
     uint32_t *hist = ghist + 3 * kBins;                     // [kBins]
@@ -156,7 +157,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     cudaGridDependencySynchronize();   // everything above ran while the previous kernel of the stream was finishing
     if (htab) {
         const HeadRec r = htab[kv];
-        L = r.L; nkeep = r.nkeep; kv_in = r.kv_in; soff = r.soff; orow = r.ooff; src_rows = L;
+        L = r.L; nkeep = r.nkeep; kv_in = r.kv_in; soff = r.soff; orow = r.ooff; krow = r.ooff; src_rows = L;
         chunk = ((L + CL - 1) / CL + 31) / 32 * 32;   // (keys_in_smem stays the launch's: the longest head decides whether the region exists)
         if (Ktab) { Kin = Ktab[r.unit]; Vin = Vtab[r.unit]; }
     }
@@ -250,7 +251,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     }
     if (nkeep >= L) {   // everything is kept (uniform over the cluster; no cluster traffic yet)
         for (int e = tid; e < n; e += kSelThreads) if (JQ_IN(orow + j0 + e, ext.out_rows, kDbgSelect, 13)) out[j0 + e] = j0 + e;
-        if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, orow, L, nkeep, Kin, Vin, Kout, Vout, src_rows, ext JQ_DBG_ARG_DEV);
+        if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, krow, L, nkeep, Kin, Vin, Kout, Vout, src_rows, ext JQ_DBG_ARG_DEV);
         return;
     }
     for (int i = tid; i < 3 * kBins; i += kSelThreads) ghist[i] = 0;
@@ -405,7 +406,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         gt_before += __popc(bg);
         eq_before += __popc(be);
     }
-    if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, orow, L, nkeep, Kin, Vin, Kout, Vout, src_rows, ext JQ_DBG_ARG_DEV);
+    if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, krow, L, nkeep, Kin, Vin, Kout, Vout, src_rows, ext JQ_DBG_ARG_DEV);
 }
 
 // Shared memory of a CTA whose cluster has `cl` CTAs, the share of the head it holds, and whether its keys stay on chip.
@@ -448,7 +449,7 @@ SelPlan choose_plan(int Hkv, int L, int sms)
 template <int CL>
 jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape &s, int nkeep, int32_t *idx, float *pooled,
                            const Workspace &w, cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout, int dev,
-                           const UnitTables *tables, int src_rows)
+                           const UnitTables *tables, int src_rows, int out_rows)
 {
     static bool attr_done[64] = {};
     if (!attr_done[dev]) {
@@ -459,7 +460,7 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
     }
     SelExtents ext;
     ext.scores = tables ? tables->total_keys : (long long)s.Hkv * s.L;
-    ext.out_rows = tables ? tables->total_rows : (long long)s.Hkv * nkeep;
+    ext.out_rows = tables ? tables->total_rows : (long long)s.Hkv * out_rows;
     ext.src_heads = tables ? tables->hpu : s.Hkv;
     // Launched with programmatic stream serialisation: the CTAs may be set up while the kernel before it in
     // the stream (the scoring kernel) drains; the kernel waits for that kernel's memory before reading anything.
@@ -476,7 +477,7 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
     if (cudaLaunchKernelEx(&cfg, select_cluster<CL>, scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, w.keys, p.chunk,
                            p.in_smem, p.raw_tile, (const uint4 *)K, (const uint4 *)V, (uint4 *)Kout, (uint4 *)Vout,
                            tables ? tables->heads : nullptr, (const uint4 *const *)(tables && Kout ? tables->K : nullptr),
-                           (const uint4 *const *)(tables && Kout ? tables->V : nullptr), src_rows, ext JQ_DBG_ARG) != cudaSuccess) {
+                           (const uint4 *const *)(tables && Kout ? tables->V : nullptr), src_rows, out_rows, ext JQ_DBG_ARG) != cudaSuccess) {
         cudaGetLastError();
         return JQ_ERR_CUDA;
     }
@@ -488,7 +489,7 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
 
 jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, float *pooled,
                         const Workspace &w, cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout,
-                        const UnitTables *tables, int src_head_rows)
+                        const UnitTables *tables, int src_head_rows, int out_head_rows)
 {
     const int src_rows = src_head_rows > s.L ? src_head_rows : s.L;
     // with tables: the plan and the shared memory follow the longest head; every head reads its own record
@@ -500,9 +501,9 @@ jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, fl
     if (!sms[dev] && cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return JQ_ERR_CUDA;
     const SelPlan p = choose_plan(s.Hkv, Lmax, sms[dev]);
     switch (p.cl) {
-    case 2: return launch_select_cl<2>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables, src_rows);
-    case 4: return launch_select_cl<4>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables, src_rows);
-    default: return launch_select_cl<8>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables, src_rows);
+    case 2: return launch_select_cl<2>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables, src_rows, out_head_rows > nkeep ? out_head_rows : nkeep);
+    case 4: return launch_select_cl<4>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables, src_rows, out_head_rows > nkeep ? out_head_rows : nkeep);
+    default: return launch_select_cl<8>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables, src_rows, out_head_rows > nkeep ? out_head_rows : nkeep);
     }
 }
 

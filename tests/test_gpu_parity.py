@@ -653,6 +653,30 @@ def test_evict_ragged_rejects_bad_arguments():
     assert jq.ragged_output_rows(s, 2, [500, 300], [10, 1000]) == 2 * (10 + 300)
 
 
+def test_evict_layer_window_kept_keeps_the_window_and_fills_the_rest():
+    """budget rows per head = the w window pairs (always) + budget - w prefix rows chosen by the window-inclusive
+    scores; expected: the oracle's windowed scores, pooled, top-(budget - w), then the window rows."""
+    wl = small_wl(3, 4, 32, 3000, 500)
+    K, V, Q, _ = W.make_layer(wl)
+    Kw = W.make_window_keys(wl, Q)
+    Vw = W.make_v(small_wl(3, 4, 32, wl.w, 1), 777)
+    s = shape_of(wl)
+    np_ = wl.budget - wl.w
+    Ko = torch.zeros((wl.Hkv, wl.budget, 128), dtype=torch.bfloat16, device="cuda"); Vo = torch.zeros_like(Ko)
+    idx = torch.full((wl.Hkv, np_), -1, dtype=torch.int32, device="cuda")
+    ws = jq.new_workspace(s)
+    jq.evict_layer_window_kept(dev_bf16(K), dev_bf16(V), dev_bf16(Q), dev_bf16(Kw), dev_bf16(Vw), s, Ko, Vo, idx, ws)
+    assert jq.last_device_status(ws) == jq.JQ_OK
+    gi, gK, gV = idx.cpu().numpy(), host_bits(Ko), host_bits(Vo)
+    pooled = oracle.pool(oracle.score_windowed(K, Q, Kw), wl.pool)
+    assert_kept_sets_agree(gi, oracle.select(pooled, np_), pooled, np_)
+    for kv in range(wl.Hkv):
+        assert np.array_equal(gK[kv, :np_], K[kv][gi[kv]]) and np.array_equal(gV[kv, :np_], V[kv][gi[kv]])
+        assert np.array_equal(gK[kv, np_:], Kw[kv]) and np.array_equal(gV[kv, np_:], Vw[kv])
+    with pytest.raises(jq.JqError):
+        jq.evict_layer_window_kept(dev_bf16(K), dev_bf16(V), dev_bf16(Q), dev_bf16(Kw), dev_bf16(Vw), shape_of(wl.with_budget(32)), Ko, Vo, idx, ws)
+
+
 # ------------------------------------------------------------------ streaming re-eviction
 
 @pytest.mark.parametrize("Hkv,g,w,n_old,n_new,budget,cap", [(2, 4, 16, 512, 100, 512, 640), (2, 4, 64, 300, 1, 200, 301),
