@@ -145,8 +145,8 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     long long soff = (long long)kv * L, orow = (long long)kv * nkeep;   // offsets of the head's scores and of its kept indices
     long long krow = (long long)kv * out_rows;                          // first row of the head in the compacted outputs
     extern __shared__ __align__(16) uint8_t sm[];
-    uint32_t *ghist = (uint32_t *)sm;                       // [3][kBins]; the leading CTA's copy accumulates the cluster
-    uint32_t *hist = ghist + 3 * kBins;                     // [kBins]
+    uint32_t *ghist = (uint32_t *)sm;                       // [kBins]; the leading CTA's copy accumulates the cluster's histogram of a round
+    uint32_t *hist = ghist + kBins;                         // [kBins]
     float *raw = (float *)(hist + kBins);                   // [raw_tile + 2*kHalo]; later the candidate keys
     uint32_t *keys_s = (uint32_t *)(raw + raw_tile + 2 * kHalo);
     __shared__ SelCtl ctl;
@@ -254,7 +254,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
         if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, krow, L, nkeep, Kin, Vin, Kout, Vout, src_rows, ext JQ_DBG_ARG_DEV);
         return;
     }
-    for (int i = tid; i < 3 * kBins; i += kSelThreads) ghist[i] = 0;
+    for (int i = tid; i < kBins; i += kSelThreads) ghist[i] = 0;
     if (tid == 0) { ctl.prefix = 0; ctl.krem = nkeep; ctl.cand_count = 0; ctl.cand_total = 0; }
     cluster.sync();
 
@@ -292,20 +292,21 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
             if (cnt && cur != 0xffffffffu) atomicAdd(&hist[cur], cnt);
         }
         __syncthreads();
-        uint32_t *g0 = cluster.map_shared_rank(ghist + round * kBins, 0);
+        uint32_t *g0 = cluster.map_shared_rank(ghist, 0);
         for (int i = tid; i < kBins; i += kSelThreads) {
             const uint32_t v = hist[i];
             if (v) atomicAdd(&g0[i], v);
         }
         cluster.sync();
         if (rank == 0) {
-            find_digit(ghist + round * kBins, ctl.krem, ctl);
+            find_digit(ghist, ctl.krem, ctl);
             if (tid < CL) {
                 SelCtl *rc = cluster.map_shared_rank(&ctl, tid);
                 rc->prefix = (prefix << width) | (uint32_t)ctl.found_prefix_digit;
                 rc->krem = ctl.found_krem;
                 rc->cand_total = ctl.found_count;
             }
+            for (int i = tid; i < kBins; i += kSelThreads) ghist[i] = 0;   // for the next round, before anybody adds to it
         }
         cluster.sync();
         if (round == 0 && ctl.cand_total <= kCandMax) {
@@ -412,17 +413,19 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
 // Shared memory of a CTA whose cluster has `cl` CTAs, the share of the head it holds, and whether its keys stay on chip.
 struct SelPlan { int cl, chunk, in_smem, raw_tile; size_t smem; };
 
-SelPlan plan_for(int L, int cl)
+// small_stage: stage the scores in pieces of kCandMax (the least the buffer must hold) instead of a CTA's whole
+// share, so that two CTAs fit on an SM; worth it when the call has more heads than clusters fit at a time.
+SelPlan plan_for(int L, int cl, bool small_stage)
 {
     SelPlan p;
     p.cl = cl;
     p.chunk = ((L + cl - 1) / cl + 31) / 32 * 32;
     p.in_smem = p.chunk <= kKeysSmemMax;
-    // the staging buffer holds a CTA's share of the scores (at most kRawTile) and later up to kCandMax candidates;
-    // sized to the shape so that two CTAs fit on an SM when the share is short
+    // the staging buffer holds a CTA's share of the scores (at most kRawTile) and later up to kCandMax candidates
     p.raw_tile = p.chunk < kRawTile ? p.chunk : kRawTile;
+    if (small_stage && p.in_smem) p.raw_tile = kCandMax;
     if (p.raw_tile < kCandMax) p.raw_tile = kCandMax;
-    p.smem = (size_t)(4 * kBins + p.raw_tile + 2 * kHalo) * 4 + (p.in_smem ? (size_t)p.chunk * 4 : 0);
+    p.smem = (size_t)(2 * kBins + p.raw_tile + 2 * kHalo) * 4 + (p.in_smem ? (size_t)p.chunk * 4 : 0);
     return p;
 }
 
@@ -433,12 +436,13 @@ SelPlan plan_for(int L, int cl)
 // time of one.
 SelPlan choose_plan(int Hkv, int L, int sms)
 {
-    SelPlan best = plan_for(L, kClMax);
+    const bool many = Hkv > sms / kClMax;        // more heads than 8-CTA clusters fit at one CTA per SM
+    SelPlan best = plan_for(L, kClMax, many);
     double best_cost = 0;
     for (int cl = kClMax; cl >= 2; cl >>= 1) {
-        const SelPlan p = plan_for(L, cl);
+        const SelPlan p = plan_for(L, cl, many);
         if (cl != kClMax && !p.in_smem) break;
-        const int per_sm = p.smem <= 113 * 1024 ? 2 : 1;
+        const int per_sm = p.smem <= 112 * 1024 + 512 ? 2 : 1;
         const int resident = sms * per_sm / cl > 0 ? sms * per_sm / cl : 1;
         const double cost = (double)((Hkv + resident - 1) / resident) * (20000.0 + 1.7 * p.chunk);
         if (cl == kClMax || cost < best_cost) { best = p; best_cost = cost; }
@@ -453,7 +457,7 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
 {
     static bool attr_done[64] = {};
     if (!attr_done[dev]) {
-        const int max_smem = (4 * kBins + kRawTile + 2 * kHalo + kKeysSmemMax) * 4;
+        const int max_smem = (2 * kBins + kRawTile + 2 * kHalo + kKeysSmemMax) * 4;
         if (cudaFuncSetAttribute(select_cluster<CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
             return JQ_ERR_CUDA;
         attr_done[dev] = true;
