@@ -295,7 +295,7 @@ jq_status jq_evict_ragged(const void *const *K, const void *const *V, const void
             GroupRec &g = h_grp[ngroups++];
             g.h0 = u0 * hpu + h0; g.nh = h0 + hpg <= heads ? hpg : heads - h0;
             g.tph = tph; g.L = Lu; g.unit = u0 + h0 / hpu; g.c20 = h0 % hpu;
-            g.sbase = h_head[g.h0].soff;
+            g.sbase = h_head[g.h0].soff; g.tph_magic = div_magic((uint32_t)tph); g.pad = 0;
             if (g.nh * tph > t.max_group_tiles) t.max_group_tiles = g.nh * tph;
         }
         u0 = u1;

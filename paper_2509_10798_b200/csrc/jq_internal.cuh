@@ -66,7 +66,11 @@ struct GroupRec {
     int tph, L;          // tiles per head, prefix length
     int unit, c20;       // the unit of head h0, and the index of head h0 within it
     long long sbase;     // offset (floats) of head h0's scores in the scores array
+    uint32_t tph_magic;  // div_magic(tph): the kernel divides tile numbers by tph with a multiplication
+    uint32_t pad;
 };
+// ceil(2^32 / d) for 2 <= d < 2^31; 2^32 - 1 for d = 1 (the kernel's fast_div corrects the estimate either way).
+static inline uint32_t div_magic(uint32_t d) { return d <= 1 ? 0xffffffffu : (uint32_t)((0x100000000ull + d - 1) / d); }
 // A KV head as the selection kernel sees it.
 struct HeadRec {
     int L, nkeep;

@@ -72,6 +72,7 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSlotCols = kTmemCols / kTSlots;
 constexpr long long kWaitCycles = 4000000000ll;  // about 2 s of SM clock per wait
 constexpr int kRing = 4;                         // grid counters per kind
+constexpr int kMergeLoads = 16;                  // partial slots a lane of the merge warp has in flight
 constexpr uint32_t kSleepLong = 256;             // ns between polls of a waiter that runs ahead (producer, stager)
 constexpr uint32_t kSleepShort = 32;             // ns between polls of a waiter on the critical path
 #ifndef JQ_POLY_OF8
@@ -113,6 +114,7 @@ struct Params {
     const GroupRec *gtab;
     const CUtensorMap *maps;
     int hpu;                 // KV heads per unit (a group may run over consecutive units of one length)
+    uint32_t grid_magic, tph_magic;   // ceil(2^32 / gridDim.x), ceil(2^32 / tph) (see fast_div)
 #ifdef JQ_DEBUG
     DebugRecord *dbg_rec;    // bounds-checked build: the violation record, and the floats in the scores array
     long long n_scores;
@@ -410,6 +412,17 @@ __device__ __forceinline__ void p1_half(uint32_t (&v)[16], int c0, int valid, fl
 
 // ------------------------------------------------------------------ schedule
 
+// x / d for x < 2^25 with magic = ceil(2^32 / d) computed on the host: one multiplication and a correction
+// instead of the compiler's division sequence (dozens of instructions and a reciprocal that would queue behind
+// the exponentials in the special-function unit; every role runs the schedule arithmetic once per segment).
+__device__ __forceinline__ uint32_t fast_div(uint32_t x, uint32_t d, uint32_t magic)
+{
+    uint32_t q = __umulhi(x, magic);
+    if (q * d > x) --q;          // for d > 1 the estimate is never low and at most one high
+    if ((q + 1) * d <= x) ++q;   // d == 1 (magic 2^32 - 1): one low
+    return q;
+}
+
 // Segment s of the 2 * ngroups segments every CTA walks: a pass over this CTA's share of one group.
 struct Seg {
     int pass, g, h0, ntiles;
@@ -428,7 +441,7 @@ __device__ __forceinline__ GroupRec group_of(int g, const Params &P)
     if (P.gtab) return P.gtab[JQ_IN(g, P.ngroups, kDbgScore, 1) ? g : 0];
     GroupRec r;
     r.h0 = g * P.hpg; r.nh = min(P.hpg, P.Hkv - r.h0);
-    r.tph = P.tph; r.L = P.L; r.unit = 0; r.c20 = r.h0;
+    r.tph = P.tph; r.L = P.L; r.unit = 0; r.c20 = r.h0; r.tph_magic = P.tph_magic;
     r.sbase = (long long)r.h0 * P.L;
     return r;
 }
@@ -445,11 +458,12 @@ __device__ __noinline__ Seg segment(int s, const Params &P)
     const GroupRec r = group_of(sg.g, P);
     sg.h0 = r.h0; sg.tph = r.tph; sg.L = r.L; sg.unit = r.unit; sg.c20 = r.c20; sg.sbase = r.sbase;
     const uint32_t T = (uint32_t)r.nh * r.tph, G = gridDim.x;
-    const uint32_t t_begin = blockIdx.x * T / G, t_end = (blockIdx.x + 1) * T / G;
+    const uint32_t t_begin = fast_div(blockIdx.x * T, G, P.grid_magic), t_end = fast_div((blockIdx.x + 1) * T, G, P.grid_magic);
     sg.ntiles = (int)(t_end - t_begin);
     const uint32_t first = (sg.pass == 1) ? t_begin : (t_end > 0 ? t_end - 1 : 0);
-    sg.kv0 = sg.h0 + (int)(first / r.tph);
-    sg.t0 = (int)(first % r.tph);
+    const uint32_t hd = fast_div(first, (uint32_t)r.tph, r.tph_magic);
+    sg.kv0 = sg.h0 + (int)hd;
+    sg.t0 = (int)(first - hd * (uint32_t)r.tph);
     return sg;
 }
 
@@ -622,8 +636,9 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                 const int h0 = gr.h0, nh = gr.nh, tph = gr.tph;
                 const uint32_t T = (uint32_t)nh * tph;
                 // This CTA's rows of the group are blockIdx.x + k G.  They are taken `rows_par` at a time, each by a
-                // sub-group of 32 / rows_par lanes that splits the row's partial slots, four loads in flight per
-                // lane; an empty partial (or one of a CTA that had no tile of the head) counts as (-inf, 0).
+                // sub-group of 32 / rows_par lanes that splits the row's partial slots, kMergeLoads loads in flight per
+                // lane (the merge is a chain of L2 round trips: the fewer, the sooner pass 2 of the group may start);
+                // an empty partial (or one of a CTA that had no tile of the head) counts as (-inf, 0).
                 const int nitems = nh * P.R;
                 const int nrows = (nitems > (int)blockIdx.x) ? (nitems - 1 - (int)blockIdx.x) / G + 1 : 0;
                 int rows_par = 1;
@@ -641,10 +656,10 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                     const float2 *src = P.part + ((size_t)kv * kSlots + kGroups * b_lo) * P.R + r;
                     float m = -INFINITY, l = 0.f;
 #pragma unroll 1
-                    for (int i0 = sub; i0 < nsl; i0 += lpr * 4) {
-                        float2 p[4];
+                    for (int i0 = sub; i0 < nsl; i0 += lpr * kMergeLoads) {
+                        float2 p[kMergeLoads];
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
+                        for (int k = 0; k < kMergeLoads; ++k) {
                             const int i = i0 + lpr * k;
                             p[k] = make_float2(-INFINITY, 0.f);
                             // (a CTA between b_lo and b_hi always has a tile of this head unless the group has fewer tiles than CTAs)
@@ -653,11 +668,11 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                         }
                         float mn = m;
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) if (p[k].y > 0.f) mn = fmaxf(mn, p[k].x);
+                        for (int k = 0; k < kMergeLoads; ++k) if (p[k].y > 0.f) mn = fmaxf(mn, p[k].x);
                         if (mn > -INFINITY) {
                             float acc = (l > 0.f) ? l * ex2(c * (m - mn)) : 0.f;
 #pragma unroll
-                            for (int k = 0; k < 4; ++k) if (p[k].y > 0.f) acc += p[k].y * ex2(c * (p[k].x - mn));
+                            for (int k = 0; k < kMergeLoads; ++k) if (p[k].y > 0.f) acc += p[k].y * ex2(c * (p[k].x - mn));
                             m = mn; l = acc;
                         }
                     }
@@ -744,6 +759,9 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             if (lane == 0) mbar_arrive(&ctl->t_empty[slot], 1);
         };
         // One look whether block uu is complete; if so its first 16 columns are requested (into va).  Warp-uniform.
+        // (With as many groups as slots a group's next block cannot be complete before the group gives its slot
+        // back, so the look is not taken at all: it sits between the hand-over and the last exponentials of a block.)
+        constexpr bool kLookAhead = kGroups < kTSlots;
         auto try_begin = [&](uint32_t uu) -> bool {
             const uint32_t slot = uu % kTSlots;
             if (!__all_sync(0xffffffffu, mbar_test(&ctl->t_full[slot], (uu / kTSlots) & 1))) return false;
@@ -807,7 +825,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                         if (c0 + 32 < kTile) JQ_TMEM_LD16(taddr + c0 + 32, va);
                         else {
                             release(slot);
-                            pre = (k + kGroups < nunits) && try_begin(uu + kGroups);
+                            if (kLookAhead) pre = (k + kGroups < nunits) && try_begin(uu + kGroups);
                         }
                         p1_half(vb, c0 + 16, valid, c, lazy, cc, st0);
                     }
@@ -858,7 +876,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
                         if (p + 1 < np) JQ_TMEM_LD16(taddr + 32 * p + 32, va);
                         else {
                             release(slot);
-                            pre = (k + kGroups < nunits) && try_begin(uu + kGroups);
+                            if (kLookAhead) pre = (k + kGroups < nunits) && try_begin(uu + kGroups);
                         }
                         exp_acc16(a01, a23, vb, cc, bias + 8 * p + 4);
                     }
@@ -1067,6 +1085,8 @@ jq_status launch_score_tc(const void *K, const void *Q, const jq_shape &s, float
         tmax = (long long)(P.hpg < s.Hkv ? P.hpg : s.Hkv) * P.tph;
     }
     const int grid = (int)(tmax < sms ? tmax : sms);
+    P.grid_magic = div_magic((uint32_t)grid);
+    P.tph_magic = tables ? 0u : div_magic((uint32_t)P.tph);
 #ifdef JQ_DEBUG
     P.dbg_rec = debug_record();
     P.n_scores = tables ? tables->total_keys : (long long)s.Hkv * s.L;
