@@ -82,6 +82,10 @@ constexpr int kPolyOf8 = JQ_POLY_OF8;            // of every 8 pairs of exponent
 // words of the workspace status block
 constexpr int kWStatus = 0, kWDone = 1, kWCnt1 = 8, kWCnt2 = 12;
 static_assert(kSlots >= kGroupsWide * 148 && kSlots >= kGroupsNarrow * 148, "one partial slot per epilogue group and CTA");
+// A group waits for its block on the slot's barrier by phase parity, which tells two consecutive fillings apart and no
+// more: a group may be at most one filling of a slot ahead of the MMA warp, which holds as long as every group has a
+// slot of its own to wait on.
+static_assert(kGroupsWide <= kTSlots && kGroupsNarrow <= kTSlots, "no more epilogue groups than accumulator slots");
 
 struct Ctl {
     uint64_t full[kMaxStages], empty[kMaxStages];
