@@ -442,7 +442,14 @@ __device__ __forceinline__ GroupRec group_of(int g, const Params &P)
 #ifdef JQ_DEBUG
     DebugRecord *dbg = P.dbg_rec;
 #endif
-    if (P.gtab) return P.gtab[JQ_IN(g, P.ngroups, kDbgScore, 1) ? g : 0];
+    if (P.gtab) {
+        // read through the read-only path: a 128-byte line holds three records, so most reads of a role hit the L1
+        const GroupRec *p = P.gtab + (JQ_IN(g, P.ngroups, kDbgScore, 1) ? g : 0);
+        GroupRec r;
+        r.h0 = __ldg(&p->h0); r.nh = __ldg(&p->nh); r.tph = __ldg(&p->tph); r.L = __ldg(&p->L);
+        r.unit = __ldg(&p->unit); r.c20 = __ldg(&p->c20); r.sbase = __ldg(&p->sbase); r.tph_magic = __ldg(&p->tph_magic);
+        return r;
+    }
     GroupRec r;
     r.h0 = g * P.hpg; r.nh = min(P.hpg, P.Hkv - r.h0);
     r.tph = P.tph; r.L = P.L; r.unit = 0; r.c20 = r.h0; r.tph_magic = P.tph_magic;
@@ -450,8 +457,19 @@ __device__ __forceinline__ GroupRec group_of(int g, const Params &P)
     return r;
 }
 
-// (Not inlined: five roles call it once per segment.)
-__device__ __noinline__ Seg segment(int s, const Params &P)
+// This CTA's share of a group of nh heads of tph tiles: a role keeps the last one it computed, since consecutive
+// groups mostly have the same shape and the divisions are then not repeated.
+struct Share {
+    int nh = -1, tph = -1;
+    int ntiles;
+    int hd1, t01;      // head (relative to the group's first) and tile within it of the share's first tile
+    int hd2, t02;      // and of its last tile, where pass 2 starts
+};
+
+// (Inlined into the four roles that call it once per segment: out of line it took 1200-1400 cycles per call, the
+// kernel parameters being read through a reference and the result returned through local memory, and while the MMA
+// warp sat in it no group got a block.)
+__device__ __forceinline__ Seg segment(int s, const Params &P, Share &sh)
 {
     Seg sg;
     const int NG = P.ngroups;
@@ -461,13 +479,19 @@ __device__ __noinline__ Seg segment(int s, const Params &P)
     else { sg.pass = 2; sg.g = s - NG; }                                   // tail: the last D groups' pass 2
     const GroupRec r = group_of(sg.g, P);
     sg.h0 = r.h0; sg.tph = r.tph; sg.L = r.L; sg.unit = r.unit; sg.c20 = r.c20; sg.sbase = r.sbase;
-    const uint32_t T = (uint32_t)r.nh * r.tph, G = gridDim.x;
-    const uint32_t t_begin = fast_div(blockIdx.x * T, G, P.grid_magic), t_end = fast_div((blockIdx.x + 1) * T, G, P.grid_magic);
-    sg.ntiles = (int)(t_end - t_begin);
-    const uint32_t first = (sg.pass == 1) ? t_begin : (t_end > 0 ? t_end - 1 : 0);
-    const uint32_t hd = fast_div(first, (uint32_t)r.tph, r.tph_magic);
-    sg.kv0 = sg.h0 + (int)hd;
-    sg.t0 = (int)(first - hd * (uint32_t)r.tph);
+    if (r.nh != sh.nh || r.tph != sh.tph) {
+        const uint32_t T = (uint32_t)r.nh * r.tph, G = gridDim.x;
+        const uint32_t t_begin = fast_div(blockIdx.x * T, G, P.grid_magic), t_end = fast_div((blockIdx.x + 1) * T, G, P.grid_magic);
+        const uint32_t last = t_end > 0 ? t_end - 1 : 0;
+        const uint32_t hd1 = fast_div(t_begin, (uint32_t)r.tph, r.tph_magic), hd2 = fast_div(last, (uint32_t)r.tph, r.tph_magic);
+        sh.nh = r.nh; sh.tph = r.tph;
+        sh.ntiles = (int)(t_end - t_begin);
+        sh.hd1 = (int)hd1; sh.t01 = (int)(t_begin - hd1 * (uint32_t)r.tph);
+        sh.hd2 = (int)hd2; sh.t02 = (int)(last - hd2 * (uint32_t)r.tph);
+    }
+    sg.ntiles = sh.ntiles;
+    sg.kv0 = sg.h0 + (sg.pass == 1 ? sh.hd1 : sh.hd2);
+    sg.t0 = sg.pass == 1 ? sh.t01 : sh.t02;
     return sg;
 }
 
@@ -533,13 +557,14 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             // ---------------------------------------------------------------- TMA producer
             if (lane == 0) {
                 uint32_t st = 0, ph = 0, qn = 0;                  // ring stage and its phase; query loads so far
+                Share share;
                 int prev_kv = -1, prev_unit = -1;
                 const CUtensorMap *head_mapK = &mapK, *head_mapQ = &mapQ;   // maps and head coordinate of the current KV head
                 int head_c2 = 0;
                 bool ok = true;
 #pragma unroll 1
                 for (int s = 0; s < nseg && ok; ++s) {
-                    const Seg sg = segment(s, P);
+                    const Seg sg = segment(s, P, share);
                     const int pass = sg.pass, ntiles = sg.ntiles, tph = sg.tph;
                     int kv = sg.kv0, tt = sg.t0;
 #pragma unroll 1
@@ -583,11 +608,12 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             // pass 2: a block's columns are the query rows it covers, rounded up to 32 (the rows past R are zero)
             const uint32_t idesc2a = instr_desc(kTile, min(128, Rpad)), idesc2b = instr_desc(kTile, max(32, Rpad - 128));
             uint32_t st = 0, ph = 0, qn = 0, u = 0;           // ring stage and phase, query loads, accumulator blocks so far
+            Share share;
             int prev_kv = -1;
             bool ok = true;
 #pragma unroll 1
             for (int s = 0; s < nseg && ok; ++s) {
-                const Seg sg = segment(s, P);
+                const Seg sg = segment(s, P, share);
                 const int pass = sg.pass, ntiles = sg.ntiles, tph = sg.tph;
                 int kv = sg.kv0, tt = sg.t0;
 #pragma unroll 1
@@ -702,9 +728,10 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
             // then feeds -M_r of each KV head of the segment into the double-buffered shared array.
             uint32_t hs = 0;
             int ok = 1;
+            Share share;
 #pragma unroll 1
             for (int s = 0; s < nseg && ok; ++s) {
-                const Seg sg = segment(s, P);
+                const Seg sg = segment(s, P, share);
                 if (sg.pass != 2 || sg.ntiles == 0) continue;
                 const int tph = sg.tph;
                 if (nblk == 2) {
@@ -754,6 +781,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
         int hs = 0;                                             // pass-2 heads of the CTA before this segment
         bool ok = true;
         uint32_t va[16], vb[16];                                // the two alternating 16-column reads
+        Share share;
 
         // Slot and parity of the CTA's accumulator block number uu; the block after this group's block uu is uu + kGroups.
         // Giving a slot back: the warp's reads of it are complete (tcgen05.wait::ld is warp-wide), one lane tells the MMA warp.
@@ -783,7 +811,7 @@ score_fused(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CU
 
 #pragma unroll 1
         for (int s = 0; s < nseg && ok; ++s) {
-            const Seg sg = segment(s, P);
+            const Seg sg = segment(s, P, share);
             const int ntiles = sg.ntiles, nunits = ntiles << bs, tph = sg.tph, L = sg.L;
             int kv = sg.kv0, tt = sg.t0, at = 0;                // tile cursor: head, tile in head, index in the segment
             int k = (grp + kGroups - (int)(u % kGroups)) % kGroups;   // this group's first block of the segment
