@@ -60,6 +60,13 @@ __device__ __forceinline__ uint32_t order_key(float x)
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
+__device__ __forceinline__ float max3f(float a, float b, float c)
+{
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
+
 // Block-wide exclusive scan of one int per thread (1024 threads).
 __device__ __forceinline__ int block_excl_scan(int v, int *warp_sums)
 {
@@ -410,6 +417,390 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
     if (Kin) copy_kept_rows<CL>(cluster, out, kv_in, krow, L, nkeep, Kin, Vin, Kout, Vout, src_rows, ext JQ_DBG_ARG_DEV);
 }
 
+// ------------------------------------------------------------------ many heads: one CTA per head, no cluster
+//
+// A call over many heads (the layers of a cache, a ragged batch) has more heads than clusters fit on the GPU, and the
+// cluster kernel's time per head is mostly the latency of its barrier-separated phases.  Here a head is one CTA that
+// keeps a histogram, a candidate list and a small staging buffer per warp in shared memory, so that several heads are
+// resident per SM, and that walks the head's scores three times, pooling on the fly.  Every warp owns a contiguous
+// share of the head and takes it 512 positions at a time: four 16-byte reads per lane in flight, staged in shared
+// memory with one quad of halo on either side, from where a lane pools four neighbouring positions.
+//   pass 1  pooled keys -> histogram of the top 11 bits (and the pooled values, when the caller wants them);
+//   pass 2  the keys that share the winning digit -> candidate list (key and position), and per warp the number of
+//           keys with a larger digit; rounds 2 and 3 run on the list, and the list then also gives every warp its
+//           number of kept keys.  (When the list would not fit, rounds 2 and 3 and the counts are passes of their own.)
+//   pass 3  ordered compaction of the kept positions, then the copy of the kept rows.
+// Same integer arithmetic as the cluster kernel: the same threshold key and the same ties, hence the same indices.
+constexpr int kStrCand = 2048;      // candidates finished in shared memory
+constexpr int kStrMaxWarps = 32;
+constexpr int kStepQuads = 128;     // quads a warp takes per step
+constexpr int kStageQuads = kStepQuads + 2;
+#ifndef JQ_STREAM_MIN_HEADS
+#define JQ_STREAM_MIN_HEADS 128
+#endif
+constexpr int kStreamMinHeads = JQ_STREAM_MIN_HEADS;   // calls with at least this many heads take this kernel
+
+struct StrCtl {
+    int scan[kStrMaxWarps + 1];
+    int digit, krem, count;         // find_digit_cta: the bin of the krem-th key, the rank within it, its population
+    int cand_count;
+    int warp_gt[kStrMaxWarps], warp_eq[kStrMaxWarps];
+};
+
+// Quad q (positions 4q .. 4q+3) of a head of L scores at s; positions outside [0, L) read as -inf.
+// vec: s is 16-byte aligned.
+__device__ __forceinline__ float4 load_quad(const float *__restrict__ s, int L, int q, bool vec, long long soff,
+                                            const SelExtents &ext JQ_DBG_PARAM)
+{
+    (void)soff; (void)ext;
+    const float ninf = -INFINITY;
+    if (q < 0 || 4 * q >= L) return make_float4(ninf, ninf, ninf, ninf);
+    if (vec && 4 * q + 4 <= L && JQ_IN(soff + 4 * q + 3, ext.scores, kDbgSelect, 22)) return *(const float4 *)(s + 4 * q);
+    float v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = (4 * q + i < L && JQ_IN(soff + 4 * q + i, ext.scores, kDbgSelect, 23)) ? s[4 * q + i] : ninf;
+    return make_float4(v[0], v[1], v[2], v[3]);
+}
+
+// The warp stages quads [base - 1, base + 129) of the head in its buffer.
+__device__ __forceinline__ void stage_quads(float4 *buf, const float *__restrict__ s, int L, int base, bool vec, long long soff,
+                                            const SelExtents &ext JQ_DBG_PARAM)
+{
+    const int lane = threadIdx.x & 31;
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = load_quad(s, L, base + 32 * u + lane, vec, soff, ext JQ_DBG_ARG_DEV);
+    float4 h = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (lane < 2) h = load_quad(s, L, lane == 0 ? base - 1 : base + kStepQuads, vec, soff, ext JQ_DBG_ARG_DEV);
+    __syncwarp();                                            // the previous step's reads of the buffer are done
+#pragma unroll
+    for (int u = 0; u < 4; ++u) buf[1 + 32 * u + lane] = v[u];
+    if (lane < 2) buf[lane == 0 ? 0 : kStageQuads - 1] = h;
+    __syncwarp();
+}
+
+// Pooled order keys (and values) of the four positions of quad `at` (0 .. 127) of the staged step.
+__device__ __forceinline__ void pooled_quad(const float4 *buf, int at, int radius, uint32_t (&key)[4], float (&best)[4])
+{
+    const float4 a = buf[at], b = buf[at + 1], c = buf[at + 2];
+    const float x[12] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w, c.x, c.y, c.z, c.w};
+    if (radius == 3) {
+        // window of 7: the four windows share x4..x7; the rest are running maxima of the three neighbours on either side
+        const float core = fmaxf(max3f(x[4], x[5], x[6]), x[7]);
+        const float l2 = fmaxf(x[2], x[3]), l1 = fmaxf(x[1], l2);
+        const float r9 = fmaxf(x[8], x[9]), r10 = fmaxf(r9, x[10]);
+        best[0] = fmaxf(core, l1);
+        best[1] = max3f(core, l2, x[8]);
+        best[2] = max3f(core, x[3], r9);
+        best[3] = fmaxf(core, r10);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float m = x[4 + i];
+#pragma unroll
+            for (int u = 1; u <= 4; ++u) if (u <= radius) m = fmaxf(m, fmaxf(x[4 + i - u], x[4 + i + u]));
+            best[i] = m;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) key[i] = order_key(best[i]);
+}
+
+// Block-wide exclusive scan of one int per thread, any number of whole warps.
+__device__ __forceinline__ int cta_excl_scan(int v, int *warp_sums)
+{
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (lane == 31) warp_sums[wid] = inc;
+    __syncthreads();
+    if (wid == 0) {
+        const int ws = lane < nw ? warp_sums[lane] : 0;
+        int winc = ws;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int n = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += n;
+        }
+        if (lane < nw) warp_sums[lane] = winc - ws;
+    }
+    __syncthreads();
+    const int excl = warp_sums[wid] + inc - v;
+    __syncthreads();
+    return excl;
+}
+
+// All threads of a CTA of 256, 512 or 1024: the bin of h[kBins] that holds the krem-th key counted from the top.
+__device__ __forceinline__ void find_digit_cta(const uint32_t *h, int krem, StrCtl &ctl)
+{
+    const int per = kBins / (int)blockDim.x;                  // 8, 4 or 2 bins per thread, descending
+    const int hi = kBins - 1 - per * (int)threadIdx.x;
+    int tot = 0;
+    for (int i = 0; i < per; ++i) tot += (int)h[hi - i];
+    int above = cta_excl_scan(tot, ctl.scan);
+    for (int i = 0; i < per; ++i) {
+        const int c = (int)h[hi - i];
+        if (above < krem && krem <= above + c) { ctl.digit = hi - i; ctl.krem = krem - above; ctl.count = c; }
+        above += c;
+    }
+    __syncthreads();
+}
+
+// Adds the digits of a thread's (up to) four neighbouring keys to the histogram: runs of equal digits as one count (the
+// max-pool leaves plateaus); digit 0xffffffff marks a key that does not take part.
+__device__ __forceinline__ void hist_add_runs(uint32_t *hist, const uint32_t (&digit)[4], int nval JQ_DBG_PARAM)
+{
+    uint32_t cur = 0xffffffffu, cnt = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (i < nval) {
+            if (digit[i] != cur) {
+                if (cnt && cur != 0xffffffffu && JQ_IN(cur, kBins, kDbgSelect, 24)) atomicAdd(&hist[cur], cnt);
+                cur = digit[i]; cnt = 0;
+            }
+            ++cnt;
+        }
+    }
+    if (cnt && cur != 0xffffffffu && JQ_IN(cur, kBins, kDbgSelect, 24)) atomicAdd(&hist[cur], cnt);
+}
+
+// grid (Hkv), block kThreads = 256 (five CTAs to an SM), 512 (two) or 1024 (one); dynamic shared memory: a staging
+// buffer of kStageQuads float4 per warp.  Arguments as for select_cluster.
+__host__ __device__ constexpr int stream_ctas_per_sm(int threads) { return threads == 256 ? 5 : threads == 512 ? 2 : 1; }
+template <int kThreads>
+__global__ void __launch_bounds__(kThreads, stream_ctas_per_sm(kThreads))
+select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, int32_t *__restrict__ idx,
+              float *__restrict__ pooled, const uint4 *__restrict__ Kin, const uint4 *__restrict__ Vin,
+              uint4 *__restrict__ Kout, uint4 *__restrict__ Vout, const HeadRec *__restrict__ htab,
+              const uint4 *const *__restrict__ Ktab, const uint4 *const *__restrict__ Vtab, int src_rows, int out_rows,
+              const SelExtents ext JQ_DBG_PARAM)
+{
+    extern __shared__ __align__(16) uint8_t sm[];
+    __shared__ uint32_t hist[kBins];
+    __shared__ uint32_t cand_key[kStrCand];
+    __shared__ int cand_pos[kStrCand];
+    __shared__ StrCtl ctl;
+    constexpr int T = kThreads, nw = T / 32;
+    const int kv = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    float4 *buf = (float4 *)sm + wid * kStageQuads;
+    int kv_in = kv;
+    long long soff = (long long)kv * L, orow = (long long)kv * nkeep, krow = (long long)kv * out_rows;
+    cudaGridDependencySynchronize();   // everything above ran while the previous kernel of the stream was finishing
+    if (htab) {
+        const HeadRec r = htab[kv];
+        L = r.L; nkeep = r.nkeep; kv_in = r.kv_in; soff = r.soff; orow = r.ooff; krow = r.ooff; src_rows = L;
+        if (Ktab) { Kin = Ktab[r.unit]; Vin = Vtab[r.unit]; }
+    }
+    if (nkeep > L) nkeep = L;
+    const float *s = scores + soff;
+    int32_t *out = idx + orow;
+    if (pooled) pooled += soff;
+    const bool vec = (((size_t)s) & 15) == 0;
+    const int nq = (L + 3) / 4;
+    // warp w owns the contiguous quads [qa, qb); every warp makes the same number of steps
+    const int segq = (nq + nw - 1) / nw;
+    const int qa = min(wid * segq, nq), qb = min(qa + segq, nq);
+
+    // ---- pass 1: histogram of the top 11 bits of the pooled keys
+    for (int i = tid; i < kBins; i += T) hist[i] = 0;
+    if (tid == 0) ctl.cand_count = 0;
+    __syncthreads();
+    for (int base = qa; base < qb; base += kStepQuads) {
+        stage_quads(buf, s, L, base, vec, soff, ext JQ_DBG_ARG_DEV);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int q = base + 32 * u + lane;
+            const int nval = q < qb ? min(4, L - 4 * q) : 0;
+            uint32_t key[4];
+            float best[4];
+            pooled_quad(buf, 32 * u + lane, radius, key, best);
+            if (pooled && nval && JQ_IN(soff + 4 * q + nval - 1, ext.scores, kDbgSelect, 25))
+                for (int i = 0; i < nval; ++i) pooled[4 * q + i] = best[i];
+            // one addition per warp when all its positions share the digit (the usual case: 128 neighbouring
+            // positions of similar size), else runs of equal digits per thread
+            const uint32_t d0 = key[0] >> 21;
+            bool same = true;
+            for (int i = 1; i < 4; ++i) if (i < nval && (key[i] >> 21) != d0) same = false;
+            const uint32_t lead = __shfl_sync(0xffffffffu, d0, 0);
+            if (__all_sync(0xffffffffu, nval == 0 || (same && d0 == lead))) {
+                const int tot = __reduce_add_sync(0xffffffffu, nval);
+                if (lane == 0 && tot && JQ_IN(lead, kBins, kDbgSelect, 24)) atomicAdd(&hist[lead], (uint32_t)tot);
+            } else {
+                const uint32_t dg[4] = {key[0] >> 21, key[1] >> 21, key[2] >> 21, key[3] >> 21};
+                hist_add_runs(hist, dg, nval JQ_DBG_ARG_DEV);
+            }
+        }
+    }
+    __syncthreads();
+    if (nkeep >= L) {                                          // everything is kept
+        for (int e = tid; e < L; e += T) if (JQ_IN(orow + e, ext.out_rows, kDbgSelect, 26)) out[e] = e;
+    } else {
+        // ---- the threshold key tau and how many keys equal to it are kept
+        find_digit_cta(hist, nkeep, ctl);
+        uint32_t pre = (uint32_t)ctl.digit;
+        int krem = ctl.krem;
+        const bool listed = ctl.count <= kStrCand;
+        if (lane == 0) { ctl.warp_gt[wid] = 0; ctl.warp_eq[wid] = 0; }
+        __syncthreads();
+        if (listed) {
+            // pass 2: the keys with the winning first digit, with their positions; the warp's keys above that digit
+            int hi_cnt = 0;
+            for (int base = qa; base < qb; base += kStepQuads) {
+                stage_quads(buf, s, L, base, vec, soff, ext JQ_DBG_ARG_DEV);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int q = base + 32 * u + lane;
+                    const int nval = q < qb ? min(4, L - 4 * q) : 0;
+                    uint32_t key[4];
+                    float best[4];
+                    pooled_quad(buf, 32 * u + lane, radius, key, best);
+                    int nhit = 0;
+                    for (int i = 0; i < 4; ++i) if (i < nval) { nhit += (key[i] >> 21) == pre; hi_cnt += (key[i] >> 21) > pre; }
+                    if (nhit) {
+                        int at = atomicAdd(&ctl.cand_count, nhit);
+                        for (int i = 0; i < 4; ++i)
+                            if (i < nval && (key[i] >> 21) == pre) {
+                                if (JQ_IN(at, kStrCand, kDbgSelect, 27)) { cand_key[at] = key[i]; cand_pos[at] = 4 * q + i; }
+                                ++at;
+                            }
+                    }
+                }
+            }
+            hi_cnt = __reduce_add_sync(0xffffffffu, hi_cnt);
+            if (lane == 0) ctl.warp_gt[wid] = hi_cnt;
+            __syncthreads();
+        }
+        const int nc = listed ? ctl.cand_count : 0;
+        for (int r2 = 1; r2 < 3; ++r2) {
+            const int sh = (r2 == 1) ? 10 : 0, wd = (r2 == 2) ? 10 : 11;
+            const uint32_t mask = (1u << wd) - 1u;
+            for (int i = tid; i < kBins; i += T) hist[i] = 0;
+            __syncthreads();
+            if (listed) {
+                for (int e = tid; e < nc; e += T) {
+                    const uint32_t k = cand_key[e];
+                    if ((k >> (sh + wd)) == pre && JQ_IN((k >> sh) & mask, kBins, kDbgSelect, 24)) atomicAdd(&hist[(k >> sh) & mask], 1u);
+                }
+            } else {
+                for (int base = qa; base < qb; base += kStepQuads) {
+                    stage_quads(buf, s, L, base, vec, soff, ext JQ_DBG_ARG_DEV);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int q = base + 32 * u + lane;
+                        const int nval = q < qb ? min(4, L - 4 * q) : 0;
+                        uint32_t key[4], dg[4];
+                        float best[4];
+                        pooled_quad(buf, 32 * u + lane, radius, key, best);
+                        for (int i = 0; i < 4; ++i) dg[i] = (key[i] >> (sh + wd)) == pre ? ((key[i] >> sh) & mask) : 0xffffffffu;
+                        hist_add_runs(hist, dg, nval JQ_DBG_ARG_DEV);
+                    }
+                }
+            }
+            __syncthreads();
+            find_digit_cta(hist, krem, ctl);
+            pre = (pre << wd) | (uint32_t)ctl.digit;
+            krem = ctl.krem;
+            __syncthreads();
+        }
+        const uint32_t tau = pre;
+        const int need_eq = krem;       // how many of the keys == tau are kept (lowest positions first)
+
+        // ---- kept keys per warp: from the list, or by a pass of its own
+        if (listed) {
+            for (int e = tid; e < nc; e += T) {
+                const uint32_t k = cand_key[e];
+                const int w = min((cand_pos[e] >> 2) / segq, nw - 1);
+                if (k > tau) atomicAdd(&ctl.warp_gt[w], 1);
+                else if (k == tau) atomicAdd(&ctl.warp_eq[w], 1);
+            }
+        } else {
+            int cgt = 0, ceq = 0;
+            for (int base = qa; base < qb; base += kStepQuads) {
+                stage_quads(buf, s, L, base, vec, soff, ext JQ_DBG_ARG_DEV);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int q = base + 32 * u + lane;
+                    const int nval = q < qb ? min(4, L - 4 * q) : 0;
+                    uint32_t key[4];
+                    float best[4];
+                    pooled_quad(buf, 32 * u + lane, radius, key, best);
+                    for (int i = 0; i < 4; ++i) if (i < nval) { cgt += key[i] > tau; ceq += key[i] == tau; }
+                }
+            }
+            cgt = __reduce_add_sync(0xffffffffu, cgt);
+            ceq = __reduce_add_sync(0xffffffffu, ceq);
+            if (lane == 0) { ctl.warp_gt[wid] = cgt; ctl.warp_eq[wid] = ceq; }
+        }
+        __syncthreads();
+        int gt_before = 0, eq_before = 0;
+        for (int w = 0; w < wid; ++w) { gt_before += ctl.warp_gt[w]; eq_before += ctl.warp_eq[w]; }
+
+        // ---- pass 3: ordered compaction (position order = warp, step, quad, position within the quad)
+        for (int base = qa; base < qb; base += kStepQuads) {
+            stage_quads(buf, s, L, base, vec, soff, ext JQ_DBG_ARG_DEV);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int q = base + 32 * u + lane;
+                const int nval = q < qb ? min(4, L - 4 * q) : 0;
+                uint32_t key[4];
+                float best[4];
+                pooled_quad(buf, 32 * u + lane, radius, key, best);
+                int g = 0, e = 0;
+                for (int i = 0; i < 4; ++i) if (i < nval) { g += key[i] > tau; e += key[i] == tau; }
+                const int mine = g | (e << 16);
+                if (!__any_sync(0xffffffffu, mine != 0)) continue;   // nothing of these 128 positions is at or above tau
+                int inc = mine;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int n = __shfl_up_sync(0xffffffffu, inc, o);
+                    if (lane >= o) inc += n;
+                }
+                const int total = __shfl_sync(0xffffffffu, inc, 31);
+                int g_here = gt_before + ((inc - mine) & 0xffff), e_here = eq_before + ((inc - mine) >> 16);
+                for (int i = 0; i < 4; ++i) {
+                    if (i >= nval) continue;
+                    if (key[i] > tau) {
+                        if (JQ_IN(g_here + min(e_here, need_eq), nkeep, kDbgSelect, 28)) out[g_here + min(e_here, need_eq)] = 4 * q + i;
+                        ++g_here;
+                    } else if (key[i] == tau) {
+                        if (e_here < need_eq && JQ_IN(g_here + e_here, nkeep, kDbgSelect, 29)) out[g_here + e_here] = 4 * q + i;
+                        ++e_here;
+                    }
+                }
+                gt_before += total & 0xffff;
+                eq_before += total >> 16;
+            }
+        }
+    }
+    if (!Kin) return;
+
+    // ---- the kept rows (256 bytes each: 16 lanes x 16 bytes), four rows in flight per 16 lanes
+    __syncthreads();
+    const int lane16 = tid & 15, grp = tid >> 4, ngrp = T >> 4;
+    for (int t0 = 4 * grp; t0 < nkeep; t0 += 4 * ngrp) {
+        int j[4];
+        uint4 a[4], b[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) j[r] = t0 + r < nkeep ? min(max(__ldcg(out + t0 + r), 0), L - 1) : 0;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const size_t src = ((size_t)kv_in * src_rows + j[r]) * 16 + lane16;
+            const bool in = t0 + r < nkeep && JQ_IN((long long)kv_in * src_rows + j[r], ext.src_heads * src_rows, kDbgSelect, 30);
+            a[r] = in ? Kin[src] : make_uint4(0u, 0u, 0u, 0u);
+            b[r] = in ? Vin[src] : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const size_t dst = (size_t)(krow + t0 + r) * 16 + lane16;
+            if (t0 + r < nkeep && JQ_IN(krow + t0 + r, ext.out_rows, kDbgSelect, 31)) { Kout[dst] = a[r]; Vout[dst] = b[r]; }
+        }
+    }
+}
+
 // Shared memory of a CTA whose cluster has `cl` CTAs, the share of the head it holds, and whether its keys stay on chip.
 struct SelPlan { int cl, chunk, in_smem, raw_tile; size_t smem; };
 
@@ -489,6 +880,51 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
     return check_launch();
 }
 
+// The many-head kernel: threads per head so that the scores of the heads in flight (a head is read four times) stay in
+// the L2 where that can be had.
+jq_status launch_select_stream(const float *scores, const jq_shape &s, int nkeep, int Lmax, int32_t *idx, float *pooled,
+                               cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout, int sms, int dev,
+                               const UnitTables *tables, int src_rows, int out_rows)
+{
+    int threads = 256;
+    for (; threads < 1024; threads *= 2) {
+        const long long resident = (long long)sms * stream_ctas_per_sm(threads), inflight = s.Hkv < resident ? s.Hkv : resident;
+        if (inflight * Lmax * 4 <= (96ll << 20)) break;
+    }
+    const auto kernel = threads == 256 ? select_stream<256> : threads == 512 ? select_stream<512> : select_stream<1024>;
+    const size_t dyn = (size_t)(threads / 32) * kStageQuads * sizeof(float4);
+    static bool attr_done[64][3] = {};
+    const int which = threads == 256 ? 0 : threads == 512 ? 1 : 2;
+    if (dev < 0 || dev >= 64) return JQ_ERR_CUDA;
+    if (!attr_done[dev][which]) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess) return JQ_ERR_CUDA;
+        attr_done[dev][which] = true;
+    }
+    SelExtents ext;
+    ext.scores = tables ? tables->total_keys : (long long)s.Hkv * s.L;
+    ext.out_rows = tables ? tables->total_rows : (long long)s.Hkv * out_rows;
+    ext.src_heads = tables ? tables->hpu : s.Hkv;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)s.Hkv);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = dyn;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // as for the cluster kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, scores, s.L, nkeep, (s.pool - 1) / 2, idx, pooled, (const uint4 *)K,
+                           (const uint4 *)V, (uint4 *)Kout, (uint4 *)Vout, tables ? tables->heads : nullptr,
+                           (const uint4 *const *)(tables && Kout ? tables->K : nullptr),
+                           (const uint4 *const *)(tables && Kout ? tables->V : nullptr), src_rows, out_rows, ext JQ_DBG_ARG) != cudaSuccess) {
+        cudaGetLastError();
+        return JQ_ERR_CUDA;
+    }
+    count_launch(1);
+    return check_launch();
+}
+
 }  // namespace
 
 jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, float *pooled,
@@ -503,6 +939,10 @@ jq_status launch_select(const float *scores, const jq_shape &s, int32_t *idx, fl
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return JQ_ERR_CUDA;
     if (!sms[dev] && cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return JQ_ERR_CUDA;
+    // many heads and a window the quad pooling covers: one CTA per head
+    if (s.Hkv >= kStreamMinHeads && (s.pool - 1) / 2 <= 4)
+        return launch_select_stream(scores, s, nkeep, Lmax, idx, pooled, st, K, V, Kout, Vout, sms[dev], dev, tables, src_rows,
+                                    out_head_rows > nkeep ? out_head_rows : nkeep);
     const SelPlan p = choose_plan(s.Hkv, Lmax, sms[dev]);
     switch (p.cl) {
     case 2: return launch_select_cl<2>(p, scores, s, nkeep, idx, pooled, w, st, K, V, Kout, Vout, dev, tables, src_rows, out_head_rows > nkeep ? out_head_rows : nkeep);
