@@ -1,5 +1,7 @@
-// Max-pool + exact top-k selection per KV head, one thread-block cluster per head: 8 CTAs when the call
-// has few heads, 4 or 2 when it has more heads than clusters fit on the GPU at a time (see choose_plan).
+// Max-pool + exact top-k selection per KV head.  Two kernels share the arithmetic: select_cluster, one
+// thread-block cluster per head (8 CTAs when the call has few heads, 4 or 2 when it has more heads than
+// clusters fit on the GPU at a time, see choose_plan), and, for calls over 128 heads or more, select_stream
+// further down, one CTA per head.  The cluster kernel:
 //
 //   1. pool: pooled[j] = max of the centred window (edges clipped), turned into an order-preserving
 //      32-bit integer key (float order == unsigned order).  Each CTA owns a contiguous share of
@@ -534,10 +536,10 @@ __device__ __forceinline__ int cta_excl_scan(int v, int *warp_sums)
     return excl;
 }
 
-// All threads of a CTA of 256, 512 or 1024: the bin of h[kBins] that holds the krem-th key counted from the top.
+// All threads of a CTA of 512 or 1024: the bin of h[kBins] that holds the krem-th key counted from the top.
 __device__ __forceinline__ void find_digit_cta(const uint32_t *h, int krem, StrCtl &ctl)
 {
-    const int per = kBins / (int)blockDim.x;                  // 8, 4 or 2 bins per thread, descending
+    const int per = kBins / (int)blockDim.x;                  // 4 or 2 bins per thread, descending
     const int hi = kBins - 1 - per * (int)threadIdx.x;
     int tot = 0;
     for (int i = 0; i < per; ++i) tot += (int)h[hi - i];
@@ -568,9 +570,9 @@ __device__ __forceinline__ void hist_add_runs(uint32_t *hist, const uint32_t (&d
     if (cnt && cur != 0xffffffffu && JQ_IN(cur, kBins, kDbgSelect, 24)) atomicAdd(&hist[cur], cnt);
 }
 
-// grid (Hkv), block kThreads = 256 (five CTAs to an SM), 512 (two) or 1024 (one); dynamic shared memory: a staging
-// buffer of kStageQuads float4 per warp.  Arguments as for select_cluster.
-__host__ __device__ constexpr int stream_ctas_per_sm(int threads) { return threads == 256 ? 5 : threads == 512 ? 2 : 1; }
+// grid (Hkv), block kThreads = 512 (two CTAs to an SM) or 1024 (one); dynamic shared memory: a staging buffer of
+// kStageQuads float4 per warp.  Arguments as for select_cluster.
+__host__ __device__ constexpr int stream_ctas_per_sm(int threads) { return threads == 512 ? 2 : 1; }
 template <int kThreads>
 __global__ void __launch_bounds__(kThreads, stream_ctas_per_sm(kThreads))
 select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, int32_t *__restrict__ idx,
@@ -880,21 +882,18 @@ jq_status launch_select_cl(const SelPlan &p, const float *scores, const jq_shape
     return check_launch();
 }
 
-// The many-head kernel: threads per head so that the scores of the heads in flight (a head is read four times) stay in
-// the L2 where that can be had.
+// The many-head kernel: 512 threads per head (measured best from 8K to 64K keys per head, 256 to 1024 heads), 1024
+// when the scores of the heads that 512 would hold in flight (a head is read three times) are far more than the L2.
 jq_status launch_select_stream(const float *scores, const jq_shape &s, int nkeep, int Lmax, int32_t *idx, float *pooled,
                                cudaStream_t st, const void *K, const void *V, void *Kout, void *Vout, int sms, int dev,
                                const UnitTables *tables, int src_rows, int out_rows)
 {
-    int threads = 256;
-    for (; threads < 1024; threads *= 2) {
-        const long long resident = (long long)sms * stream_ctas_per_sm(threads), inflight = s.Hkv < resident ? s.Hkv : resident;
-        if (inflight * Lmax * 4 <= (96ll << 20)) break;
-    }
-    const auto kernel = threads == 256 ? select_stream<256> : threads == 512 ? select_stream<512> : select_stream<1024>;
+    const long long resident = (long long)sms * stream_ctas_per_sm(512), inflight = s.Hkv < resident ? s.Hkv : resident;
+    const int threads = inflight * Lmax * 4 <= (96ll << 20) ? 512 : 1024;
+    const auto kernel = threads == 512 ? select_stream<512> : select_stream<1024>;
     const size_t dyn = (size_t)(threads / 32) * kStageQuads * sizeof(float4);
-    static bool attr_done[64][3] = {};
-    const int which = threads == 256 ? 0 : threads == 512 ? 1 : 2;
+    static bool attr_done[64][2] = {};
+    const int which = threads == 512 ? 0 : 1;
     if (dev < 0 || dev >= 64) return JQ_ERR_CUDA;
     if (!attr_done[dev][which]) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess) return JQ_ERR_CUDA;

@@ -63,6 +63,15 @@ cases = [(1, 1, 1, 1, 1, 1), (1, 1, 1, 5, 3, 3), (2, 4, 16, 129, 7, 7), (2, 4, 1
 for c in cases:
     whole_pass(wl_of(*c))
 
+# selection over many heads (one CTA of 512 or 1024 threads per head): odd lengths, ties, budgets at and above L
+for Hkv, L, B, p in [(129, 1023, 77, 9), (130, 4001, 4001, 7), (300, 70000, 500, 7), (128, 200001, 1000, 5)]:
+    s = jq.shape(Hkv, Hkv, L, 1, B, p)
+    ws = jq.new_workspace(s)
+    for sc in (torch.rand((Hkv, L), device="cuda"), torch.randint(0, 5, (Hkv, L), device="cuda").float()):
+        idx = torch.zeros((Hkv, min(B, L)), dtype=torch.int32, device="cuda")
+        jq.select_topk(sc, s, idx, ws, pooled=torch.empty_like(sc))
+        assert jq.last_device_status(ws) == jq.JQ_OK
+
 # several units in one call: lengths and budgets of their own, groups that run over units of one length
 base = wl_of(2, 4, 32, 5000, 400)
 Ls, Bs = [3000, 130, 130, 5000, 1, 2049, 2049, 2049], [400, 1000, 7, 64, 3, 2049, 100, 5]

@@ -115,9 +115,12 @@ def test_select_bit_exact(Hkv, L, B, p, kind):
     assert np.array_equal(got_idx, want_idx)
 
 
-# With many heads the selection kernel runs smaller clusters (4 or 2 CTAs per head instead of 8): same results.
+# With many heads the selection runs smaller clusters (4 or 2 CTAs per head instead of 8) and, from 128 heads on, the
+# kernel that gives every head one CTA of 512 or 1024 threads (1024 in the last case): same results.
+# The tied inputs put more keys into the winning histogram bin than its candidate list holds.
 @pytest.mark.parametrize("Hkv,L,B,p", [(64, 4096, 512, 7), (160, 5000, 700, 7), (300, 1000, 100, 5), (148, 40000, 2048, 7),
-                                       (200, 1, 1, 7), (200, 5, 9, 7), (100, 33, 10, 3), (256, 70001, 300, 1)])
+                                       (200, 1, 1, 7), (200, 5, 9, 7), (100, 33, 10, 3), (256, 70001, 300, 1),
+                                       (130, 4001, 4001, 9), (129, 1023, 77, 9), (400, 70000, 500, 7), (128, 200001, 1000, 9)])
 @pytest.mark.parametrize("kind", ["random", "ties"])
 def test_select_many_heads_bit_exact(Hkv, L, B, p, kind):
     rng = np.random.default_rng(Hkv * 7 + L)
@@ -131,10 +134,11 @@ def test_select_many_heads_bit_exact(Hkv, L, B, p, kind):
     assert np.array_equal(got_idx, want_idx)
 
 
-def test_select_all_equal_keeps_lowest_indices():
-    s32 = np.full((2, 5000), 0.25, np.float32)
-    idx, _ = gpu_select(s32, jq.shape(2, 2, 5000, 1, 777, 7))
-    assert np.array_equal(idx, np.tile(np.arange(777, dtype=np.int32), (2, 1)))
+@pytest.mark.parametrize("Hkv", [2, 150])
+def test_select_all_equal_keeps_lowest_indices(Hkv):
+    s32 = np.full((Hkv, 5000), 0.25, np.float32)
+    idx, _ = gpu_select(s32, jq.shape(Hkv, Hkv, 5000, 1, 777, 7))
+    assert np.array_equal(idx, np.tile(np.arange(777, dtype=np.int32), (Hkv, 1)))
 
 
 # ------------------------------------------------------------------ compaction (step 6), bit-exact
