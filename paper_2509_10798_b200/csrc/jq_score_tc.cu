@@ -55,13 +55,7 @@ namespace {
 
 constexpr int kTile = 128;                       // keys per tile
 constexpr int kMaxStages = 5;                    // K ring depth (5 when R <= 128, 3 above)
-#ifndef JQ_GROUPS_NARROW
-#define JQ_GROUPS_NARROW 3
-#endif
-#ifndef JQ_GROUPS_WIDE
-#define JQ_GROUPS_WIDE 4
-#endif
-constexpr int kGroupsNarrow = JQ_GROUPS_NARROW, kGroupsWide = JQ_GROUPS_WIDE;   // epilogue groups for R <= 128 / R > 128
+constexpr int kGroupsNarrow = 3, kGroupsWide = 4;   // epilogue groups for R <= 128 / R > 128
 constexpr int kTSlots = 4;                       // accumulator slots in tensor memory
 constexpr int kSpecialWarps = 4;                 // producer, MMA, merge, stage: one warpgroup
 __host__ __device__ constexpr int threads_for(int groups) { return (kSpecialWarps + 4 * groups) * 32; }
@@ -75,10 +69,7 @@ constexpr int kRing = 4;                         // grid counters per kind
 constexpr int kMergeLoads = 16;                  // partial slots a lane of the merge warp has in flight
 constexpr uint32_t kSleepLong = 256;             // ns between polls of a waiter that runs ahead (producer, stager)
 constexpr uint32_t kSleepShort = 32;             // ns between polls of a waiter on the critical path
-#ifndef JQ_POLY_OF8
-#define JQ_POLY_OF8 2
-#endif
-constexpr int kPolyOf8 = JQ_POLY_OF8;            // of every 8 pairs of exponentials, this many go to the FMA pipe
+constexpr int kPolyOf8 = 2;                      // of every 8 pairs of exponentials, this many go to the FMA pipe
 // words of the workspace status block
 constexpr int kWStatus = 0, kWDone = 1, kWCnt1 = 8, kWCnt2 = 12;
 static_assert(kSlots >= kGroupsWide * 148 && kSlots >= kGroupsNarrow * 148, "one partial slot per epilogue group and CTA");

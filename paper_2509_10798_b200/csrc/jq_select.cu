@@ -437,10 +437,7 @@ constexpr int kStrCand = 2048;      // candidates finished in shared memory
 constexpr int kStrMaxWarps = 32;
 constexpr int kStepQuads = 128;     // quads a warp takes per step
 constexpr int kStageQuads = kStepQuads + 2;
-#ifndef JQ_STREAM_MIN_HEADS
-#define JQ_STREAM_MIN_HEADS 128
-#endif
-constexpr int kStreamMinHeads = JQ_STREAM_MIN_HEADS;   // calls with at least this many heads take this kernel
+constexpr int kStreamMinHeads = 128;   // calls with at least this many heads take this kernel
 
 struct StrCtl {
     int scan[kStrMaxWarps + 1];
