@@ -429,7 +429,7 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
 // memory with one quad of halo on either side, from where a lane pools four neighbouring positions.
 //   pass 1  pooled keys -> histogram of the top 11 bits (and the pooled values, when the caller wants them);
 //   pass 2  the keys that share the winning digit -> candidate list (key and position), and per warp the number of
-//           keys with a larger digit; rounds 2 and 3 run on the list, and the list then also gives every warp its
+//           keys with a larger digit (passes 2 and 3 pool only the quads whose 12 staged scores reach the threshold); rounds 2 and 3 run on the list, and the list then also gives every warp its
 //           number of kept keys.  (When the list would not fit, rounds 2 and 3 and the counts are passes of their own.)
 //   pass 3  ordered compaction of the kept positions, then the copy of the kept rows.
 // Same integer arithmetic as the cluster kernel: the same threshold key and the same ties, hence the same indices.
@@ -503,6 +503,16 @@ __device__ __forceinline__ void pooled_quad(const float4 *buf, int at, int radiu
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) key[i] = order_key(best[i]);
+}
+
+// Order key of the largest of the 12 staged scores around quad `at`: an upper bound of the quad's four pooled keys
+// (every window lies inside those 12), so a quad whose bound is below a threshold holds nothing at or above it and
+// the passes that only look for such keys skip its pooling.
+__device__ __forceinline__ uint32_t quad_bound_key(const float4 *buf, int at)
+{
+    const float4 a = buf[at], b = buf[at + 1], c = buf[at + 2];
+    const float m = max3f(max3f(a.x, a.y, a.z), max3f(a.w, b.x, b.y), max3f(max3f(b.z, b.w, c.x), max3f(c.y, c.z, c.w), -INFINITY));
+    return order_key(m);
 }
 
 // Block-wide exclusive scan of one int per thread, any number of whole warps.
@@ -654,6 +664,7 @@ select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, in
                 for (int u = 0; u < 4; ++u) {
                     const int q = base + 32 * u + lane;
                     const int nval = q < qb ? min(4, L - 4 * q) : 0;
+                    if (nval == 0 || (quad_bound_key(buf, 32 * u + lane) >> 21) < pre) continue;
                     uint32_t key[4];
                     float best[4];
                     pooled_quad(buf, 32 * u + lane, radius, key, best);
@@ -691,6 +702,7 @@ select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, in
                     for (int u = 0; u < 4; ++u) {
                         const int q = base + 32 * u + lane;
                         const int nval = q < qb ? min(4, L - 4 * q) : 0;
+                        if (nval == 0 || (quad_bound_key(buf, 32 * u + lane) >> (sh + wd)) < pre) continue;
                         uint32_t key[4], dg[4];
                         float best[4];
                         pooled_quad(buf, 32 * u + lane, radius, key, best);
@@ -724,6 +736,7 @@ select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, in
                 for (int u = 0; u < 4; ++u) {
                     const int q = base + 32 * u + lane;
                     const int nval = q < qb ? min(4, L - 4 * q) : 0;
+                    if (nval == 0 || quad_bound_key(buf, 32 * u + lane) < tau) continue;
                     uint32_t key[4];
                     float best[4];
                     pooled_quad(buf, 32 * u + lane, radius, key, best);
@@ -745,13 +758,14 @@ select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, in
             for (int u = 0; u < 4; ++u) {
                 const int q = base + 32 * u + lane;
                 const int nval = q < qb ? min(4, L - 4 * q) : 0;
-                uint32_t key[4];
+                const bool may = nval != 0 && quad_bound_key(buf, 32 * u + lane) >= tau;
+                if (!__any_sync(0xffffffffu, may)) continue;         // nothing of these 128 quads is at or above tau
+                uint32_t key[4] = {0u, 0u, 0u, 0u};
                 float best[4];
-                pooled_quad(buf, 32 * u + lane, radius, key, best);
+                if (may) pooled_quad(buf, 32 * u + lane, radius, key, best);
                 int g = 0, e = 0;
-                for (int i = 0; i < 4; ++i) if (i < nval) { g += key[i] > tau; e += key[i] == tau; }
+                for (int i = 0; i < 4; ++i) if (may && i < nval) { g += key[i] > tau; e += key[i] == tau; }
                 const int mine = g | (e << 16);
-                if (!__any_sync(0xffffffffu, mine != 0)) continue;   // nothing of these 128 positions is at or above tau
                 int inc = mine;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -761,7 +775,7 @@ select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, in
                 const int total = __shfl_sync(0xffffffffu, inc, 31);
                 int g_here = gt_before + ((inc - mine) & 0xffff), e_here = eq_before + ((inc - mine) >> 16);
                 for (int i = 0; i < 4; ++i) {
-                    if (i >= nval) continue;
+                    if (!may || i >= nval) continue;
                     if (key[i] > tau) {
                         if (JQ_IN(g_here + min(e_here, need_eq), nkeep, kDbgSelect, 28)) out[g_here + min(e_here, need_eq)] = 4 * q + i;
                         ++g_here;
