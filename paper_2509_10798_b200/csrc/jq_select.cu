@@ -425,8 +425,9 @@ select_cluster(const float *__restrict__ scores, int L, int nkeep, int radius, i
 // cluster kernel's time per head is mostly the latency of its barrier-separated phases.  Here a head is one CTA that
 // keeps a histogram, a candidate list and a small staging buffer per warp in shared memory, so that several heads are
 // resident per SM, and that walks the head's scores three times, pooling on the fly.  Every warp owns a contiguous
-// share of the head and takes it 512 positions at a time: four 16-byte reads per lane in flight, staged in shared
-// memory with one quad of halo on either side, from where a lane pools four neighbouring positions.
+// share of the head and takes it 512 positions at a time: four 16-byte asynchronous copies per lane into one of the
+// warp's two staging buffers, with one quad of halo on either side, from where a lane pools four neighbouring
+// positions while the copies of the next 512 positions are in flight.
 //   pass 1  pooled keys -> histogram of the top 11 bits (and the pooled values, when the caller wants them);
 //   pass 2  the keys that share the winning digit -> candidate list (key and position), and per warp the number of
 //           keys with a larger digit (passes 2 and 3 pool only the quads whose 12 staged scores reach the threshold); rounds 2 and 3 run on the list, and the list then also gives every warp its
@@ -461,21 +462,46 @@ __device__ __forceinline__ float4 load_quad(const float *__restrict__ s, int L, 
     return make_float4(v[0], v[1], v[2], v[3]);
 }
 
-// The warp stages quads [base - 1, base + 129) of the head in its buffer.
-__device__ __forceinline__ void stage_quads(float4 *buf, const float *__restrict__ s, int L, int base, bool vec, long long soff,
+// The warp requests quads [base - 1, base + 129) of the head into one of its two buffers: 16-byte asynchronous copies
+// for the quads that lie inside the head (and are aligned), plain stores of -inf-padded values for the others.
+__device__ __forceinline__ void stage_issue(float4 *dst, const float *__restrict__ s, int L, int base, bool vec, long long soff,
                                             const SelExtents &ext JQ_DBG_PARAM)
 {
     const int lane = threadIdx.x & 31;
-    float4 v[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) v[u] = load_quad(s, L, base + 32 * u + lane, vec, soff, ext JQ_DBG_ARG_DEV);
-    float4 h = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (lane < 2) h = load_quad(s, L, lane == 0 ? base - 1 : base + kStepQuads, vec, soff, ext JQ_DBG_ARG_DEV);
-    __syncwarp();                                            // the previous step's reads of the buffer are done
-#pragma unroll
-    for (int u = 0; u < 4; ++u) buf[1 + 32 * u + lane] = v[u];
-    if (lane < 2) buf[lane == 0 ? 0 : kStageQuads - 1] = h;
+    for (int u = 0; u < 5; ++u) {
+        if (u == 4 && lane >= 2) break;
+        const int q = u < 4 ? base + 32 * u + lane : (lane == 0 ? base - 1 : base + kStepQuads);
+        float4 *d = dst + (u < 4 ? 1 + 32 * u + lane : (lane == 0 ? 0 : kStageQuads - 1));
+        if (vec && q >= 0 && 4 * q + 4 <= L && JQ_IN(soff + 4 * q + 3, ext.scores, kDbgSelect, 22))
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(d)), "l"(s + 4 * q) : "memory");
+        else
+            *d = load_quad(s, L, q, vec, soff, ext JQ_DBG_ARG_DEV);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// The staged quads of the step at `base` of the warp's walk over [qa, qb), 128 quads per step: waits for the step's
+// copies and has the next step's under way (two buffers per warp), so that a step's reads from memory overlap the
+// pooling of the step before.  Every lane of the warp calls it once per step, in order.
+__device__ __forceinline__ const float4 *stage_step(float4 *bufs, const float *__restrict__ s, int L, int base, int qa, int qb, bool vec,
+                                                    long long soff, const SelExtents &ext JQ_DBG_PARAM)
+{
+    const int step = (base - qa) / kStepQuads;
+    float4 *cur = bufs + (step & 1) * kStageQuads, *nxt = bufs + ((step + 1) & 1) * kStageQuads;
+    if (step == 0) {
+        __syncwarp();                                        // the reads of an earlier pass are done
+        stage_issue(cur, s, L, base, vec, soff, ext JQ_DBG_ARG_DEV);
+    }
+    __syncwarp();                                            // the previous step's reads of the other buffer are done
+    if (base + kStepQuads < qb) {
+        stage_issue(nxt, s, L, base + kStepQuads, vec, soff, ext JQ_DBG_ARG_DEV);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
     __syncwarp();
+    return cur;
 }
 
 // Pooled order keys (and values) of the four positions of quad `at` (0 .. 127) of the staged step.
@@ -577,7 +603,7 @@ __device__ __forceinline__ void hist_add_runs(uint32_t *hist, const uint32_t (&d
     if (cnt && cur != 0xffffffffu && JQ_IN(cur, kBins, kDbgSelect, 24)) atomicAdd(&hist[cur], cnt);
 }
 
-// grid (Hkv), block kThreads = 512 (two CTAs to an SM) or 1024 (one); dynamic shared memory: a staging buffer of
+// grid (Hkv), block kThreads = 512 (two CTAs to an SM) or 1024 (one); dynamic shared memory: two staging buffers of
 // kStageQuads float4 per warp.  Arguments as for select_cluster.
 __host__ __device__ constexpr int stream_ctas_per_sm(int threads) { return threads == 512 ? 2 : 1; }
 template <int kThreads>
@@ -595,7 +621,7 @@ select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, in
     __shared__ StrCtl ctl;
     constexpr int T = kThreads, nw = T / 32;
     const int kv = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    float4 *buf = (float4 *)sm + wid * kStageQuads;
+    float4 *buf = (float4 *)sm + wid * 2 * kStageQuads;   // the warp's two staging buffers
     int kv_in = kv;
     long long soff = (long long)kv * L, orow = (long long)kv * nkeep, krow = (long long)kv * out_rows;
     cudaGridDependencySynchronize();   // everything above ran while the previous kernel of the stream was finishing
@@ -619,14 +645,14 @@ select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, in
     if (tid == 0) ctl.cand_count = 0;
     __syncthreads();
     for (int base = qa; base < qb; base += kStepQuads) {
-        stage_quads(buf, s, L, base, vec, soff, ext JQ_DBG_ARG_DEV);
+        const float4 *bf = stage_step(buf, s, L, base, qa, qb, vec, soff, ext JQ_DBG_ARG_DEV);
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int q = base + 32 * u + lane;
             const int nval = q < qb ? min(4, L - 4 * q) : 0;
             uint32_t key[4];
             float best[4];
-            pooled_quad(buf, 32 * u + lane, radius, key, best);
+            pooled_quad(bf, 32 * u + lane, radius, key, best);
             if (pooled && nval && JQ_IN(soff + 4 * q + nval - 1, ext.scores, kDbgSelect, 25))
                 for (int i = 0; i < nval; ++i) pooled[4 * q + i] = best[i];
             // one addition per warp when all its positions share the digit (the usual case: 128 neighbouring
@@ -659,15 +685,15 @@ select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, in
             // pass 2: the keys with the winning first digit, with their positions; the warp's keys above that digit
             int hi_cnt = 0;
             for (int base = qa; base < qb; base += kStepQuads) {
-                stage_quads(buf, s, L, base, vec, soff, ext JQ_DBG_ARG_DEV);
+                const float4 *bf = stage_step(buf, s, L, base, qa, qb, vec, soff, ext JQ_DBG_ARG_DEV);
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int q = base + 32 * u + lane;
                     const int nval = q < qb ? min(4, L - 4 * q) : 0;
-                    if (nval == 0 || (quad_bound_key(buf, 32 * u + lane) >> 21) < pre) continue;
+                    if (nval == 0 || (quad_bound_key(bf, 32 * u + lane) >> 21) < pre) continue;
                     uint32_t key[4];
                     float best[4];
-                    pooled_quad(buf, 32 * u + lane, radius, key, best);
+                    pooled_quad(bf, 32 * u + lane, radius, key, best);
                     int nhit = 0;
                     for (int i = 0; i < 4; ++i) if (i < nval) { nhit += (key[i] >> 21) == pre; hi_cnt += (key[i] >> 21) > pre; }
                     if (nhit) {
@@ -697,15 +723,15 @@ select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, in
                 }
             } else {
                 for (int base = qa; base < qb; base += kStepQuads) {
-                    stage_quads(buf, s, L, base, vec, soff, ext JQ_DBG_ARG_DEV);
+                    const float4 *bf = stage_step(buf, s, L, base, qa, qb, vec, soff, ext JQ_DBG_ARG_DEV);
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const int q = base + 32 * u + lane;
                         const int nval = q < qb ? min(4, L - 4 * q) : 0;
-                        if (nval == 0 || (quad_bound_key(buf, 32 * u + lane) >> (sh + wd)) < pre) continue;
+                        if (nval == 0 || (quad_bound_key(bf, 32 * u + lane) >> (sh + wd)) < pre) continue;
                         uint32_t key[4], dg[4];
                         float best[4];
-                        pooled_quad(buf, 32 * u + lane, radius, key, best);
+                        pooled_quad(bf, 32 * u + lane, radius, key, best);
                         for (int i = 0; i < 4; ++i) dg[i] = (key[i] >> (sh + wd)) == pre ? ((key[i] >> sh) & mask) : 0xffffffffu;
                         hist_add_runs(hist, dg, nval JQ_DBG_ARG_DEV);
                     }
@@ -731,15 +757,15 @@ select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, in
         } else {
             int cgt = 0, ceq = 0;
             for (int base = qa; base < qb; base += kStepQuads) {
-                stage_quads(buf, s, L, base, vec, soff, ext JQ_DBG_ARG_DEV);
+                const float4 *bf = stage_step(buf, s, L, base, qa, qb, vec, soff, ext JQ_DBG_ARG_DEV);
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int q = base + 32 * u + lane;
                     const int nval = q < qb ? min(4, L - 4 * q) : 0;
-                    if (nval == 0 || quad_bound_key(buf, 32 * u + lane) < tau) continue;
+                    if (nval == 0 || quad_bound_key(bf, 32 * u + lane) < tau) continue;
                     uint32_t key[4];
                     float best[4];
-                    pooled_quad(buf, 32 * u + lane, radius, key, best);
+                    pooled_quad(bf, 32 * u + lane, radius, key, best);
                     for (int i = 0; i < 4; ++i) if (i < nval) { cgt += key[i] > tau; ceq += key[i] == tau; }
                 }
             }
@@ -753,16 +779,16 @@ select_stream(const float *__restrict__ scores, int L, int nkeep, int radius, in
 
         // ---- pass 3: ordered compaction (position order = warp, step, quad, position within the quad)
         for (int base = qa; base < qb; base += kStepQuads) {
-            stage_quads(buf, s, L, base, vec, soff, ext JQ_DBG_ARG_DEV);
+            const float4 *bf = stage_step(buf, s, L, base, qa, qb, vec, soff, ext JQ_DBG_ARG_DEV);
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int q = base + 32 * u + lane;
                 const int nval = q < qb ? min(4, L - 4 * q) : 0;
-                const bool may = nval != 0 && quad_bound_key(buf, 32 * u + lane) >= tau;
+                const bool may = nval != 0 && quad_bound_key(bf, 32 * u + lane) >= tau;
                 if (!__any_sync(0xffffffffu, may)) continue;         // nothing of these 128 quads is at or above tau
                 uint32_t key[4] = {0u, 0u, 0u, 0u};
                 float best[4];
-                if (may) pooled_quad(buf, 32 * u + lane, radius, key, best);
+                if (may) pooled_quad(bf, 32 * u + lane, radius, key, best);
                 int g = 0, e = 0;
                 for (int i = 0; i < 4; ++i) if (may && i < nval) { g += key[i] > tau; e += key[i] == tau; }
                 const int mine = g | (e << 16);
@@ -902,7 +928,7 @@ jq_status launch_select_stream(const float *scores, const jq_shape &s, int nkeep
     const long long resident = (long long)sms * stream_ctas_per_sm(512), inflight = s.Hkv < resident ? s.Hkv : resident;
     const int threads = inflight * Lmax * 4 <= (96ll << 20) ? 512 : 1024;
     const auto kernel = threads == 512 ? select_stream<512> : select_stream<1024>;
-    const size_t dyn = (size_t)(threads / 32) * kStageQuads * sizeof(float4);
+    const size_t dyn = (size_t)(threads / 32) * 2 * kStageQuads * sizeof(float4);
     static bool attr_done[64][2] = {};
     const int which = threads == 512 ? 0 : 1;
     if (dev < 0 || dev >= 64) return JQ_ERR_CUDA;
